@@ -1,0 +1,220 @@
+/* asyncflow.h -- C ABI of the B200 (sm_100a) scoring path for streaming GRPO post-training.
+ *
+ * The library implements the device-side hot path shared by the actor-inference,
+ * reference-inference and actor-update tasks of AsyncFlow (arXiv 2507.01663): micro-batches of
+ * variable-length responses are gathered from a sample-indexed columnar store, scored by the LM
+ * head with a fused online log-softmax, and reduced to the clipped GRPO policy loss (forward and
+ * backward).  The paper fixes the data flow; it prints no formula for the numerics, which are
+ * the textbook definitions stated with each entry point below.
+ *
+ * Conventions
+ *   - "dev" pointers are device pointers on the context's device, "host" pointers are host
+ *     pointers.  All buffers are owned by the caller; the library owns only its context and
+ *     the workspace inside it.
+ *   - Every call enqueues its kernels on `stream` (a cudaStream_t passed as void*; NULL is the
+ *     legacy default stream) and returns without synchronising, unless noted.
+ *   - The return code reports what the host can see (null pointers, sizes, alignment, capacity,
+ *     index lists, CUDA launch errors).  Conditions only the device can see (a target id outside
+ *     [0, V), a watchdog expiry inside a kernel) set bits of a sticky device error word that
+ *     af_check_device_errors reads; affected outputs are NaN; no kernel traps.
+ *   - A context serves one stream at a time: calls on one context must not overlap on the GPU
+ *     (they share its workspace).  Use one context per concurrent stream.
+ *   - Workspace grows on demand with cudaMalloc (which may synchronise).  Call af_reserve once
+ *     with the largest sizes to keep allocation out of the hot calls.
+ *   - Only compute capability 10.0 devices are accepted.  There is no CPU path.
+ */
+#ifndef ASYNCFLOW_H_
+#define ASYNCFLOW_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct af_ctx af_ctx;
+
+typedef enum {
+  AF_OK = 0,
+  AF_ERR_INVALID_ARG = -1,        /* null pointer, negative size, bad enum value            */
+  AF_ERR_SHAPE = -2,              /* size outside what the kernels support (see each call)   */
+  AF_ERR_ALIGNMENT = -3,          /* pointer or row pitch not 16-byte aligned                */
+  AF_ERR_CAPACITY = -4,           /* caller's output buffers too small                       */
+  AF_ERR_INDEX = -5,              /* sample index outside [0, N)                             */
+  AF_ERR_WORKSPACE = -6,          /* workspace allocation failed                             */
+  AF_ERR_CUDA = -7,               /* a CUDA runtime / driver call failed                     */
+  AF_ERR_UNSUPPORTED_DEVICE = -8, /* device is not compute capability 10.0                   */
+  AF_ERR_DEVICE_FLAGGED = -9      /* af_check_device_errors found the error word non-zero    */
+} af_status;
+
+/* bits of the device error word */
+#define AF_DEVERR_TARGET_RANGE 1u /* a target id was outside [0, V): that token's outputs are NaN */
+#define AF_DEVERR_WATCHDOG 2u     /* a bounded wait inside a kernel ran out; results invalid      */
+#define AF_DEVERR_CU_SEQLENS 4u   /* cu_seqlens not non-decreasing from 0 to T                     */
+
+/* Create / destroy a context on CUDA device `device`.  af_create fails with
+ * AF_ERR_UNSUPPORTED_DEVICE unless the device is compute capability 10.0.  af_destroy
+ * synchronises the device and frees the workspace. */
+af_status af_create(af_ctx** out, int device);
+af_status af_destroy(af_ctx* ctx);
+const char* af_status_string(af_status s);
+
+/* Pre-size the workspace for micro-batches of up to max_T tokens and max_B sequences at head
+ * shape (d, V).  with_backward != 0 also reserves the scratch of af_policy_loss_backward.
+ * Synchronous (allocates). */
+af_status af_reserve(af_ctx* ctx, int64_t max_T, int32_t max_B, int32_t d, int32_t V,
+                     int32_t with_backward);
+
+/* Bytes of device workspace currently held by the context. */
+int64_t af_workspace_bytes(const af_ctx* ctx);
+
+/* Tuning knobs of the fused LM-head kernels (0 keeps the default): `v_splits` = number of
+ * vocabulary ranges one token tile is split into across CTAs; `bwd_token_block` = tokens per
+ * backward block (scratch is proportional to it). */
+af_status af_set_tuning(af_ctx* ctx, int32_t v_splits, int32_t bwd_token_block);
+
+/* Synchronise `stream`, read and clear the sticky device error word.  Returns AF_OK when it was
+ * zero, else AF_ERR_DEVICE_FLAGGED with the bits in *flags (nullable). */
+af_status af_check_device_errors(af_ctx* ctx, uint32_t* flags, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * af_pack_microbatch -- sample-index list -> cu_seqlens-packed tensors.
+ *
+ * The store is the paper's 2-D columnar structure restricted to one device (Section 4.3 "Data
+ * Plane"): rows are samples addressed by a global index, columns are task-specific components,
+ * and a task reads only the columns it asks for (NULL = not requested).  The index list is the
+ * metadata a controller hands out; the worker on the device fetches the data (Section 4.2
+ * "Interaction Interface").  Sample i owns token rows tok_offset[i] .. tok_offset[i+1]-1 of every
+ * per-token column.
+ *
+ * For j in [0, B): cu_seqlens[j+1] = cu_seqlens[j] + len(idx[j]); the rows of sample idx[j] are
+ * copied, bit for bit, to packed rows cu_seqlens[j] .. cu_seqlens[j+1]-1 of each requested
+ * column; adv_seq[j] = adv[idx[j]]; seq_id[t] = j.  Duplicate indices are gathered twice.
+ *
+ * Errors: AF_ERR_INDEX for an index outside [0, N); AF_ERR_CAPACITY if T or B exceed the output
+ * capacities or T >= 2^31; AF_ERR_ALIGNMENT unless d % 8 == 0 and hidden pointers are 16-byte
+ * aligned.  *T_out (host) receives the packed token count before the call returns.  B == 0 is
+ * valid and writes cu_seqlens[0] = 0 only.
+ * ------------------------------------------------------------------------------------------- */
+typedef struct {
+  int64_t n_samples;               /* N                                                       */
+  int32_t d;                       /* hidden size (elements per token row)                    */
+  int32_t reserved;
+  const int64_t* tok_offset_host;  /* [N+1] host: lets the host size the batch without a sync */
+  const void* hidden;              /* [sum L, d] bf16, dev, row-major                         */
+  const int32_t* target;           /* [sum L] dev, or NULL                                    */
+  const float* old_logp;           /* [sum L] dev, or NULL                                    */
+  const float* ref_logp;           /* [sum L] dev, or NULL                                    */
+  const float* adv;                /* [N] dev, or NULL                                        */
+} af_store_view;
+
+typedef struct {
+  int64_t token_capacity;          /* rows available in the per-token outputs                 */
+  int32_t seq_capacity;            /* cu_seqlens holds seq_capacity + 1 entries               */
+  int32_t reserved;
+  int32_t* cu_seqlens;             /* [B+1] dev (required)                                    */
+  void* hidden;                    /* [T, d] bf16 dev, or NULL iff store.hidden is NULL       */
+  int32_t* target;                 /* [T] dev, NULL iff store.target is NULL                  */
+  float* old_logp;                 /* [T] dev, NULL iff store.old_logp is NULL                */
+  float* ref_logp;                 /* [T] dev, NULL iff store.ref_logp is NULL                */
+  float* adv_seq;                  /* [B] dev, NULL iff store.adv is NULL                     */
+  int32_t* seq_id;                 /* [T] dev, or NULL                                        */
+} af_packed;
+
+af_status af_pack_microbatch(af_ctx* ctx, const af_store_view* store, const int32_t* idx_host,
+                             int32_t B, const af_packed* out, int64_t* T_out, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * af_token_logprob -- LM-head projection fused with an online log-softmax (the last stage of
+ * the `compute_log_prob` task of the paper's backend interface, Appendix "Backend-level
+ * interface"; forward-only for reference / actor inference, Section 6.4).
+ *
+ * For each token t:  z_tv = sum_k hidden[t,k] * W[v,k]  (bf16 x bf16, fp32 accumulation; the
+ * [T,V] logits are never written to memory);  lse_t = log sum_v exp z_tv;
+ * logp_t = z_{t,target[t]} - lse_t;  entropy_t = lse_t - sum_v softmax_tv * z_tv.
+ *
+ * hidden [T,d] bf16 dev, W [V,d] bf16 dev (one row per vocabulary id), both row-major and
+ * 16-byte aligned, d % 8 == 0, 1 <= d, 1 <= V, 0 <= T < 2^31.  logp (required), entropy and lse
+ * (nullable) are [T] fp32 dev.  A target outside [0,V) yields NaN logp and AF_DEVERR_TARGET_RANGE.
+ * ------------------------------------------------------------------------------------------- */
+af_status af_token_logprob(af_ctx* ctx, const void* hidden, const void* W, const int32_t* target,
+                           int64_t T, int32_t d, int32_t V, float* logp, float* entropy,
+                           float* lse, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * af_grpo_advantage -- group-normalised advantages: "rewards normalized within a group of
+ * responses to the same prompt" (paper Section 6.1 "RL algorithms"; no critic).
+ *
+ * For each group g with members I_g (n_g = |I_g|):  mu = mean r;  sigma = sqrt(sum (r-mu)^2 /
+ * (n_g - ddof));  adv_i = (r_i - mu) / (sigma + eps_adv).  A group of equal rewards gets zeros.
+ *
+ * reward [N] fp32 dev.  group_id [N] int32 dev with values in [0, n_groups) in any order, or
+ * NULL for contiguous equal groups (sample i belongs to group i / (N / n_groups); then
+ * N % n_groups must be 0).  With group_id given the kernel scans the id array once per group
+ * (deterministic, no float atomics) and N * n_groups must stay below 2^33 (AF_ERR_SHAPE).
+ * ddof is 0 or 1.  adv [N] fp32 dev.
+ * ------------------------------------------------------------------------------------------- */
+af_status af_grpo_advantage(af_ctx* ctx, const float* reward, const int32_t* group_id, int64_t N,
+                            int32_t n_groups, float eps_adv, int32_t ddof, float* adv,
+                            void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * af_policy_loss -- clipped-ratio GRPO policy loss with a k3 KL penalty against the reference
+ * log-probs (the loss of the paper's actor-update task, Section 6.4; GRPO, Section 6.1).
+ *
+ * Token t of sequence i, A = adv_seq[i]:
+ *   rho = exp(logp - old);  pg = -min(rho*A, clip(rho, 1-clip_lo, 1+clip_hi)*A);
+ *   delta = ref - logp;  k3 = exp(delta) - delta - 1;  l = pg + kl_coef*k3.
+ *   A token counts as clipped iff clip(rho)*A < rho*A (strict).
+ * agg_mode 0: loss = loss_scale * mean_i( mean_{t in i} l_t ); agg_mode 1: loss_scale * mean_t l_t.
+ * pg_loss and kl_mean aggregate pg and k3 the same way; clip_frac = #clipped / T;
+ * entropy_mean = sum entropy / T (0 if entropy is NULL).
+ * dlogp[t] = w_t * ( clipped ? 0 : -A*rho ) + w_t * kl_coef * (1 - exp(delta)), w_t the weight of
+ * token t in the aggregation (loss_scale/(B*L_i) or loss_scale/T).  Entropy carries no gradient.
+ *
+ * logp, old_logp, ref_logp, entropy (nullable), dlogp (nullable): [T] fp32 dev; adv_seq [B] fp32
+ * dev; cu_seqlens [B+1] int32 dev, non-decreasing, cu_seqlens[0] = 0, cu_seqlens[B] = T.
+ * `out` is a device struct, valid when the stream reaches the end of the call.  Sums are taken
+ * in a fixed order: results are bit-reproducible from run to run.
+ * ------------------------------------------------------------------------------------------- */
+typedef struct {
+  float clip_lo, clip_hi;
+  float kl_coef;
+  int32_t agg_mode;
+  float loss_scale;
+} af_loss_params;
+
+typedef struct {
+  float loss, pg_loss, kl_mean, clip_frac, entropy_mean;
+  int32_t reserved;
+  int64_t n_tokens;
+} af_loss_out;
+
+af_status af_policy_loss(af_ctx* ctx, const float* logp, const float* old_logp,
+                         const float* ref_logp, const float* entropy, const float* adv_seq,
+                         const int32_t* cu_seqlens, int32_t B, int64_t T,
+                         const af_loss_params* params, af_loss_out* out, float* dlogp,
+                         void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * af_policy_loss_backward -- gradient of the loss through log-softmax and the LM head (the
+ * forward-backward actor-update task, paper Section 6.4), without materialising [T,V].
+ *
+ *   dZ_tv = dlogp[t] * ( 1{v == target[t]} - exp(z_tv - lse[t]) )      (z recomputed per block)
+ *   d_hidden[t,:] = sum_v dZ_tv * W[v,:]          -> [T,d] bf16
+ *   d_W[v,:]      = sum_t dZ_tv * hidden[t,:]     -> [V,d] fp32 (added to d_W if accumulate_dW)
+ *
+ * dZ is rounded to bf16 for the two tensor-core products (fp32 accumulation).  Tokens are
+ * processed in blocks; the scratch (dZ of one block, transposed copies of W and hidden) lives
+ * in the context's workspace and does not grow with T beyond the hidden copy.
+ * Requirements: d % 8 == 0, V % 8 == 0, 16-byte aligned pointers, 0 <= T < 2^31.
+ * ------------------------------------------------------------------------------------------- */
+af_status af_policy_loss_backward(af_ctx* ctx, const void* hidden, const void* W,
+                                  const int32_t* target, const float* lse, const float* dlogp,
+                                  int64_t T, int32_t d, int32_t V, void* d_hidden, float* d_W,
+                                  int32_t accumulate_dW, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ASYNCFLOW_H_ */

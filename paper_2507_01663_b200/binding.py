@@ -1,0 +1,220 @@
+"""Thin ctypes binding of ``libasyncflow.so`` -- argument marshalling only.
+
+Each function mirrors the C entry point of the same name in ``include/asyncflow.h``.  Tensors
+are torch CUDA tensors used as plain device buffers (``data_ptr()``); streams are torch streams.
+There is no CPU path: importing this module without the built library, or calling it without a
+B200, raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libasyncflow.so")
+
+AF_OK = 0
+STATUS_NAMES = {0: "AF_OK", -1: "AF_ERR_INVALID_ARG", -2: "AF_ERR_SHAPE", -3: "AF_ERR_ALIGNMENT",
+                -4: "AF_ERR_CAPACITY", -5: "AF_ERR_INDEX", -6: "AF_ERR_WORKSPACE", -7: "AF_ERR_CUDA",
+                -8: "AF_ERR_UNSUPPORTED_DEVICE", -9: "AF_ERR_DEVICE_FLAGGED"}
+DEVERR_TARGET_RANGE, DEVERR_WATCHDOG, DEVERR_CU_SEQLENS = 1, 2, 4
+
+EXPORTS = ["af_create", "af_destroy", "af_status_string", "af_reserve", "af_workspace_bytes",
+           "af_set_tuning", "af_check_device_errors", "af_pack_microbatch", "af_token_logprob",
+           "af_grpo_advantage", "af_policy_loss", "af_policy_loss_backward"]
+
+
+class AfError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {STATUS_NAMES.get(status, status)}")
+
+
+class StoreView(C.Structure):
+    _fields_ = [("n_samples", C.c_int64), ("d", C.c_int32), ("reserved", C.c_int32),
+                ("tok_offset_host", C.c_void_p), ("hidden", C.c_void_p), ("target", C.c_void_p),
+                ("old_logp", C.c_void_p), ("ref_logp", C.c_void_p), ("adv", C.c_void_p)]
+
+
+class Packed(C.Structure):
+    _fields_ = [("token_capacity", C.c_int64), ("seq_capacity", C.c_int32), ("reserved", C.c_int32),
+                ("cu_seqlens", C.c_void_p), ("hidden", C.c_void_p), ("target", C.c_void_p),
+                ("old_logp", C.c_void_p), ("ref_logp", C.c_void_p), ("adv_seq", C.c_void_p),
+                ("seq_id", C.c_void_p)]
+
+
+class LossParams(C.Structure):
+    _fields_ = [("clip_lo", C.c_float), ("clip_hi", C.c_float), ("kl_coef", C.c_float),
+                ("agg_mode", C.c_int32), ("loss_scale", C.c_float)]
+
+
+class LossOut(C.Structure):
+    _fields_ = [("loss", C.c_float), ("pg_loss", C.c_float), ("kl_mean", C.c_float),
+                ("clip_frac", C.c_float), ("entropy_mean", C.c_float), ("reserved", C.c_int32),
+                ("n_tokens", C.c_int64)]
+
+
+_lib = None
+
+
+def load_library() -> C.CDLL:
+    """dlopen the in-tree library; fail loudly if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2507_01663_b200.build` "
+                          "(there is no fallback implementation)")
+    lib = C.CDLL(LIB_PATH)
+    vp, i32, i64, f32 = C.c_void_p, C.c_int32, C.c_int64, C.c_float
+    lib.af_create.argtypes = [C.POINTER(vp), C.c_int]
+    lib.af_destroy.argtypes = [vp]
+    lib.af_status_string.argtypes = [C.c_int]
+    lib.af_status_string.restype = C.c_char_p
+    lib.af_reserve.argtypes = [vp, i64, i32, i32, i32, i32]
+    lib.af_workspace_bytes.argtypes = [vp]
+    lib.af_workspace_bytes.restype = i64
+    lib.af_set_tuning.argtypes = [vp, i32, i32]
+    lib.af_check_device_errors.argtypes = [vp, C.POINTER(C.c_uint32), vp]
+    lib.af_pack_microbatch.argtypes = [vp, C.POINTER(StoreView), vp, i32, C.POINTER(Packed),
+                                       C.POINTER(i64), vp]
+    lib.af_token_logprob.argtypes = [vp, vp, vp, vp, i64, i32, i32, vp, vp, vp, vp]
+    lib.af_grpo_advantage.argtypes = [vp, vp, vp, i64, i32, f32, i32, vp, vp]
+    lib.af_policy_loss.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i64, C.POINTER(LossParams), vp,
+                                   vp, vp]
+    lib.af_policy_loss_backward.argtypes = [vp, vp, vp, vp, vp, vp, i64, i32, i32, vp, vp, i32, vp]
+    for name in EXPORTS:
+        if name not in ("af_status_string", "af_workspace_bytes"):
+            getattr(lib, name).restype = C.c_int
+    _lib = lib
+    return lib
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("device buffers must be contiguous CUDA tensors")
+    return C.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> C.c_void_p:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return C.c_void_p(s.cuda_stream)
+
+
+def _check(status: int, where: str):
+    if status != AF_OK:
+        raise AfError(status, where)
+
+
+class Context:
+    """Owner of an ``af_ctx`` (workspace + device error word) on one CUDA device."""
+
+    def __init__(self, device: int = 0):
+        self.lib = load_library()
+        self.device = device
+        h = C.c_void_p()
+        _check(self.lib.af_create(C.byref(h), device), "af_create")
+        self.handle = h
+
+    def close(self):
+        if getattr(self, "handle", None):
+            self.lib.af_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- housekeeping ------------------------------------------------------------------------
+    def reserve(self, max_T: int, max_B: int, d: int, V: int, with_backward: bool = False):
+        _check(self.lib.af_reserve(self.handle, max_T, max_B, d, V, int(with_backward)), "af_reserve")
+
+    def workspace_bytes(self) -> int:
+        return int(self.lib.af_workspace_bytes(self.handle))
+
+    def set_tuning(self, v_splits: int = 0, bwd_token_block: int = 0):
+        _check(self.lib.af_set_tuning(self.handle, v_splits, bwd_token_block), "af_set_tuning")
+
+    def check_device_errors(self, stream=None) -> int:
+        """Synchronise the stream; return the device error bits (0 = none) and clear them."""
+        flags = C.c_uint32(0)
+        st = self.lib.af_check_device_errors(self.handle, C.byref(flags), _stream(stream))
+        if st not in (AF_OK, -9):
+            raise AfError(st, "af_check_device_errors")
+        return int(flags.value)
+
+    # -- the five entry points ---------------------------------------------------------------
+    def pack_microbatch(self, store: dict, idx_host: np.ndarray, out: dict, stream=None) -> int:
+        """``store``: tok_offset_host (np.int64 [N+1]), d, and device columns hidden / target /
+        old_logp / ref_logp / adv (missing or None = not requested).  ``out``: device buffers
+        cu_seqlens, hidden, target, old_logp, ref_logp, adv_seq, seq_id.  Returns T."""
+        off = np.ascontiguousarray(store["tok_offset_host"], dtype=np.int64)
+        idx = np.ascontiguousarray(idx_host, dtype=np.int32)
+        sv = StoreView(n_samples=off.shape[0] - 1, d=int(store["d"]), reserved=0,
+                       tok_offset_host=off.ctypes.data, hidden=_ptr(store.get("hidden")),
+                       target=_ptr(store.get("target")), old_logp=_ptr(store.get("old_logp")),
+                       ref_logp=_ptr(store.get("ref_logp")), adv=_ptr(store.get("adv")))
+        cu = out["cu_seqlens"]
+        cap_t = min([out[k].shape[0] for k in ("hidden", "target", "old_logp", "ref_logp", "seq_id")
+                     if out.get(k) is not None] or [0])
+        pk = Packed(token_capacity=cap_t, seq_capacity=cu.shape[0] - 1, reserved=0, cu_seqlens=_ptr(cu),
+                    hidden=_ptr(out.get("hidden")), target=_ptr(out.get("target")),
+                    old_logp=_ptr(out.get("old_logp")), ref_logp=_ptr(out.get("ref_logp")),
+                    adv_seq=_ptr(out.get("adv_seq")), seq_id=_ptr(out.get("seq_id")))
+        T = C.c_int64(0)
+        st = self.lib.af_pack_microbatch(self.handle, C.byref(sv), C.c_void_p(idx.ctypes.data),
+                                         idx.shape[0], C.byref(pk), C.byref(T), _stream(stream))
+        _check(st, "af_pack_microbatch")
+        return int(T.value)
+
+    def token_logprob(self, hidden, W, target, logp, entropy=None, lse=None, T=None, stream=None):
+        T = hidden.shape[0] if T is None else T
+        d, V = W.shape[1], W.shape[0]
+        _check(self.lib.af_token_logprob(self.handle, _ptr(hidden), _ptr(W), _ptr(target), T, d, V,
+                                         _ptr(logp), _ptr(entropy), _ptr(lse), _stream(stream)),
+               "af_token_logprob")
+
+    def grpo_advantage(self, reward, group_id, n_groups, adv, eps_adv=1e-6, ddof=0, N=None, stream=None):
+        N = reward.shape[0] if N is None else N
+        _check(self.lib.af_grpo_advantage(self.handle, _ptr(reward), _ptr(group_id), N, n_groups,
+                                          eps_adv, ddof, _ptr(adv), _stream(stream)), "af_grpo_advantage")
+
+    def policy_loss(self, logp, old_logp, ref_logp, adv_seq, cu_seqlens, out, dlogp=None, entropy=None,
+                    clip_lo=0.2, clip_hi=0.2, kl_coef=0.04, agg_mode=0, loss_scale=1.0, B=None, T=None,
+                    stream=None):
+        """``out``: device uint8 tensor of ``ctypes.sizeof(LossOut)`` bytes (see read_loss_out)."""
+        B = cu_seqlens.shape[0] - 1 if B is None else B
+        T = logp.shape[0] if T is None else T
+        prm = LossParams(clip_lo, clip_hi, kl_coef, agg_mode, loss_scale)
+        _check(self.lib.af_policy_loss(self.handle, _ptr(logp), _ptr(old_logp), _ptr(ref_logp),
+                                       _ptr(entropy), _ptr(adv_seq), _ptr(cu_seqlens), B, T,
+                                       C.byref(prm), _ptr(out), _ptr(dlogp), _stream(stream)),
+               "af_policy_loss")
+
+    def policy_loss_backward(self, hidden, W, target, lse, dlogp, d_hidden, d_W, accumulate_dW=False,
+                             T=None, stream=None):
+        T = hidden.shape[0] if T is None else T
+        d, V = W.shape[1], W.shape[0]
+        _check(self.lib.af_policy_loss_backward(self.handle, _ptr(hidden), _ptr(W), _ptr(target),
+                                                _ptr(lse), _ptr(dlogp), T, d, V, _ptr(d_hidden),
+                                                _ptr(d_W), int(accumulate_dW), _stream(stream)),
+               "af_policy_loss_backward")
+
+
+def new_loss_out(device) -> torch.Tensor:
+    return torch.zeros(C.sizeof(LossOut), dtype=torch.uint8, device=device)
+
+
+def read_loss_out(buf: torch.Tensor) -> dict:
+    """Copy the device ``af_loss_out`` to the host (synchronises) and return it as a dict."""
+    raw = buf.cpu().numpy().tobytes()
+    o = LossOut.from_buffer_copy(raw)
+    return {k: getattr(o, k) for k, _ in LossOut._fields_ if k != "reserved"}

@@ -1,0 +1,157 @@
+// af_grpo_advantage kernels: adv_i = (r_i - mean_g) / (std_g + eps) within each prompt's group.
+//
+// Contiguous groups (group_id == NULL): a block stages a run of whole groups in shared memory
+// with 128-bit loads, reduces each group with warp shuffles (two passes: mean, then squared
+// deviations), and writes the advantages back coalesced -- 4 B read + 4 B written per sample.
+// Arbitrary membership (group_id given): one block per group scans the id array; sums are taken
+// in a fixed thread/iteration order, so the result is reproducible without float atomics.
+#include "common.cuh"
+
+namespace af {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kStage = 4096;             // samples staged per block iteration (16 KB)
+constexpr int kMaxGroupsStaged = 1024;   // groups per block iteration
+
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// Sum over `team` consecutive lanes (team a power of two <= 32).
+__device__ __forceinline__ double team_sum(double v, int team) {
+  for (int o = team >> 1; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// Statistics are accumulated in fp64: a group of equal, non-dyadic rewards must come out with
+// deviations ~1e-17 (as in exact arithmetic: zero), not ~1e-8, because they are divided by eps.
+__device__ __forceinline__ double inv_scale(double ssq, int64_t n, int ddof, float eps) {
+  const int64_t denom = n - ddof;
+  const double sigma = denom > 0 ? sqrt(ssq / (double)denom) : 0.0;
+  return 1.0 / (sigma + (double)eps);
+}
+
+// Groups of equal size G, G <= kStage: each block iteration owns `gpb` whole groups.
+__global__ void __launch_bounds__(kThreads) advantage_contiguous_kernel(
+    const float* __restrict__ reward, float* __restrict__ adv, int64_t n_groups, int G, int gpb,
+    float eps, int ddof) {
+  __shared__ __align__(16) float sr[kStage];
+  __shared__ double s_mu[kMaxGroupsStaged];   // per staged group
+  __shared__ double s_inv[kMaxGroupsStaged];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  // team of lanes per group: smallest power of two >= G, capped at a warp
+  int team = 1;
+  while (team < G && team < 32) team <<= 1;
+  const int teams_per_warp = 32 / team;
+  const int64_t n_iter = (n_groups + gpb - 1) / gpb;
+  for (int64_t it = blockIdx.x; it < n_iter; it += gridDim.x) {
+    const int64_t g0 = it * gpb;
+    const int ng = (int)((n_groups - g0) < gpb ? (n_groups - g0) : gpb);
+    const int64_t base = g0 * G;
+    const int cnt = ng * G;
+    // stage: vector loads when the run is 16-byte aligned
+    if (((base & 3) == 0) && ((reinterpret_cast<uintptr_t>(reward) & 15) == 0)) {
+      const float4* r4 = reinterpret_cast<const float4*>(reward + base);
+      for (int i = threadIdx.x; i < (cnt >> 2); i += kThreads)
+        reinterpret_cast<float4*>(sr)[i] = __ldg(r4 + i);
+      for (int i = (cnt & ~3) + threadIdx.x; i < cnt; i += kThreads) sr[i] = __ldg(reward + base + i);
+    } else {
+      for (int i = threadIdx.x; i < cnt; i += kThreads) sr[i] = __ldg(reward + base + i);
+    }
+    __syncthreads();
+    if (G == 1) {
+      for (int i = threadIdx.x; i < cnt; i += kThreads) adv[base + i] = 0.f;  // (r - r) / (0 + eps)
+      __syncthreads();
+      continue;
+    }
+    // statistics: one team of lanes per group
+    const int teams = (kThreads / 32) * teams_per_warp;
+    for (int gl = warp * teams_per_warp + lane / team; gl - (lane / team) < ng; gl += teams) {
+      // all lanes of the warp iterate together; lanes of a team past the end idle with zeros
+      const bool live = gl < ng;
+      const int tl = lane % team;
+      double s = 0.0;
+      if (live) for (int k = tl; k < G; k += team) s += (double)sr[gl * G + k];
+      s = team_sum(s, team);
+      const double mu = s / (double)G;
+      double q = 0.0;
+      if (live) for (int k = tl; k < G; k += team) { const double dv = (double)sr[gl * G + k] - mu; q += dv * dv; }
+      q = team_sum(q, team);
+      if (live && tl == 0) { s_mu[gl] = mu; s_inv[gl] = inv_scale(q, G, ddof, eps); }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < cnt; i += kThreads) {
+      const int gl = i / G;
+      adv[base + i] = (float)(((double)sr[i] - s_mu[gl]) * s_inv[gl]);
+    }
+    __syncthreads();
+  }
+}
+
+__device__ double block_sum(double v, double* scratch) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  v = warp_sum(v);
+  __syncthreads();
+  if (lane == 0) scratch[warp] = v;
+  __syncthreads();
+  double t = 0.0;
+  for (int w = 0; w < kThreads / 32; ++w) t += scratch[w];  // fixed order, same in every thread
+  return t;
+}
+
+// One block per group: members are where group_id == g (or the contiguous range when ids is NULL
+// and the group is too large to stage).
+__global__ void __launch_bounds__(kThreads) advantage_scan_kernel(
+    const float* __restrict__ reward, const int32_t* __restrict__ ids, float* __restrict__ adv,
+    int64_t N, int64_t G_contig, float eps, int ddof) {
+  __shared__ double scratch[kThreads / 32];
+  const int g = blockIdx.x;
+  const int64_t lo = ids ? 0 : (int64_t)g * G_contig;
+  const int64_t hi = ids ? N : lo + G_contig;
+  double s = 0.0, c = 0.0;
+  for (int64_t i = lo + threadIdx.x; i < hi; i += kThreads)
+    if (!ids || __ldg(ids + i) == g) { s += (double)__ldg(reward + i); c += 1.0; }
+  const double n = block_sum(c, scratch);
+  const double tot = block_sum(s, scratch);
+  if (n == 0.0) return;
+  const double mu = tot / n;
+  double q = 0.0;
+  for (int64_t i = lo + threadIdx.x; i < hi; i += kThreads)
+    if (!ids || __ldg(ids + i) == g) { const double dv = (double)__ldg(reward + i) - mu; q += dv * dv; }
+  const double ssq = block_sum(q, scratch);
+  const double inv = inv_scale(ssq, (int64_t)n, ddof, eps);
+  for (int64_t i = lo + threadIdx.x; i < hi; i += kThreads)
+    if (!ids || __ldg(ids + i) == g) adv[i] = (float)(((double)__ldg(reward + i) - mu) * inv);
+}
+
+}  // namespace
+
+cudaError_t launch_advantage(const float* reward, const int32_t* group_id, int64_t N,
+                             int32_t n_groups, float eps_adv, int32_t ddof, float* adv,
+                             int sm_count, cudaStream_t s) {
+  if (N == 0 || n_groups == 0) return cudaSuccess;
+  if (group_id == nullptr) {
+    const int64_t G = N / n_groups;
+    if (G <= kStage && G >= 1) {
+      int gpb = (int)(kStage / G);
+      // keep every SM busy before making block iterations large
+      const int64_t want = (n_groups + (int64_t)sm_count * 4 - 1) / ((int64_t)sm_count * 4);
+      if (gpb > want) gpb = (int)(want > 0 ? want : 1);
+      if (gpb > kMaxGroupsStaged) gpb = kMaxGroupsStaged;
+      int64_t iters = (n_groups + gpb - 1) / gpb;
+      int blocks = (int)(iters < (int64_t)sm_count * 8 ? iters : (int64_t)sm_count * 8);
+      advantage_contiguous_kernel<<<blocks, kThreads, 0, s>>>(reward, adv, n_groups, (int)G, gpb,
+                                                              eps_adv, ddof);
+    } else {
+      advantage_scan_kernel<<<n_groups, kThreads, 0, s>>>(reward, nullptr, adv, N, G, eps_adv, ddof);
+    }
+  } else {
+    advantage_scan_kernel<<<n_groups, kThreads, 0, s>>>(reward, group_id, adv, N, 0, eps_adv, ddof);
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace af

@@ -1,0 +1,298 @@
+// C ABI of the asyncflow library: argument validation, context and workspace management,
+// tensor-map encoding.  All arithmetic lives in the kernels of the other translation units.
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "common.cuh"
+
+namespace af {
+
+af_status ws_grow(Buf& b, size_t bytes) {
+  if (bytes <= b.cap) return AF_OK;
+  if (b.p) { cudaFree(b.p); b.p = nullptr; b.cap = 0; }
+  size_t want = (bytes + 255) & ~(size_t)255;
+  if (cudaMalloc(&b.p, want) != cudaSuccess) { b.p = nullptr; cudaGetLastError(); return AF_ERR_WORKSPACE; }
+  b.cap = want;
+  return AF_OK;
+}
+
+af_status encode_bf16_2d(const af_ctx* ctx, CUtensorMap* map, const void* base, uint64_t rows,
+                         uint64_t cols, uint64_t pitch_bytes, uint32_t box_rows) {
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {pitch_bytes};
+  cuuint32_t box[2] = {64, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = ctx->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims,
+                           strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? AF_OK : AF_ERR_CUDA;
+}
+
+namespace {
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+struct DeviceGuard {
+  int prev = -1;
+  bool ok = true;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+    if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+  }
+  ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+}  // namespace
+}  // namespace af
+
+using namespace af;
+
+extern "C" {
+
+const char* af_status_string(af_status s) {
+  switch (s) {
+    case AF_OK: return "ok";
+    case AF_ERR_INVALID_ARG: return "invalid argument";
+    case AF_ERR_SHAPE: return "unsupported shape";
+    case AF_ERR_ALIGNMENT: return "pointer or pitch not 16-byte aligned";
+    case AF_ERR_CAPACITY: return "output capacity exceeded";
+    case AF_ERR_INDEX: return "sample index out of range";
+    case AF_ERR_WORKSPACE: return "workspace allocation failed";
+    case AF_ERR_CUDA: return "CUDA call failed";
+    case AF_ERR_UNSUPPORTED_DEVICE: return "device is not compute capability 10.0";
+    case AF_ERR_DEVICE_FLAGGED: return "device error word set";
+  }
+  return "unknown status";
+}
+
+af_status af_create(af_ctx** out, int device) {
+  if (!out) return AF_ERR_INVALID_ARG;
+  *out = nullptr;
+  int count = 0;
+  if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) {
+    cudaGetLastError();
+    return AF_ERR_UNSUPPORTED_DEVICE;
+  }
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return AF_ERR_CUDA;
+  if (prop.major != 10 || prop.minor != 0) return AF_ERR_UNSUPPORTED_DEVICE;
+  DeviceGuard guard(device);
+  if (!guard.ok) return AF_ERR_CUDA;
+  af_ctx* c = new (std::nothrow) af_ctx();
+  if (!c) return AF_ERR_WORKSPACE;
+  c->device = device;
+  c->sm_count = prop.multiProcessorCount;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess || !fn) {
+    delete c;
+    return AF_ERR_CUDA;
+  }
+  c->encode = reinterpret_cast<EncodeTiledFn>(fn);
+  if (cudaMalloc(&c->d_err, 256) != cudaSuccess || cudaMemset(c->d_err, 0, 256) != cudaSuccess) {
+    delete c;
+    return AF_ERR_WORKSPACE;
+  }
+  af_status st = ws_grow(c->loss_ws, loss_workspace_bytes(c->sm_count));
+  if (st == AF_OK && cudaMemset(c->loss_ws.p, 0, c->loss_ws.cap) != cudaSuccess) st = AF_ERR_CUDA;
+  if (st != AF_OK) { af_destroy(c); return st; }
+  *out = c;
+  return AF_OK;
+}
+
+af_status af_destroy(af_ctx* c) {
+  if (!c) return AF_ERR_INVALID_ARG;
+  DeviceGuard guard(c->device);
+  cudaDeviceSynchronize();
+  Buf* bufs[] = {&c->partial, &c->loss_ws, &c->pack_meta, &c->wt, &c->ht, &c->dz, &c->dzt};
+  for (Buf* b : bufs) if (b->p) cudaFree(b->p);
+  for (int i = 0; i < kPackRing; ++i) {
+    if (c->pack_host[i]) cudaFreeHost(c->pack_host[i]);
+    if (c->pack_evt_live[i]) cudaEventDestroy(c->pack_evt[i]);
+  }
+  if (c->d_err) cudaFree(c->d_err);
+  delete c;
+  return AF_OK;
+}
+
+int64_t af_workspace_bytes(const af_ctx* c) {
+  if (!c) return 0;
+  return (int64_t)(c->partial.cap + c->loss_ws.cap + c->pack_meta.cap + c->wt.cap + c->ht.cap +
+                   c->dz.cap + c->dzt.cap);
+}
+
+af_status af_set_tuning(af_ctx* c, int32_t v_splits, int32_t bwd_token_block) {
+  if (!c || v_splits < 0 || bwd_token_block < 0) return AF_ERR_INVALID_ARG;
+  if (bwd_token_block % 128 != 0) return AF_ERR_SHAPE;
+  c->v_splits = v_splits;
+  c->bwd_token_block = bwd_token_block;
+  return AF_OK;
+}
+
+af_status af_check_device_errors(af_ctx* c, uint32_t* flags, void* stream) {
+  if (!c) return AF_ERR_INVALID_ARG;
+  DeviceGuard guard(c->device);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  unsigned int h = 0;
+  if (cudaMemcpyAsync(&h, c->d_err, sizeof(h), cudaMemcpyDeviceToHost, s) != cudaSuccess) return AF_ERR_CUDA;
+  if (cudaMemsetAsync(c->d_err, 0, sizeof(h), s) != cudaSuccess) return AF_ERR_CUDA;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return AF_ERR_CUDA;
+  if (flags) *flags = h;
+  return h == 0 ? AF_OK : AF_ERR_DEVICE_FLAGGED;
+}
+
+static size_t pack_meta_bytes(int32_t B) {
+  // [src_row int64 x B][cu int32 x (B+1)][idx int32 x B], each part 16-byte aligned
+  size_t a = ((size_t)B * 8 + 15) & ~(size_t)15;
+  size_t b = ((size_t)(B + 1) * 4 + 15) & ~(size_t)15;
+  size_t c = ((size_t)B * 4 + 15) & ~(size_t)15;
+  return a + b + c + 16;
+}
+
+af_status af_reserve(af_ctx* c, int64_t max_T, int32_t max_B, int32_t d, int32_t V,
+                     int32_t with_backward) {
+  if (!c || max_T < 0 || max_B < 0 || d < 1 || V < 1) return AF_ERR_INVALID_ARG;
+  if (max_T >= ((int64_t)1 << 31)) return AF_ERR_SHAPE;
+  DeviceGuard guard(c->device);
+  af_status st = AF_OK;
+  if (max_T > 0) {
+    const int S = logprob_pick_splits(max_T, V, c->sm_count, c->v_splits);
+    // small batches pick more splits than large ones; reserve for the larger of both products
+    size_t need = (size_t)S * (size_t)max_T;
+    size_t small = (size_t)c->sm_count * 128 * 2;
+    if (need < small) need = small;
+    st = ws_grow(c->partial, need * 16);
+    if (st != AF_OK) return st;
+  }
+  st = ws_grow(c->pack_meta, pack_meta_bytes(max_B));
+  if (st != AF_OK) return st;
+  if (with_backward) {
+    // sizes are recomputed (and grown if needed) by the backward call itself
+    st = launch_backward(c, nullptr, nullptr, nullptr, nullptr, nullptr, max_T, d, V, nullptr, nullptr,
+                         -1 /* reserve only */, nullptr);
+  }
+  return st;
+}
+
+af_status af_pack_microbatch(af_ctx* c, const af_store_view* store, const int32_t* idx_host,
+                             int32_t B, const af_packed* out, int64_t* T_out, void* stream) {
+  if (!c || !store || !out || B < 0 || (B > 0 && !idx_host) || !store->tok_offset_host ||
+      !out->cu_seqlens || store->n_samples < 0 || store->d < 1)
+    return AF_ERR_INVALID_ARG;
+  if ((store->hidden == nullptr) != (out->hidden == nullptr) ||
+      (store->target == nullptr) != (out->target == nullptr) ||
+      (store->old_logp == nullptr) != (out->old_logp == nullptr) ||
+      (store->ref_logp == nullptr) != (out->ref_logp == nullptr) ||
+      (store->adv == nullptr) != (out->adv_seq == nullptr))
+    return AF_ERR_INVALID_ARG;
+  if (store->hidden && (store->d % 8 != 0 || !aligned16(store->hidden) || !aligned16(out->hidden)))
+    return AF_ERR_ALIGNMENT;
+  if (B > out->seq_capacity) return AF_ERR_CAPACITY;
+  DeviceGuard guard(c->device);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+
+  // staging slot (pinned): wait until the copy that last used it has been consumed
+  const int slot = c->pack_slot;
+  c->pack_slot = (slot + 1) % kPackRing;
+  if (c->pack_evt_live[slot] && cudaEventSynchronize(c->pack_evt[slot]) != cudaSuccess) return AF_ERR_CUDA;
+  const size_t bytes = pack_meta_bytes(B);
+  if (c->pack_host_cap[slot] < bytes) {
+    if (c->pack_host[slot]) cudaFreeHost(c->pack_host[slot]);
+    c->pack_host[slot] = nullptr; c->pack_host_cap[slot] = 0;
+    size_t want = bytes < 4096 ? 4096 : bytes * 2;
+    if (cudaMallocHost(&c->pack_host[slot], want) != cudaSuccess) { cudaGetLastError(); return AF_ERR_WORKSPACE; }
+    c->pack_host_cap[slot] = want;
+  }
+  af_status st = ws_grow(c->pack_meta, bytes);
+  if (st != AF_OK) return st;
+
+  const size_t off_cu = ((size_t)B * 8 + 15) & ~(size_t)15;
+  const size_t off_idx = off_cu + (((size_t)(B + 1) * 4 + 15) & ~(size_t)15);
+  char* hb = static_cast<char*>(c->pack_host[slot]);
+  int64_t* h_src = reinterpret_cast<int64_t*>(hb);
+  int32_t* h_cu = reinterpret_cast<int32_t*>(hb + off_cu);
+  int32_t* h_idx = reinterpret_cast<int32_t*>(hb + off_idx);
+  int64_t T = 0;
+  h_cu[0] = 0;
+  for (int32_t j = 0; j < B; ++j) {
+    const int64_t i = idx_host[j];
+    if (i < 0 || i >= store->n_samples) return AF_ERR_INDEX;
+    const int64_t lo = store->tok_offset_host[i], hi = store->tok_offset_host[i + 1];
+    if (hi < lo) return AF_ERR_INVALID_ARG;
+    h_src[j] = lo;
+    h_idx[j] = (int32_t)i;
+    T += hi - lo;
+    if (T >= ((int64_t)1 << 31)) return AF_ERR_CAPACITY;
+    h_cu[j + 1] = (int32_t)T;
+  }
+  if (T_out) *T_out = T;
+  if (T > out->token_capacity) return AF_ERR_CAPACITY;
+
+  char* db = static_cast<char*>(c->pack_meta.p);
+  if (cudaMemcpyAsync(db, hb, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return AF_ERR_CUDA;
+  if (!c->pack_evt_live[slot]) {
+    if (cudaEventCreateWithFlags(&c->pack_evt[slot], cudaEventDisableTiming) != cudaSuccess) return AF_ERR_CUDA;
+    c->pack_evt_live[slot] = true;
+  }
+  if (cudaEventRecord(c->pack_evt[slot], s) != cudaSuccess) return AF_ERR_CUDA;
+  PackSeqTable tab{reinterpret_cast<const int64_t*>(db), reinterpret_cast<const int32_t*>(db + off_cu),
+                   reinterpret_cast<const int32_t*>(db + off_idx)};
+  return launch_pack(*store, *out, tab, B, T, c->sm_count, s) == cudaSuccess ? AF_OK : AF_ERR_CUDA;
+}
+
+af_status af_token_logprob(af_ctx* c, const void* hidden, const void* W, const int32_t* target,
+                           int64_t T, int32_t d, int32_t V, float* logp, float* entropy, float* lse,
+                           void* stream) {
+  if (!c || T < 0 || d < 1 || V < 1) return AF_ERR_INVALID_ARG;
+  if (T == 0) return AF_OK;
+  if (!hidden || !W || !target || !logp) return AF_ERR_INVALID_ARG;
+  if (T >= ((int64_t)1 << 31)) return AF_ERR_SHAPE;
+  if (d % 8 != 0 || !aligned16(hidden) || !aligned16(W)) return AF_ERR_ALIGNMENT;
+  DeviceGuard guard(c->device);
+  return launch_token_logprob(c, hidden, W, target, T, d, V, logp, entropy, lse,
+                              static_cast<cudaStream_t>(stream));
+}
+
+af_status af_grpo_advantage(af_ctx* c, const float* reward, const int32_t* group_id, int64_t N,
+                            int32_t n_groups, float eps_adv, int32_t ddof, float* adv, void* stream) {
+  if (!c || N < 0 || n_groups < 0 || (ddof != 0 && ddof != 1) || !(eps_adv >= 0.f)) return AF_ERR_INVALID_ARG;
+  if (N == 0) return AF_OK;
+  if (!reward || !adv || n_groups < 1) return AF_ERR_INVALID_ARG;
+  if (!group_id && N % n_groups != 0) return AF_ERR_SHAPE;
+  if (group_id && (double)N * (double)n_groups >= 8589934592.0) return AF_ERR_SHAPE;
+  DeviceGuard guard(c->device);
+  return launch_advantage(reward, group_id, N, n_groups, eps_adv, ddof, adv, c->sm_count,
+                          static_cast<cudaStream_t>(stream)) == cudaSuccess ? AF_OK : AF_ERR_CUDA;
+}
+
+af_status af_policy_loss(af_ctx* c, const float* logp, const float* old_logp, const float* ref_logp,
+                         const float* entropy, const float* adv_seq, const int32_t* cu_seqlens,
+                         int32_t B, int64_t T, const af_loss_params* params, af_loss_out* out,
+                         float* dlogp, void* stream) {
+  if (!c || !params || !out || !cu_seqlens || B < 0 || T < 0) return AF_ERR_INVALID_ARG;
+  if (T > 0 && (!logp || !old_logp || !ref_logp || !adv_seq || B < 1)) return AF_ERR_INVALID_ARG;
+  if (params->agg_mode != 0 && params->agg_mode != 1) return AF_ERR_INVALID_ARG;
+  if (T >= ((int64_t)1 << 31)) return AF_ERR_SHAPE;
+  DeviceGuard guard(c->device);
+  return launch_policy_loss(logp, old_logp, ref_logp, entropy, adv_seq, cu_seqlens, B, T, *params, out,
+                            dlogp, c->loss_ws.p, c->d_err, c->sm_count,
+                            static_cast<cudaStream_t>(stream)) == cudaSuccess ? AF_OK : AF_ERR_CUDA;
+}
+
+af_status af_policy_loss_backward(af_ctx* c, const void* hidden, const void* W, const int32_t* target,
+                                  const float* lse, const float* dlogp, int64_t T, int32_t d, int32_t V,
+                                  void* d_hidden, float* d_W, int32_t accumulate_dW, void* stream) {
+  if (!c || T < 0 || d < 1 || V < 1) return AF_ERR_INVALID_ARG;
+  if (!hidden || !W || !target || !lse || !dlogp || !d_hidden || !d_W) {
+    if (T > 0 || !d_W) return AF_ERR_INVALID_ARG;
+  }
+  if (T >= ((int64_t)1 << 31)) return AF_ERR_SHAPE;
+  if (d % 8 != 0 || V % 8 != 0) return AF_ERR_ALIGNMENT;
+  if (!aligned16(hidden) || !aligned16(W) || !aligned16(d_hidden) || !aligned16(d_W)) return AF_ERR_ALIGNMENT;
+  DeviceGuard guard(c->device);
+  return launch_backward(c, hidden, W, target, lse, dlogp, T, d, V, d_hidden, d_W,
+                         accumulate_dW ? 1 : 0, static_cast<cudaStream_t>(stream));
+}
+
+}  // extern "C"

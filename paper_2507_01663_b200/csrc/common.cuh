@@ -1,0 +1,93 @@
+// Shared host-side declarations of the asyncflow library: the context, workspace buffers and
+// the internal launchers each .cu file provides to the C-ABI layer (api.cu).
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/asyncflow.h"
+
+namespace af {
+
+constexpr int kPackRing = 8;  // pinned staging slots for af_pack_microbatch metadata
+
+struct Buf {
+  void* p = nullptr;
+  size_t cap = 0;
+};
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+}  // namespace af
+
+struct af_ctx {
+  int device = 0;
+  int sm_count = 0;
+  af::EncodeTiledFn encode = nullptr;
+  unsigned int* d_err = nullptr;  // sticky device error word
+
+  // tuning
+  int v_splits = 0;         // 0 = automatic
+  int bwd_token_block = 0;  // 0 = default
+
+  // workspace (device)
+  af::Buf partial;    // [splits, T] float4 online-softmax partials
+  af::Buf loss_ws;    // per-block partial sums + ticket of the loss reduction
+  af::Buf pack_meta;  // per-call sequence table of af_pack_microbatch
+  af::Buf wt;         // W^T  [d, V]      bf16 (backward)
+  af::Buf ht;         // H^T  [d, T_pad]  bf16 (backward)
+  af::Buf dz;         // dZ   [Tc, V]     bf16 (backward, one token block)
+  af::Buf dzt;        // dZ^T [V, Tc]     bf16 (backward, one token block)
+
+  // pinned staging ring for pack metadata
+  void* pack_host[af::kPackRing] = {};
+  size_t pack_host_cap[af::kPackRing] = {};
+  cudaEvent_t pack_evt[af::kPackRing] = {};
+  bool pack_evt_live[af::kPackRing] = {};
+  int pack_slot = 0;
+};
+
+namespace af {
+
+af_status ws_grow(Buf& b, size_t bytes);
+
+// Encode a 2-D bf16 tensor map: `rows` x `cols` elements, row pitch `pitch_bytes`, box of
+// `box_rows` x 64 elements, 128-byte swizzle, zero fill outside the tensor.
+af_status encode_bf16_2d(const af_ctx* ctx, CUtensorMap* map, const void* base, uint64_t rows,
+                         uint64_t cols, uint64_t pitch_bytes, uint32_t box_rows);
+
+// ---- launchers (each returns the cudaGetLastError of its launches) --------------------------
+struct PackSeqTable {     // device views into ctx->pack_meta for one call
+  const int64_t* src_row; // [B] first store row of sequence j
+  const int32_t* cu;      // [B+1]
+  const int32_t* idx;     // [B]
+};
+cudaError_t launch_pack(const af_store_view& st, const af_packed& out, const PackSeqTable& tab,
+                        int32_t B, int64_t T, int sm_count, cudaStream_t s);
+
+cudaError_t launch_advantage(const float* reward, const int32_t* group_id, int64_t N,
+                             int32_t n_groups, float eps_adv, int32_t ddof, float* adv,
+                             int sm_count, cudaStream_t s);
+
+size_t loss_workspace_bytes(int sm_count);
+cudaError_t launch_policy_loss(const float* logp, const float* old_logp, const float* ref_logp,
+                               const float* entropy, const float* adv_seq, const int32_t* cu,
+                               int32_t B, int64_t T, const af_loss_params& p, af_loss_out* out,
+                               float* dlogp, void* ws, unsigned int* d_err, int sm_count,
+                               cudaStream_t s);
+
+int logprob_pick_splits(int64_t T, int32_t V, int sm_count, int requested);
+af_status launch_token_logprob(af_ctx* ctx, const void* hidden, const void* W,
+                               const int32_t* target, int64_t T, int32_t d, int32_t V,
+                               float* logp, float* entropy, float* lse, cudaStream_t s);
+
+af_status launch_backward(af_ctx* ctx, const void* hidden, const void* W, const int32_t* target,
+                          const float* lse, const float* dlogp, int64_t T, int32_t d, int32_t V,
+                          void* d_hidden, float* d_W, int32_t accumulate_dW, cudaStream_t s);
+
+}  // namespace af

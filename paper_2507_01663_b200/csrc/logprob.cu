@@ -1,0 +1,151 @@
+// af_token_logprob: LM-head GEMM (tcgen05 / TMEM, TMA-fed) with the online log-softmax, target
+// pick and entropy sums fused into its epilogue, so the [T,V] logits never leave the SM.
+//
+// Each epilogue thread owns one token row.  Sweeping the vocabulary tiles of its unit it keeps
+//   m = running max,  s = sum exp(z - m),  u = sum exp(z - m) * z,  zy = z at the target
+// in registers.  A unit covers one of S vocabulary ranges; the S partial states of a token are
+// written to the workspace and combined by merge_partials_kernel:
+//   lse = M + log sum_i s_i e^{m_i - M},  logp = zy - lse,  entropy = lse - (sum_i u_i e^{m_i-M}) / S.
+#include "common.cuh"
+#include "umma.cuh"
+
+namespace af {
+namespace {
+
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+__device__ __forceinline__ float ex2f(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+struct LogprobEpi {
+  struct Params {
+    const int32_t* target;  // [T]
+    float4* partial;        // [S, T]
+    int T, V;
+  };
+  struct State {
+    float m, s, u, zy;
+    int y;
+  };
+  static __device__ __forceinline__ void unit_begin(State& st, const Params& p, int row, int, int) {
+    st.m = -INFINITY; st.s = 0.f; st.u = 0.f; st.zy = -INFINITY;
+    st.y = row < p.T ? __ldg(p.target + row) : -1;
+  }
+  static __device__ __forceinline__ void chunk(State& st, const Params& p, int, int col0,
+                                               const uint32_t (&v)[32]) {
+    if (col0 >= p.V) return;
+    float z[32];
+#pragma unroll
+    for (int j = 0; j < 32; ++j) z[j] = __uint_as_float(v[j]);
+    if (col0 + 32 > p.V) {  // ragged vocabulary tail: columns >= V hold zero-fill, not logits
+#pragma unroll
+      for (int j = 0; j < 32; ++j) if (col0 + j >= p.V) z[j] = -1.0e30f;
+    }
+    float mx = z[0];
+#pragma unroll
+    for (int j = 1; j < 32; ++j) mx = fmaxf(mx, z[j]);
+    const float m_new = fmaxf(st.m, mx);
+    const float sc = ex2f((st.m - m_new) * kLog2e);  // 0 on the first chunk (m = -inf)
+    float s = st.s * sc, u = st.u * sc;
+    const float nm = -m_new * kLog2e;
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+      const float e = ex2f(fmaf(z[j], kLog2e, nm));
+      s += e;
+      u = fmaf(e, z[j], u);
+    }
+    st.m = m_new; st.s = s; st.u = u;
+    const int yl = st.y - col0;
+    if (yl >= 0 && yl < 32) {
+#pragma unroll
+      for (int j = 0; j < 32; ++j) if (j == yl) st.zy = z[j];
+    }
+  }
+  static __device__ __forceinline__ void unit_end(State& st, const Params& p, int row, int split) {
+    if (row < p.T) p.partial[(size_t)split * p.T + row] = make_float4(st.m, st.s, st.u, st.zy);
+  }
+};
+
+__global__ void __launch_bounds__(256) merge_partials_kernel(
+    const float4* __restrict__ partial, const int32_t* __restrict__ target, int T, int V, int S,
+    float* __restrict__ logp, float* __restrict__ entropy, float* __restrict__ lse_out,
+    unsigned int* d_err) {
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= T) return;
+  float M = -INFINITY;
+  for (int i = 0; i < S; ++i) M = fmaxf(M, __ldg(&partial[(size_t)i * T + t]).x);
+  float s = 0.f, u = 0.f, zy = -INFINITY;
+  for (int i = 0; i < S; ++i) {
+    const float4 q = __ldg(&partial[(size_t)i * T + t]);
+    const float w = ex2f((q.x - M) * kLog2e);
+    s = fmaf(q.y, w, s);
+    u = fmaf(q.z, w, u);
+    zy = fmaxf(zy, q.w);  // exactly one range holds the target; the others report -inf
+  }
+  const float lse = M + kLn2 * log2f(s);
+  const int y = __ldg(target + t);
+  float lp = zy - lse;
+  if (y < 0 || y >= V) {
+    lp = __int_as_float(0x7fc00000);
+    atomicOr(d_err, AF_DEVERR_TARGET_RANGE);
+  }
+  logp[t] = lp;
+  if (entropy) entropy[t] = lse - u / s;
+  if (lse_out) lse_out[t] = lse;
+}
+
+}  // namespace
+
+int logprob_pick_splits(int64_t T, int32_t V, int sm_count, int requested) {
+  const int m_tiles = (int)((T + umma::kBM - 1) / umma::kBM);
+  const int n_tiles = (V + umma::kBN - 1) / umma::kBN;
+  int S = requested > 0 ? requested : 4;
+  if (requested <= 0 && m_tiles * S < sm_count) S = (sm_count + m_tiles - 1) / (m_tiles > 0 ? m_tiles : 1);
+  if (S > n_tiles) S = n_tiles;
+  if (S < 1) S = 1;
+  return S;
+}
+
+af_status launch_token_logprob(af_ctx* ctx, const void* hidden, const void* W,
+                               const int32_t* target, int64_t T, int32_t d, int32_t V,
+                               float* logp, float* entropy, float* lse, cudaStream_t s) {
+  if (T == 0) return AF_OK;
+  const int S = logprob_pick_splits(T, V, ctx->sm_count, ctx->v_splits);
+  af_status st = ws_grow(ctx->partial, (size_t)S * (size_t)T * sizeof(float4));
+  if (st != AF_OK) return st;
+
+  CUtensorMap ta, tb;
+  st = encode_bf16_2d(ctx, &ta, hidden, (uint64_t)T, (uint64_t)d, (uint64_t)d * 2, umma::kBM);
+  if (st != AF_OK) return st;
+  st = encode_bf16_2d(ctx, &tb, W, (uint64_t)V, (uint64_t)d, (uint64_t)d * 2, umma::kBN);
+  if (st != AF_OK) return st;
+
+  umma::GemmShape g;
+  g.M = (int)T; g.N = V; g.K = d;
+  g.m_tiles = (int)((T + umma::kBM - 1) / umma::kBM);
+  g.n_tiles = (V + umma::kBN - 1) / umma::kBN;
+  g.splits = S;
+  g.k_blocks = (d + umma::kBK - 1) / umma::kBK;
+  LogprobEpi::Params ep{target, (float4*)ctx->partial.p, (int)T, V};
+
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(umma::gemm_kernel<LogprobEpi>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             umma::kSmemBytes) != cudaSuccess) return AF_ERR_CUDA;
+    attr_set = true;
+  }
+  const int64_t units = (int64_t)g.m_tiles * S;
+  const int grid = (int)(units < ctx->sm_count ? units : ctx->sm_count);
+  umma::gemm_kernel<LogprobEpi><<<grid, umma::kThreads, umma::kSmemBytes, s>>>(ta, tb, g, ep, ctx->d_err);
+  if (cudaGetLastError() != cudaSuccess) return AF_ERR_CUDA;
+  merge_partials_kernel<<<(int)((T + 255) / 256), 256, 0, s>>>((const float4*)ctx->partial.p, target,
+                                                              (int)T, V, S, logp, entropy, lse,
+                                                              ctx->d_err);
+  return cudaGetLastError() == cudaSuccess ? AF_OK : AF_ERR_CUDA;
+}
+
+}  // namespace af

@@ -1,0 +1,317 @@
+// Blackwell (sm_100a) building blocks: mbarrier, TMA tile loads, tcgen05 MMA with TMEM
+// accumulators -- inline PTX only -- and the warp-specialised persistent GEMM main loop every
+// tensor-core kernel of the library is built on.
+//
+//   C[M,N] = A[M,K] * B[N,K]^T     A, B bf16, both K-major (row-major with K contiguous);
+//   fp32 accumulation in tensor memory; the epilogue functor consumes the accumulator tile.
+//
+// CTA = 6 warps.  warp 0: TMA producer (one elected lane).  warp 1: allocates TMEM and issues
+// tcgen05.mma (one elected lane).  warps 2-5: epilogue, one TMEM lane (= output row) per thread.
+// Shared memory holds a ring of kStages {A 128x64, B 256x64} bf16 tiles in the 128-byte swizzle
+// TMA writes and the MMA descriptors expect; TMEM holds two 128x256 fp32 accumulators so the
+// epilogue of tile i overlaps the MMAs of tile i+1.
+//
+// Every wait is bounded: a wait that exceeds kWaitLimitNs raises AF_DEVERR_WATCHDOG, makes all
+// roles leave their loops, frees TMEM and returns.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace af {
+namespace umma {
+
+constexpr int kBM = 128;          // rows of A per tile  (UMMA M)
+constexpr int kBN = 256;          // rows of B per tile  (UMMA N)
+constexpr int kBK = 64;           // K elements per stage = one 128-byte swizzle row
+constexpr int kUmmaK = 16;        // K per tcgen05.mma for 16-bit inputs
+constexpr int kStages = 4;
+constexpr int kABytes = kBM * kBK * 2;
+constexpr int kBBytes = kBN * kBK * 2;
+constexpr int kStageBytes = kABytes + kBBytes;            // 48 KB
+constexpr int kTmemCols = 512;                            // 2 accumulators x 256 fp32 columns
+constexpr int kThreads = 192;
+constexpr int kEpiThreads = 128;
+constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr unsigned long long kWaitLimitNs = 4000000000ull;
+constexpr unsigned int kWatchdogBit = 2u;                 // AF_DEVERR_WATCHDOG
+
+// ------------------------------------------------------------------------------------------
+// PTX wrappers
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ unsigned long long globaltimer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void fence_mbar_init() {
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false if the CTA is aborting (some wait ran out of time).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = globaltimer_ns();
+  uint32_t spins = 0;
+  while (!mbar_try_wait(bar, parity)) {
+    if ((++spins & 63u) == 0u) {
+      if (*abort_flag) return false;
+      if (globaltimer_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+    }
+  }
+  return true;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst_smem, const CUtensorMap* map, uint32_t bar,
+                                            int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst_smem), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* map) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() {
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after() {
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]^T, 128 x 256 x 16, bf16 inputs, fp32 accumulate.
+__device__ __forceinline__ void mma_bf16_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                            uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// Arrive on `bar` once every MMA issued so far by this thread has completed.
+__device__ __forceinline__ void mma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// 32 consecutive fp32 columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() {
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory matrix descriptor for a K-major bf16 tile stored as rows of 128 bytes with the
+// 128-byte swizzle (what TMA writes for a 64-element-wide box): 8-row groups are 1024 bytes
+// apart (stride byte offset), the leading byte offset is unused for this layout.
+__device__ __forceinline__ uint64_t smem_desc_k_sw128(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);  // start address, 16-byte units
+  d |= (uint64_t)1 << 16;                        // leading byte offset (ignored when swizzled)
+  d |= (uint64_t)(1024 >> 4) << 32;              // stride byte offset
+  d |= (uint64_t)1 << 46;                        // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;                        // layout: 128-byte swizzle
+  return d;
+}
+// Instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = 256.
+__host__ __device__ constexpr uint32_t instr_desc_bf16_f32(int m, int n) {
+  return (1u << 4)                         // D format: fp32
+         | (1u << 7) | (1u << 10)          // A, B format: bf16
+         | ((uint32_t)(n >> 3) << 17)      // N / 8
+         | ((uint32_t)(m >> 4) << 24);     // M / 16
+}
+
+// ------------------------------------------------------------------------------------------
+// Work decomposition shared by all three roles.
+// A unit is one token/row tile (m_tile) times a contiguous range of B tiles (split s of S);
+// CTA b processes units b, b + grid, b + 2 grid, ...  Consecutive units share the m_tile, so
+// the CTAs running at one time work on grid/S row tiles and sweep the B tiles together: the
+// A panels stay L2-resident and every B tile is fetched from HBM once per wave.
+// ------------------------------------------------------------------------------------------
+struct GemmShape {
+  int M, N, K;          // logical extents (rows of A, rows of B, reduction length)
+  int m_tiles, n_tiles; // ceil(M/128), ceil(N/256)
+  int splits;           // S: n-tile ranges per m_tile
+  int k_blocks;         // ceil(K/64)
+};
+__device__ __forceinline__ int split_begin(const GemmShape& g, int s) {
+  return (int)(((long long)g.n_tiles * s) / g.splits);
+}
+
+// The epilogue functor E provides:
+//   struct Params;  struct State;
+//   static __device__ void unit_begin(State&, const Params&, int row, int m_tile, int split);
+//   static __device__ void chunk(State&, const Params&, int row, int col0, const uint32_t (&v)[32]);
+//        -- 32 fp32 accumulator columns col0 .. col0+31 of output row `row` (bit patterns)
+//   static __device__ void unit_end(State&, const Params&, int row, int split);
+template <class E>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+            const GemmShape g, const typename E::Params ep, unsigned int* d_err) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t tiles = (raw + 1023u) & ~1023u;                 // 1024-byte aligned tile ring
+  const uint32_t bars = tiles + kStages * kStageBytes;           // barriers behind the ring
+  // barrier addresses
+  auto full_bar = [&](int s) { return bars + 8u * s; };
+  auto empty_bar = [&](int s) { return bars + 8u * (kStages + s); };
+  auto tfull_bar = [&](int a) { return bars + 8u * (2 * kStages + a); };
+  auto tempty_bar = [&](int a) { return bars + 8u * (2 * kStages + 2 + a); };
+  const uint32_t tmem_slot = bars + 8u * (2 * kStages + 4);
+  volatile uint32_t* tmem_slot_ptr =
+      reinterpret_cast<volatile uint32_t*>(smem_raw + (tmem_slot - raw));
+  __shared__ int abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), kEpiThreads); }
+    fence_mbar_init();
+    tma_prefetch_desc(&tmap_a);
+    tma_prefetch_desc(&tmap_b);
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot_ptr;
+
+  const int total_units = g.m_tiles * g.splits;
+
+  if (warp == 0) {
+    // ---------------------------------------------------------------- TMA producer
+    if (lane == 0) {
+      int stage = 0; uint32_t phase = 0; bool ok = true;
+      for (int u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
+        const int m_tile = u / g.splits, s = u % g.splits;
+        const int nb = split_begin(g, s), ne = split_begin(g, s + 1);
+        for (int nt = nb; nt < ne && ok; ++nt) {
+          for (int kb = 0; kb < g.k_blocks; ++kb) {
+            if (!mbar_wait(empty_bar(stage), phase ^ 1u, &abort_flag)) { ok = false; break; }
+            const uint32_t a_dst = tiles + stage * kStageBytes;
+            mbar_arrive_expect_tx(full_bar(stage), kStageBytes);
+            tma_load_2d(a_dst, &tmap_a, full_bar(stage), kb * kBK, m_tile * kBM);
+            tma_load_2d(a_dst + kABytes, &tmap_b, full_bar(stage), kb * kBK, nt * kBN);
+            if (++stage == kStages) { stage = 0; phase ^= 1u; }
+          }
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ---------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = instr_desc_bf16_f32(kBM, kBN);
+      int stage = 0; uint32_t phase = 0; uint32_t tile_count = 0; bool ok = true;
+      for (int u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
+        const int s = u % g.splits;
+        const int nb = split_begin(g, s), ne = split_begin(g, s + 1);
+        for (int nt = nb; nt < ne && ok; ++nt, ++tile_count) {
+          const uint32_t acc = tile_count & 1u, acc_phase = (tile_count >> 1) & 1u;
+          if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, &abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t d_tmem = tmem_base + acc * kBN;
+          for (int kb = 0; kb < g.k_blocks; ++kb) {
+            if (!mbar_wait(full_bar(stage), phase, &abort_flag)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t a_addr = tiles + stage * kStageBytes;
+            const uint64_t a_desc = smem_desc_k_sw128(a_addr);
+            const uint64_t b_desc = smem_desc_k_sw128(a_addr + kABytes);
+#pragma unroll
+            for (int k = 0; k < kBK / kUmmaK; ++k) {
+              // advance both descriptors by k * 32 bytes inside the swizzle row (16-byte units)
+              mma_bf16_ss(d_tmem, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)(k * 2), idesc,
+                          (kb | k) != 0 ? 1u : 0u);
+            }
+            mma_commit(empty_bar(stage));  // smem slot reusable once these MMAs have read it
+            if (++stage == kStages) { stage = 0; phase ^= 1u; }
+          }
+          if (ok) mma_commit(tfull_bar(acc));  // accumulator complete
+        }
+      }
+    }
+    __syncwarp();
+  } else {
+    // ---------------------------------------------------------------- epilogue (warps 2..5)
+    const int quarter = warp & 3;                       // TMEM lanes this warp may touch
+    const int row_in_tile = quarter * 32 + lane;
+    uint32_t tile_count = 0; bool ok = true;
+    typename E::State st;
+    for (int u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
+      const int m_tile = u / g.splits, s = u % g.splits;
+      const int nb = split_begin(g, s), ne = split_begin(g, s + 1);
+      const int row = m_tile * kBM + row_in_tile;
+      E::unit_begin(st, ep, row, m_tile, s);
+      for (int nt = nb; nt < ne && ok; ++nt, ++tile_count) {
+        const uint32_t acc = tile_count & 1u, acc_phase = (tile_count >> 1) & 1u;
+        if (!mbar_wait(tfull_bar(acc), acc_phase, &abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * kBN;
+#pragma unroll 1
+        for (int c = 0; c < kBN / 32; ++c) {
+          uint32_t v[32];
+          tmem_ld32(t_row + c * 32, v);
+          tmem_ld_wait();
+          E::chunk(st, ep, row, nt * kBN + c * 32, v);
+        }
+        tc_fence_before();
+        mbar_arrive(tempty_bar(acc));
+      }
+      if (ok) E::unit_end(st, ep, row, s);
+    }
+  }
+
+  // ---------------------------------------------------------------- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && abort_flag) atomicOr(d_err, kWatchdogBit);
+  if (warp == 1) {
+    if (abort_flag) __nanosleep(1000000);  // let copies in flight land before the CTA retires
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+}  // namespace umma
+}  // namespace af
