@@ -1,0 +1,362 @@
+#!/usr/bin/env python
+"""Benchmark of the GRPO scoring hot path on B200.
+
+One *step* = one pass of the whole path over one synthetic batch shaped like the Qwen2.5-7B
+workload (512 responses, ~1.1 M scored tokens): group advantages -> pack by sample index ->
+fused LM-head log-prob / entropy -> clipped policy loss + k3 KL (with dL/dlogp).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload cfg2]
+
+Prints ONE JSON line (rank 0).  ``value`` is scored tokens/s over all ranks with the inputs
+resident in HBM; ``e2e`` is the same metric with the store columns starting in pinned host
+memory (host->device copies and the device->host read of the loss inside the timed region).
+``--impl reference`` times the fp64 CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2507_01663_b200 import workloads as wl  # noqa: E402
+
+METRIC = "scored tokens/sec (logprob+GRPO loss) at Qwen-7B head; % dense-BF16 peak"
+UNIT = "tokens/s"
+KERNELS_PER_STEP = 6  # advantage, pack columns, pack rows, fused LM-head GEMM, partial merge, loss
+
+
+# ------------------------------------------------------------------------------------------
+# helpers
+# ------------------------------------------------------------------------------------------
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.QUERY}",
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._pump, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+def rank_workload(name: str, rank: int) -> wl.Workload:
+    """Weak scaling: every rank scores its own batch of the same shape (own seed => own lengths)."""
+    return wl.make_workload(name, seed_offset=1000 * rank)
+
+
+def reduce_over_ranks(ms_local: float, tokens_local: int, world: int):
+    """(max over ranks of the step time, sum over ranks of the tokens)."""
+    if world == 1:
+        return ms_local, tokens_local
+    import torch.distributed as dist
+    dev = torch.device("cuda", torch.cuda.current_device()) if dist.get_backend() == "nccl" else torch.device("cpu")
+    t = torch.tensor([ms_local], dtype=torch.float64, device=dev)
+    n = torch.tensor([tokens_local], dtype=torch.int64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(n, op=dist.ReduceOp.SUM)
+    return float(t.item()), int(n.item())
+
+
+# ------------------------------------------------------------------------------------------
+# the CUDA arm
+# ------------------------------------------------------------------------------------------
+class ScoringJob:
+    """Device buffers of one rank and the step function that runs the path through the C ABI."""
+
+    def __init__(self, w: wl.Workload, device: torch.device):
+        from paper_2507_01663_b200 import binding as B
+        self.B, self.w, self.dev = B, w, device
+        self.ctx = B.Context(device.index or 0)
+        T = w.total_tokens
+        self.T = T
+        self.store = {
+            "hidden": wl.gen_hidden(w, device), "target": wl.gen_target(w, device),
+        }
+        self.W = wl.gen_weight(w, device)
+        self.reward = wl.gen_reward(w, device)
+        centre = wl.centre_logp_estimate(w, self.store["hidden"], self.W, self.store["target"])
+        self.store["old_logp"] = centre + wl.gen_noise(w, wl.S_OLD, T, device)
+        self.store["ref_logp"] = centre + wl.gen_noise(w, wl.S_REF, T, device)
+        del centre
+        self.adv = torch.empty(w.N, device=device)
+        self.idx = wl.arrival_order(w)
+        self.off = w.tok_offset
+        self.packed = {
+            "cu_seqlens": torch.zeros(w.N + 1, dtype=torch.int32, device=device),
+            "hidden": torch.empty(T, w.d, dtype=torch.bfloat16, device=device),
+            "target": torch.empty(T, dtype=torch.int32, device=device),
+            "old_logp": torch.empty(T, device=device), "ref_logp": torch.empty(T, device=device),
+            "adv_seq": torch.empty(w.N, device=device),
+        }
+        self.logp, self.ent, self.lse, self.dlogp = (torch.empty(T, device=device) for _ in range(4))
+        self.loss_out = B.new_loss_out(device)
+        self.ctx.reserve(T, w.N, w.d, w.V)
+        self.gemm_events = []
+
+    def step(self, time_gemm: bool = False):
+        w, c = self.w, self.ctx
+        c.grpo_advantage(self.reward, None, w.n_prompts, self.adv)
+        store = {"tok_offset_host": self.off, "d": w.d, "adv": self.adv, **self.store}
+        T = c.pack_microbatch(store, self.idx, self.packed)
+        if time_gemm:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+        c.token_logprob(self.packed["hidden"], self.W, self.packed["target"], self.logp, self.ent, self.lse, T=T)
+        if time_gemm:
+            e1.record()
+            self.gemm_events.append((e0, e1))
+        c.policy_loss(self.logp, self.packed["old_logp"], self.packed["ref_logp"], self.packed["adv_seq"],
+                      self.packed["cu_seqlens"], self.loss_out, self.dlogp, self.ent,
+                      w.clip_eps, w.clip_eps, w.kl_coef, 0, 1.0, B=w.N, T=T)
+        return T
+
+    # -- end-to-end: store columns start in pinned host memory ------------------------------
+    def make_host_store(self):
+        self.host = {k: torch.empty(v.shape, dtype=v.dtype, pin_memory=True) for k, v in self.store.items()}
+        self.host["reward"] = torch.empty(self.reward.shape, dtype=self.reward.dtype, pin_memory=True)
+        for k, v in self.store.items():
+            self.host[k].copy_(v)
+        self.host["reward"].copy_(self.reward)
+        torch.cuda.synchronize()
+        self.h2d_bytes = sum(t.numel() * t.element_size() for t in self.host.values())
+        self.host_loss = torch.empty(self.loss_out.shape, dtype=torch.uint8, pin_memory=True)
+
+    def step_e2e(self):
+        for k, v in self.store.items():
+            v.copy_(self.host[k], non_blocking=True)
+        self.reward.copy_(self.host["reward"], non_blocking=True)
+        T = self.step()
+        self.host_loss.copy_(self.loss_out, non_blocking=True)
+        return T
+
+
+def timed_loop(fn, steps: int, world: int):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+    return e0.elapsed_time(e1)
+
+
+def cpu_oracle_sample(w: wl.Workload, hidden_rows: torch.Tensor, W_bits: np.ndarray, target_rows: np.ndarray,
+                      reward: np.ndarray):
+    """One pass of the oracle, as it stands, over a sample of `n` tokens forming one sequence of
+    the batch: pack -> log-prob -> advantage (all N responses) -> loss.  Returns seconds."""
+    from oracle import grpo_oracle as O
+    n = hidden_rows.shape[0]
+    t0 = time.perf_counter()
+    packed = O.pack_microbatch_ref(np.array([0, n]), [0], {"hidden": wl.bf16_bits(hidden_rows), "target": target_rows})
+    logp, ent, lse = O.token_logprob_ref(packed["hidden"], W_bits, packed["target"])
+    adv = O.grpo_advantage_ref(reward, w.group_id, w.n_prompts)
+    O.policy_loss_ref(logp, logp + 0.1, logp - 0.1, adv[:1], packed["cu_seqlens"], w.clip_eps, w.clip_eps,
+                      w.kl_coef, entropy=ent)
+    return time.perf_counter() - t0
+
+
+def blas_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return max(n) if n else (os.cpu_count() or 1)
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def run_ours(args):
+    rank, local_rank, world = dist_env()
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (there is no CPU path)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    w = rank_workload(args.workload, rank)
+    job = ScoringJob(w, dev)
+    peaks = measured_peaks()
+
+    for _ in range(args.warmup):
+        job.step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    ms_total = timed_loop(lambda: job.step(time_gemm=True), args.steps, world)
+    clocks = sampler.stop() if rank == 0 else None
+    gemm_ms = float(np.mean([a.elapsed_time(b) for a, b in job.gemm_events]))
+    ms_step, tokens = reduce_over_ranks(ms_total / args.steps, job.T, world)
+    flags = job.ctx.check_device_errors()
+    if flags:
+        raise RuntimeError(f"device error word set: {flags}")
+    loss = job.B.read_loss_out(job.loss_out)["loss"]
+
+    # end to end from pinned host memory
+    job.make_host_store()
+    for _ in range(max(1, min(args.warmup, 2))):
+        job.step_e2e()
+    ms_e2e_total = timed_loop(job.step_e2e, args.steps, world)
+    ms_e2e, _ = reduce_over_ranks(ms_e2e_total / args.steps, job.T, world)
+
+    flops = 2.0 * job.T * w.d * w.V
+    achieved = flops / (gemm_ms * 1e-3) / 1e12
+    peak = peaks["bf16_tflops_sustained"]
+    line = {
+        "metric": METRIC, "value": tokens / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"{args.workload}: Qwen2.5-7B-shaped head d={w.d} V={w.V}, {w.N} responses "
+                               f"({w.n_prompts} prompts x {w.group_size}), {job.T} scored tokens per GPU, "
+                               "one arrival-ordered packed micro-batch",
+                   "l2": "inputs (hidden states >> 126 MB L2) exceed L2; no flush needed",
+                   "loss": {"clip_eps": w.clip_eps, "kl_coef": w.kl_coef, "agg": "seq-mean-token-mean"}},
+        "roofline": {"bound": "tensor", "kernel": "fused LM-head GEMM + online log-softmax (af_token_logprob)",
+                     "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                     "peak_source": f"bf16_tflops_sustained, {peaks['source']}",
+                     "frac_of_burst": achieved / peaks["bf16_tflops"], "frac_of_nominal_2250": achieved / 2250.0,
+                     "kernel_ms": gemm_ms, "traffic": None},
+        "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": job.h2d_bytes,
+                "d2h_bytes_per_step": int(job.loss_out.numel()), "ms_per_step": ms_e2e},
+        "gpu_launches": KERNELS_PER_STEP * args.steps,
+        "clocks": clocks, "loss": loss,
+    }
+    if rank == 0 and world == 1:
+        n = args.cpu_sample
+        rows = job.packed["hidden"][:n].cpu()
+        W_bits = wl.bf16_bits(job.W)
+        secs = cpu_oracle_sample(w, rows, W_bits, job.packed["target"][:n].cpu().numpy(), job.reward.cpu().numpy())
+        line["cpu_baseline"] = {"value": n / secs, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+                                "sample": f"first {n} packed tokens as one sequence through pack/log-prob/loss "
+                                          f"oracles at full V={w.V}, advantage oracle over all {w.N} responses; "
+                                          f"{secs:.1f} s"}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+# ------------------------------------------------------------------------------------------
+# the reference arm: the CPU oracle on bounded samples
+# ------------------------------------------------------------------------------------------
+def run_reference(args):
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    w = wl.make_workload(args.workload)
+    n = args.cpu_sample
+    W_bits = wl.bf16_bits(wl.gen_weight(w, "cpu"))
+    reward = wl.gen_reward(w).numpy()
+    target = wl.gen_target(w).numpy()
+    times = []
+    for s in range(args.warmup + args.steps):
+        rows = wl.gen_hidden(w, "cpu", row_start=s * n, rows=n)
+        secs = cpu_oracle_sample(w, rows, W_bits, target[s * n:(s + 1) * n], reward)
+        if s >= args.warmup:
+            times.append(secs)
+    ms = 1e3 * float(np.mean(times))
+    value = n / (ms * 1e-3)
+    sample = f"{n} tokens per step as one sequence at full V={w.V} (pack/log-prob/loss oracles), advantage over {w.N} responses"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{args.workload}: Qwen2.5-7B-shaped head d={w.d} V={w.V}; bounded sample: {sample}"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--cpu-sample", type=int, default=256, help="tokens in the CPU-oracle sample")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -80,7 +80,7 @@ __global__ void __launch_bounds__(kThreads) policy_loss_kernel(
         if (t >= seq_end) {  // run of sequence j ends: scale it once, move to the next sequence
           acc_pg += run_pg * inv_len; acc_kl += run_kl * inv_len;
           run_pg = 0.f; run_kl = 0.f;
-          do { ++j; seq_end = __ldg(cu + j + 1); } while (t >= seq_end && j < B - 1);
+          while (t >= seq_end && j < B - 1) { ++j; seq_end = __ldg(cu + j + 1); }
           A = __ldg(adv_seq + j);
           inv_len = prm.agg_mode == 0 ? 1.f / (float)(seq_end - __ldg(cu + j)) : 1.f;
         }

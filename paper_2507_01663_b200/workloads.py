@@ -161,35 +161,39 @@ def _fixed_total_lengths(seed, n, lo, hi, total):
     return L
 
 
-def make_workload(name: str) -> Workload:
+def make_workload(name: str, seed_offset: int = 0) -> Workload:
     """The five evaluation workloads (``cfg1`` .. ``cfg5``) and reduced test variants (``*_mini``).
 
     Mini variants keep the structure (group sizes, length law, ragged tails) at sizes a CPU
     oracle evaluates in seconds; their V is deliberately not a multiple of the GEMM tile.
+    ``seed_offset`` derives an independent draw of the same shape (one per data-parallel rank).
     """
+    base = {"cfg1": 0, "cfg2": 1, "cfg3": 2, "cfg4": 3, "cfg5": 4,
+            "cfg2_mini": 11, "cfg3_mini": 12, "cfg4_mini": 13, "cfg5_mini": 14}
+    if name not in base:
+        raise KeyError(name)
+    sd = base[name] + seed_offset
     if name == "cfg1":
-        return Workload(name, 0, 256, 4096, 8, 4, _uniform_lengths(0, 32, 16, 64), "bernoulli:0.5")
+        return Workload(name, sd, 256, 4096, 8, 4, _uniform_lengths(sd, 32, 16, 64), "bernoulli:0.5")
     if name == "cfg2":
-        return Workload(name, 1, 3584, 152064, 64, 8, _uniform_lengths(1, 512, 256, 4096), "bernoulli:0.3")
+        return Workload(name, sd, 3584, 152064, 64, 8, _uniform_lengths(sd, 512, 256, 4096), "bernoulli:0.3")
     if name == "cfg3":
-        return Workload(name, 2, 5120, 152064, 32, 16, _lognormal_lengths(2, 512, 1024, 1.0, 64, 8192), "uniform")
+        return Workload(name, sd, 5120, 152064, 32, 16, _lognormal_lengths(sd, 512, 1024, 1.0, 64, 8192), "uniform")
     if name == "cfg4":
-        return Workload(name, 3, 3584, 152064, 16, 8, _fixed_total_lengths(3, 128, 64, 1024, 65536),
+        return Workload(name, sd, 3584, 152064, 16, 8, _fixed_total_lengths(sd, 128, 64, 1024, 65536),
                         "bernoulli:0.5", backward=True)
     if name == "cfg5":
-        return Workload(name, 4, 3584, 152064, 64, 64, _pareto_lengths(4, 4096, 128, 1.5, 16384),
+        return Workload(name, sd, 3584, 152064, 64, 64, _pareto_lengths(sd, 4096, 128, 1.5, 16384),
                         "bernoulli:0.3", token_budget=32768)
     if name == "cfg2_mini":
-        return Workload(name, 11, 512, 8200, 8, 8, _uniform_lengths(11, 64, 32, 300), "bernoulli:0.3")
+        return Workload(name, sd, 512, 8200, 8, 8, _uniform_lengths(sd, 64, 32, 300), "bernoulli:0.3")
     if name == "cfg3_mini":
-        return Workload(name, 12, 640, 5000, 4, 16, _lognormal_lengths(12, 64, 96, 1.0, 8, 700), "uniform")
+        return Workload(name, sd, 640, 5000, 4, 16, _lognormal_lengths(sd, 64, 96, 1.0, 8, 700), "uniform")
     if name == "cfg4_mini":
-        return Workload(name, 13, 512, 8192, 4, 8, _fixed_total_lengths(13, 32, 8, 64, 1024),
+        return Workload(name, sd, 512, 8192, 4, 8, _fixed_total_lengths(sd, 32, 8, 64, 1024),
                         "bernoulli:0.5", backward=True)
-    if name == "cfg5_mini":
-        return Workload(name, 14, 256, 4104, 8, 16, _pareto_lengths(14, 128, 8, 1.5, 512),
-                        "bernoulli:0.3", token_budget=1024)
-    raise KeyError(name)
+    return Workload(name, sd, 256, 4104, 8, 16, _pareto_lengths(sd, 128, 8, 1.5, 512),
+                    "bernoulli:0.3", token_budget=1024)
 
 
 # ----------------------------------------------------------------------------------------
@@ -287,3 +291,18 @@ def shard_prompts(n_prompts: int, world_size: int, rank: int) -> range:
 def bf16_bits(t: torch.Tensor) -> np.ndarray:
     """Raw bf16 bit patterns of a tensor as a numpy uint16 array (numpy has no bf16 dtype)."""
     return t.detach().cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
+
+
+def centre_logp_estimate(w: Workload, hidden: torch.Tensor, weight: torch.Tensor,
+                         target: torch.Tensor, chunk: int = 1 << 16) -> torch.Tensor:
+    """A cheap stand-in for "the current log-prob" used only to centre synthetic old / ref
+    log-probs where scoring every token on the CPU is out of reach: the target logit (one dot
+    product per token) minus the Gaussian estimate ln V + |h|^2 w_std^2 / 2 of the normaliser a
+    random head produces.  Inputs are perturbed around it by ``gen_noise``; nothing is checked
+    against it."""
+    out = torch.empty(hidden.shape[0], dtype=torch.float32, device=hidden.device)
+    for s in range(0, hidden.shape[0], chunk):
+        h = hidden[s:s + chunk].float()
+        zy = (h * weight[target[s:s + chunk].long()].float()).sum(1)
+        out[s:s + chunk] = zy - (math.log(w.V) + 0.5 * (w.w_std ** 2) * (h * h).sum(1))
+    return out

@@ -1,0 +1,176 @@
+"""af_grpo_advantage and af_policy_loss against the oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import grpo_oracle as O
+from paper_2507_01663_b200 import workloads as wl
+from gpu_util import ADV_TOL, LOSS_RTOL, device, f32, i32, np_of, rel
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    from paper_2507_01663_b200 import binding as B
+    c = B.Context(0)
+    yield c
+    c.close()
+
+
+# ---------------------------------------------------------------- advantage
+@pytest.mark.parametrize("name", ["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
+@pytest.mark.parametrize("ddof", [0, 1])
+def test_advantage_workload_rewards(ctx, name, ddof):
+    w = wl.make_workload(name)
+    dev = device()
+    r = wl.gen_reward(w, dev)
+    ref = O.grpo_advantage_ref(np_of(r), w.group_id, w.n_prompts, 1e-6, ddof)
+    adv = torch.full((w.N,), 9.0, device=dev)
+    ctx.grpo_advantage(r, None, w.n_prompts, adv, 1e-6, ddof)                 # contiguous groups
+    assert np.abs(np_of(adv) - ref).max() <= ADV_TOL
+    adv2 = torch.full((w.N,), 9.0, device=dev)
+    ctx.grpo_advantage(r, i32(w.group_id), w.n_prompts, adv2, 1e-6, ddof)     # explicit ids
+    assert np.abs(np_of(adv2) - ref).max() <= ADV_TOL
+    # ids in arbitrary order
+    perm = wl.arrival_order(w)
+    adv3 = torch.full((w.N,), 9.0, device=dev)
+    ctx.grpo_advantage(r[torch.as_tensor(perm.astype(np.int64), device=dev)].contiguous(),
+                       i32(w.group_id[perm]), w.n_prompts, adv3, 1e-6, ddof)
+    assert np.abs(np_of(adv3) - ref[perm]).max() <= ADV_TOL
+    assert ctx.check_device_errors() == 0
+
+
+@pytest.mark.parametrize("G", [1, 2, 3, 5, 8, 31, 32, 33, 64, 100, 1000, 5000])
+def test_advantage_group_sizes(ctx, G):
+    n_groups = 37 if G < 1000 else 3
+    N = G * n_groups
+    r = wl.uniform01(G, wl.S_REWARD, 0, N, device())
+    ref = O.grpo_advantage_ref(np_of(r), np.arange(N) // G, n_groups, 1e-6, 0)
+    adv = torch.full((N,), 9.0, device=device())
+    ctx.grpo_advantage(r, None, n_groups, adv)
+    assert np.abs(np_of(adv) - ref).max() <= ADV_TOL
+
+
+def test_advantage_degenerate_groups(ctx):
+    # equal rewards inside a group (also non-dyadic values) give exactly-zero-sized advantages
+    r = f32([0.3] * 8 + [1.0] * 8 + [0.0] * 8 + [0.1, 0.7, 0.1, 0.7, 0.1, 0.7, 0.1, 0.7])
+    adv = torch.full((32,), 9.0, device=device())
+    ctx.grpo_advantage(r, None, 4, adv)
+    ref = O.grpo_advantage_ref(np_of(r), np.arange(32) // 8, 4, 1e-6, 0)
+    a = np_of(adv)
+    assert np.abs(a - ref).max() <= ADV_TOL and np.abs(a[:24]).max() <= ADV_TOL
+    assert np.allclose(np.abs(a[24:]), 1.0, atol=1e-4)
+    # many groups (bandwidth shape): still element-exact against the oracle on a sample
+    N, G = 1 << 20, 8
+    rr = (wl.uniform01(3, wl.S_REWARD, 0, N, device()) < 0.3).float()
+    out = torch.empty(N, device=device())
+    ctx.grpo_advantage(rr, None, N // G, out)
+    sl = slice(1000 * G, 1200 * G)
+    ref2 = O.grpo_advantage_ref(np_of(rr[sl]), np.arange(200 * G) // G, 200, 1e-6, 0)
+    assert np.abs(np_of(out[sl]) - ref2).max() <= ADV_TOL
+    # empty input is a no-op; N not divisible by the group count is refused
+    from paper_2507_01663_b200.binding import AfError
+    ctx.grpo_advantage(r, None, 4, adv, N=0)
+    with pytest.raises(AfError) as e:
+        ctx.grpo_advantage(r, None, 5, adv)
+    assert e.value.status == -2
+
+
+# ---------------------------------------------------------------- loss
+def loss_inputs(w, T, lens, seed_shift=0):
+    """logp around a random head's magnitude; old / ref = logp + N(0, 0.1) as in the workloads."""
+    logp = wl.gen_surrogate_logp(w, T)
+    old = logp + wl.gen_noise(w, wl.S_OLD, T, start=seed_shift)
+    ref = logp + wl.gen_noise(w, wl.S_REF, T, start=seed_shift)
+    ent = torch.abs(wl.normal01(w.seed, wl.S_MISC, 0, T)) + 5.0
+    return logp, old, ref, ent
+
+
+def run_loss(ctx, logp, old, ref, ent, adv_seq, cu, **kw):
+    from paper_2507_01663_b200 import binding as B
+    dev = device()
+    T = logp.shape[0]
+    out = B.new_loss_out(dev)
+    g = torch.full((max(T, 1),), 9.0, device=dev)
+    ctx.policy_loss(logp.to(dev), old.to(dev), ref.to(dev), f32(adv_seq), i32(cu), out, g,
+                    None if ent is None else ent.to(dev), T=T, **kw)
+    res = B.read_loss_out(out)
+    return res, np_of(g)[:T]
+
+
+def compare_loss(res, g, ref, T, clip_lo=0.2, clip_hi=0.2):
+    for k in ("loss", "pg_loss", "kl_mean", "entropy_mean"):
+        assert rel(res[k], ref[k]) <= LOSS_RTOL or abs(res[k] - ref[k]) < 1e-9, (k, res[k], ref[k])
+    assert res["n_tokens"] == T
+    # tokens whose ratio sits on a clip bound to within fp32 rounding may fall on either side
+    rho = ref["rho"]
+    near = (np.abs(rho - (1 - clip_lo)) < 1e-5) | (np.abs(rho - (1 + clip_hi)) < 1e-5)
+    assert abs(res["clip_frac"] - ref["clip_frac"]) <= (near.sum() + 0.5) / max(T, 1) + 1e-7
+    ok = ~near
+    scale = np.abs(ref["dlogp"]).max() if T else 1.0
+    assert np.abs(g[ok] - ref["dlogp"][ok]).max(initial=0.0) <= 1e-5 * scale + 1e-12
+
+
+@pytest.mark.parametrize("name", ["cfg1", "cfg2_mini", "cfg3_mini", "cfg5_mini"])
+@pytest.mark.parametrize("agg_mode", [0, 1])
+def test_loss_on_workload_batches(ctx, name, agg_mode):
+    w = wl.make_workload(name)
+    r = np_of(wl.gen_reward(w))
+    adv = O.grpo_advantage_ref(r, w.group_id, w.n_prompts)
+    for mb in wl.microbatches(w)[:4]:
+        lens = w.lengths[mb]
+        cu = np.concatenate([[0], np.cumsum(lens)])
+        T = int(cu[-1])
+        logp, old, ref, ent = loss_inputs(w, T, lens)
+        kw = dict(clip_lo=w.clip_eps, clip_hi=w.clip_eps, kl_coef=w.kl_coef, agg_mode=agg_mode, loss_scale=1.0)
+        res, g = run_loss(ctx, logp, old, ref, ent, adv[mb], cu, **kw)
+        oref = O.policy_loss_ref(logp.numpy(), old.numpy(), ref.numpy(), adv[mb].astype(np.float32), cu,
+                                 entropy=ent.numpy(), **kw)
+        compare_loss(res, g, oref, T)
+        assert 0.0 < oref["clip_frac"] < 0.9 or name == "cfg1"
+    assert ctx.check_device_errors() == 0
+
+
+@pytest.mark.parametrize("lens", [[1], [4], [1, 1, 1], [1023, 1, 1024, 2, 1025], [5, 0, 7, 0, 0, 3], [4097], [3] * 700])
+def test_loss_ragged_and_tiny_sequences(ctx, lens):
+    w = wl.make_workload("cfg1")
+    cu = np.concatenate([[0], np.cumsum(lens)])
+    T = int(cu[-1])
+    logp, old, ref, ent = loss_inputs(w, T, lens, seed_shift=17)
+    A = np_of(wl.normal01(5, wl.S_MISC, 0, len(lens)))
+    for agg_mode in (0, 1):
+        kw = dict(clip_lo=0.2, clip_hi=0.28, kl_coef=0.04, agg_mode=agg_mode, loss_scale=0.5)
+        res, g = run_loss(ctx, logp, old, ref, None, A, cu, **kw)
+        oref = O.policy_loss_ref(logp.numpy(), old.numpy(), ref.numpy(), A, cu, **kw)
+        compare_loss(res, g, oref, T, 0.2, 0.28)
+        assert res["entropy_mean"] == 0.0
+
+
+def test_loss_identities_on_device(ctx):
+    w = wl.make_workload("cfg2_mini")
+    lens = w.lengths[:16]
+    cu = np.concatenate([[0], np.cumsum(lens)])
+    T = int(cu[-1])
+    logp, old, ref, ent = loss_inputs(w, T, lens)
+    A = np_of(wl.normal01(6, wl.S_MISC, 0, 16))
+    # old == current: ratio 1, nothing clipped, pg loss = -mean advantage; ref == current: no KL
+    res, g = run_loss(ctx, logp, logp, logp, ent, A, cu, kl_coef=0.04)
+    assert res["clip_frac"] == 0.0 and res["kl_mean"] == 0.0
+    assert rel(res["pg_loss"], -float(np.mean(A.astype(np.float64)))) <= 1e-5
+    # empty batch
+    res0, _ = run_loss(ctx, logp[:0], old[:0], ref[:0], None, A[:0], [0])
+    assert res0["loss"] == 0.0 and res0["n_tokens"] == 0
+    # run-to-run bitwise reproducibility
+    r1, g1 = run_loss(ctx, logp, old, ref, ent, A, cu)
+    r2, g2 = run_loss(ctx, logp, old, ref, ent, A, cu)
+    assert r1 == r2 and g1.tobytes() == g2.tobytes()
+
+
+def test_loss_bad_cu_seqlens_is_flagged(ctx):
+    from paper_2507_01663_b200 import binding as B
+    w = wl.make_workload("cfg1")
+    logp, old, ref, ent = loss_inputs(w, 64, [64])
+    run_loss(ctx, logp, old, ref, None, [1.0, 1.0], [0, 32, 60])      # cu[B] != T
+    assert ctx.check_device_errors() & B.DEVERR_CU_SEQLENS
+    assert ctx.check_device_errors() == 0

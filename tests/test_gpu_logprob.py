@@ -1,0 +1,146 @@
+"""af_token_logprob against the fp64 oracle, element by element."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import grpo_oracle as O
+from paper_2507_01663_b200 import workloads as wl
+from gpu_util import LOGP_TOL, device, np_of
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    from paper_2507_01663_b200 import binding as B
+    c = B.Context(0)
+    yield c
+    c.close()
+
+
+def run_case(ctx, H, W, y, splits=0):
+    dev = device()
+    T = H.shape[0]
+    Hd, Wd, yd = H.to(dev), W.to(dev), y.to(dev)
+    logp, ent, lse = (torch.full((T,), 9.0, device=dev) for _ in range(3))
+    ctx.set_tuning(splits, 0)
+    ctx.token_logprob(Hd, Wd, yd, logp, ent, lse)
+    flags = ctx.check_device_errors()
+    ctx.set_tuning(0, 0)
+    return np_of(logp), np_of(ent), np_of(lse), flags
+
+
+def random_case(T, d, V, seed, w_scale=None):
+    H = wl._normal_matrix(seed, wl.S_HIDDEN, T, d, 1.0, "cpu")
+    W = wl._normal_matrix(seed, wl.S_W, V, d, w_scale if w_scale else 1.0 / math.sqrt(d), "cpu")
+    y = wl.randint(seed, wl.S_TARGET, 0, T, V).to(torch.int32)
+    return H, W, y
+
+
+def check(ctx, H, W, y, splits=0):
+    logp, ent, lse, flags = run_case(ctx, H, W, y, splits)
+    r_logp, r_ent, r_lse = O.token_logprob_ref(wl.bf16_bits(H), wl.bf16_bits(W), y.numpy())
+    assert flags == 0
+    assert np.abs(logp - r_logp).max() <= LOGP_TOL
+    assert np.abs(ent - r_ent).max() <= LOGP_TOL
+    assert np.abs(lse - r_lse).max() <= LOGP_TOL
+
+
+def test_cfg1_full(ctx):
+    w = wl.make_workload("cfg1")
+    check(ctx, wl.gen_hidden(w), wl.gen_weight(w), wl.gen_target(w))
+
+
+@pytest.mark.parametrize("name", ["cfg2_mini", "cfg3_mini", "cfg5_mini"])
+def test_mini_workloads(ctx, name):
+    w = wl.make_workload(name)
+    check(ctx, wl.gen_hidden(w), wl.gen_weight(w), wl.gen_target(w))
+
+
+# T spans one row, a ragged tile, several tiles; V below / across / ragged past the 256-wide tile;
+# d below, equal to and ragged past the 64-wide K block (d % 8 == 0 is the ABI's requirement)
+@pytest.mark.parametrize("T,d,V", [(1, 8, 2), (5, 8, 10), (127, 64, 255), (128, 64, 256), (129, 72, 257),
+                                   (300, 200, 1000), (777, 512, 8200), (1025, 1096, 3001), (2100, 3584, 2304)])
+def test_shapes(ctx, T, d, V):
+    check(ctx, *random_case(T, d, V, seed=T + d + V))
+
+
+@pytest.mark.parametrize("splits", [1, 2, 3, 7, 16])
+def test_vocabulary_split_counts_agree(ctx, splits):
+    H, W, y = random_case(600, 256, 5000, seed=42)
+    check(ctx, H, W, y, splits)
+
+
+def test_targets_at_tile_and_split_edges(ctx):
+    T, d, V = 512, 128, 2050
+    H, W, _ = random_case(T, d, V, seed=7)
+    edges = [0, 31, 32, 255, 256, 257, 511, 512, 1023, 1024, 1025, 2047, 2048, 2049]
+    y = torch.tensor([edges[i % len(edges)] for i in range(T)], dtype=torch.int32)
+    for splits in (1, 4, 9):
+        check(ctx, H, W, y, splits)
+
+
+def test_degenerate_distributions(ctx):
+    T, d, V = 130, 64, 700
+    H, _, y = random_case(T, d, V, seed=3)
+    # zero weights: uniform distribution, logp = -ln V, entropy = ln V
+    logp, ent, lse, flags = run_case(ctx, H, torch.zeros(V, d, dtype=torch.bfloat16), y)
+    assert flags == 0 and np.abs(logp + math.log(V)).max() < 1e-5 and np.abs(ent - math.log(V)).max() < 1e-5
+    # one dominant logit (|z| ~ 500): logp -> 0 at the winner, very negative elsewhere, entropy -> 0
+    Hd = torch.full((T, d), 1.0, dtype=torch.bfloat16)
+    Wd = torch.zeros(V, d, dtype=torch.bfloat16)
+    Wd[5] = 8.0
+    yd = torch.full((T,), 5, dtype=torch.int32)
+    yd[1::2] = 6
+    check(ctx, Hd, Wd, yd)
+    # large negative and positive logits together, identical rows give identical results
+    Wm = wl._normal_matrix(5, wl.S_W, V, d, 1.5, "cpu")
+    Hs = H[:1].repeat(T, 1).contiguous()
+    logp, ent, lse, _ = run_case(ctx, Hs, Wm, torch.full((T,), 9, dtype=torch.int32))
+    assert np.all(logp == logp[0]) and np.all(ent == ent[0])
+    check(ctx, Hs, Wm, torch.full((T,), 9, dtype=torch.int32))
+
+
+def test_target_out_of_range_is_flagged_not_faulted(ctx):
+    from paper_2507_01663_b200 import binding as B
+    H, W, y = random_case(200, 64, 300, seed=11)
+    y[3] = 300
+    y[150] = -1
+    logp, ent, lse, flags = run_case(ctx, H, W, y)
+    assert flags & B.DEVERR_TARGET_RANGE
+    assert np.isnan(logp[3]) and np.isnan(logp[150]) and np.isfinite(np.delete(logp, [3, 150])).all()
+    y[3], y[150] = 0, 1
+    r = O.token_logprob_ref(wl.bf16_bits(H), wl.bf16_bits(W), y.numpy())
+    assert np.abs(np.delete(logp, [3, 150]) - np.delete(r[0], [3, 150])).max() <= LOGP_TOL
+    assert np.abs(ent - r[1]).max() <= LOGP_TOL           # entropy does not depend on the target
+    assert ctx.check_device_errors() == 0                 # the word is cleared by the read
+
+
+def test_host_argument_errors(ctx):
+    from paper_2507_01663_b200.binding import AfError
+    dev = device()
+    H = torch.zeros(4, 12, dtype=torch.bfloat16, device=dev)     # d % 8 != 0
+    W = torch.zeros(16, 12, dtype=torch.bfloat16, device=dev)
+    y = torch.zeros(4, dtype=torch.int32, device=dev)
+    out = torch.zeros(4, device=dev)
+    with pytest.raises(AfError) as e:
+        ctx.token_logprob(H, W, y, out)
+    assert e.value.status == -3
+    H8 = torch.zeros(4, 16, dtype=torch.bfloat16, device=dev)
+    W8 = torch.zeros(16, 16, dtype=torch.bfloat16, device=dev)
+    buf = torch.zeros(4 * 16 + 8, dtype=torch.bfloat16, device=dev)
+    with pytest.raises(AfError) as e:
+        ctx.token_logprob(buf[4:4 + 64].view(4, 16), W8, y, out)   # base pointer 8 bytes off
+    assert e.value.status == -3
+    ctx.token_logprob(H8, W8, y, out, T=0)                        # empty batch is a no-op
+    assert ctx.check_device_errors() == 0
+
+
+def test_bitwise_reproducible(ctx):
+    H, W, y = random_case(900, 256, 4096, seed=21)
+    a = run_case(ctx, H, W, y)
+    b = run_case(ctx, H, W, y)
+    for x, z in zip(a[:3], b[:3]):
+        assert x.tobytes() == z.tobytes()
