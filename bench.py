@@ -348,7 +348,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2")
-    ap.add_argument("--cpu-sample", type=int, default=256, help="tokens in the CPU-oracle sample")
+    ap.add_argument("--cpu-sample", type=int, default=1536, help="tokens in the CPU-oracle sample")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
