@@ -214,6 +214,36 @@ af_status af_policy_loss_backward(af_ctx* ctx, const void* hidden, const void* W
                                   int64_t T, int32_t d, int32_t V, void* d_hidden, float* d_W,
                                   int32_t accumulate_dW, void* stream);
 
+/* ---------------------------------------------------------------------------------------------
+ * af_token_logprob_static -- af_token_logprob for callers that are not allowed to allocate.
+ *
+ * (The paper has no counterpart for this call; it exists for the sake of embedding.)  Some hosts
+ * of this library cannot call cudaMalloc on the path that scores tokens: code running while a
+ * memory pool owns the whole device, a serving loop with a frozen memory plan, a plug-in handed
+ * only the buffers its caller chose to give it.  For them this entry point computes exactly what
+ * af_token_logprob computes -- same kernels, same arguments, same results -- but takes no
+ * context and keeps its only scratch (the per-split online-softmax partials) in a fixed array
+ * inside the library's device image: 2 MiB + 256 B that every GPU loading the library holds
+ * until the process exits.  It never calls cudaMalloc, cudaFree or an allocating library routine.
+ *
+ * Limit: 0 <= T <= 32768 tokens per call (AF_ERR_CAPACITY above that); d, V, pointers and
+ * alignment as for af_token_logprob.  Runs on the current CUDA device, which must be compute
+ * capability 10.0.
+ * First call on a device: resolves the array's device address, reads the SM count, fetches the
+ * tensor-map encoder and sets the kernel's shared-memory limit (and, with lazy module loading,
+ * loads the kernels).  Make that first call before any stream capture begins.
+ * Sharing: every call on a device uses the same array.  Nothing in it has to start at zero (a
+ * call overwrites each partial before reading it, so stale contents of an earlier call are
+ * harmless), but two calls that overlap on the GPU -- different streams, no ordering -- race on
+ * it and corrupt each other's results.  Serialise them (one stream, or events).
+ * device_flags: optional device pointer to a caller-owned uint32 that receives the AF_DEVERR_*
+ * bits (OR-ed in; clear it yourself).  With NULL the bits are dropped; a target outside [0, V)
+ * still shows as a NaN log-prob.
+ * ------------------------------------------------------------------------------------------- */
+af_status af_token_logprob_static(const void* hidden, const void* W, const int32_t* target,
+                                  int64_t T, int32_t d, int32_t V, float* logp, float* entropy,
+                                  float* lse, uint32_t* device_flags, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

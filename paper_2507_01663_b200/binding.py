@@ -25,7 +25,7 @@ DEVERR_TARGET_RANGE, DEVERR_WATCHDOG, DEVERR_CU_SEQLENS = 1, 2, 4
 
 EXPORTS = ["af_create", "af_destroy", "af_status_string", "af_reserve", "af_workspace_bytes",
            "af_set_tuning", "af_check_device_errors", "af_pack_microbatch", "af_token_logprob",
-           "af_grpo_advantage", "af_policy_loss", "af_policy_loss_backward"]
+           "af_grpo_advantage", "af_policy_loss", "af_policy_loss_backward", "af_token_logprob_static"]
 
 
 class AfError(RuntimeError):
@@ -87,6 +87,7 @@ def load_library() -> C.CDLL:
     lib.af_policy_loss.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i64, C.POINTER(LossParams), vp,
                                    vp, vp]
     lib.af_policy_loss_backward.argtypes = [vp, vp, vp, vp, vp, vp, i64, i32, i32, vp, vp, i32, vp]
+    lib.af_token_logprob_static.argtypes = [vp, vp, vp, i64, i32, i32, vp, vp, vp, vp, vp]
     for name in EXPORTS:
         if name not in ("af_status_string", "af_workspace_bytes"):
             getattr(lib, name).restype = C.c_int
@@ -218,3 +219,16 @@ def read_loss_out(buf: torch.Tensor) -> dict:
     raw = buf.cpu().numpy().tobytes()
     o = LossOut.from_buffer_copy(raw)
     return {k: getattr(o, k) for k, _ in LossOut._fields_ if k != "reserved"}
+
+
+def token_logprob_static(hidden, W, target, logp, entropy=None, lse=None, device_flags=None, T=None,
+                         stream=None):
+    """``af_token_logprob_static``: the scoring call without a context and without any allocation
+    (scratch is a fixed array inside the library; at most 32768 tokens per call).  Runs on the
+    current CUDA device; calls sharing a device must not overlap on the GPU."""
+    lib = load_library()
+    T = hidden.shape[0] if T is None else T
+    d, V = W.shape[1], W.shape[0]
+    _check(lib.af_token_logprob_static(_ptr(hidden), _ptr(W), _ptr(target), T, d, V, _ptr(logp),
+                                       _ptr(entropy), _ptr(lse), _ptr(device_flags), _stream(stream)),
+           "af_token_logprob_static")

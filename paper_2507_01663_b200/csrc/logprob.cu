@@ -6,6 +6,8 @@
 // in registers.  A unit covers one of S vocabulary ranges; the S partial states of a token are
 // written to the workspace and combined by merge_partials_kernel:
 //   lse = M + log sum_i s_i e^{m_i - M},  logp = zy - lse,  entropy = lse - (sum_i u_i e^{m_i-M}) / S.
+#include <mutex>
+
 #include "common.cuh"
 #include "umma.cuh"
 
@@ -149,3 +151,126 @@ af_status launch_token_logprob(af_ctx* ctx, const void* hidden, const void* W,
 }
 
 }  // namespace af
+
+// =============================================================================================
+// af_token_logprob_static -- the same scoring call for callers that must not allocate.
+//
+// The online-softmax partials normally live in the context's cudaMalloc'ed workspace.  Here they
+// live in a fixed array that is part of the library's device image, so the call needs no
+// context and performs no allocation of its own.  The array's name is only a host-side handle
+// in host code: its device address is looked up once per device with cudaGetSymbolAddress and
+// that pointer is what the kernels receive.
+// =============================================================================================
+namespace af {
+namespace {
+
+constexpr int64_t kStaticMaxTokens = 32768;                       // largest T the call accepts
+constexpr int64_t kStaticPartialSlots = 4 * kStaticMaxTokens;     // float4 slots: splits x tokens
+constexpr size_t kStaticHeaderBytes = 256;                        // private error word lives here
+constexpr size_t kStaticScratchBytes = kStaticHeaderBytes + (size_t)kStaticPartialSlots * sizeof(float4);
+
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];   // 2 MiB + 256 B
+
+constexpr int kStaticMaxDevices = 64;
+struct StaticDeviceState {
+  bool ready = false;
+  unsigned char* scratch = nullptr;  // device address of g_static_scratch on this device
+  int sm_count = 0;
+};
+StaticDeviceState g_static_state[kStaticMaxDevices];
+EncodeTiledFn g_static_encode = nullptr;
+std::mutex g_static_mutex;
+
+// Once per device, with that device current: resolve the scratch address, read the SM count,
+// fetch the tensor-map encoder and raise the kernel's dynamic shared memory limit.
+af_status static_setup(int dev, StaticDeviceState** out) {
+  if (dev < 0 || dev >= kStaticMaxDevices) return AF_ERR_UNSUPPORTED_DEVICE;
+  std::lock_guard<std::mutex> lock(g_static_mutex);
+  StaticDeviceState& st = g_static_state[dev];
+  if (!st.ready) {
+    int major = 0, minor = 0, sms = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&minor, cudaDevAttrComputeCapabilityMinor, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+      return AF_ERR_CUDA;
+    if (major != 10 || minor != 0) return AF_ERR_UNSUPPORTED_DEVICE;
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) {
+      cudaGetLastError();
+      return AF_ERR_CUDA;
+    }
+    if (!g_static_encode) {
+      void* fn = nullptr;
+      cudaDriverEntryPointQueryResult qres;
+      if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+          qres != cudaDriverEntryPointSuccess || !fn)
+        return AF_ERR_CUDA;
+      g_static_encode = reinterpret_cast<EncodeTiledFn>(fn);
+    }
+    if (cudaFuncSetAttribute(umma::gemm_kernel<LogprobEpi>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             umma::kSmemBytes) != cudaSuccess)
+      return AF_ERR_CUDA;
+    st.scratch = static_cast<unsigned char*>(p);
+    st.sm_count = sms;
+    st.ready = true;
+  }
+  *out = &st;
+  return AF_OK;
+}
+
+af_status static_encode_2d(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols,
+                           uint32_t box_rows) {
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {cols * 2};
+  cuuint32_t box[2] = {64, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return g_static_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides,
+                         box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                         CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS
+             ? AF_OK : AF_ERR_CUDA;
+}
+
+}  // namespace
+}  // namespace af
+
+extern "C" af_status af_token_logprob_static(const void* hidden, const void* W, const int32_t* target,
+                                             int64_t T, int32_t d, int32_t V, float* logp,
+                                             float* entropy, float* lse, uint32_t* device_flags,
+                                             void* stream) {
+  using namespace af;
+  if (T < 0 || d < 1 || V < 1) return AF_ERR_INVALID_ARG;
+  if (T > kStaticMaxTokens) return AF_ERR_CAPACITY;   // the fixed scratch holds 32768 tokens at most
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return AF_ERR_CUDA;
+  StaticDeviceState* st = nullptr;
+  af_status rc = static_setup(dev, &st);
+  if (rc != AF_OK) return rc;
+  if (T == 0) return AF_OK;
+  if (!hidden || !W || !target || !logp) return AF_ERR_INVALID_ARG;
+  if (d % 8 != 0 || (reinterpret_cast<uintptr_t>(hidden) & 15u) || (reinterpret_cast<uintptr_t>(W) & 15u))
+    return AF_ERR_ALIGNMENT;
+
+  int S = logprob_pick_splits(T, V, st->sm_count, 0);
+  if ((int64_t)S * T > kStaticPartialSlots) S = (int)(kStaticPartialSlots / T);
+  unsigned int* err_word = device_flags ? device_flags : reinterpret_cast<unsigned int*>(st->scratch);
+  float4* partial = reinterpret_cast<float4*>(st->scratch + kStaticHeaderBytes);
+
+  CUtensorMap ta, tb;
+  if ((rc = static_encode_2d(&ta, hidden, (uint64_t)T, (uint64_t)d, umma::kBM)) != AF_OK) return rc;
+  if ((rc = static_encode_2d(&tb, W, (uint64_t)V, (uint64_t)d, umma::kBN)) != AF_OK) return rc;
+  umma::GemmShape g;
+  g.M = (int)T; g.N = V; g.K = d;
+  g.m_tiles = (int)((T + umma::kBM - 1) / umma::kBM);
+  g.n_tiles = (V + umma::kBN - 1) / umma::kBN;
+  g.splits = S;
+  g.k_blocks = (d + umma::kBK - 1) / umma::kBK;
+  LogprobEpi::Params ep{target, partial, (int)T, V};
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const int64_t units = (int64_t)g.m_tiles * S;
+  const int grid = (int)(units < st->sm_count ? units : st->sm_count);
+  umma::gemm_kernel<LogprobEpi><<<grid, umma::kThreads, umma::kSmemBytes, s>>>(ta, tb, g, ep, err_word);
+  if (cudaGetLastError() != cudaSuccess) return AF_ERR_CUDA;
+  merge_partials_kernel<<<(int)((T + 255) / 256), 256, 0, s>>>(partial, target, (int)T, V, S, logp, entropy,
+                                                              lse, err_word);
+  return cudaGetLastError() == cudaSuccess ? AF_OK : AF_ERR_CUDA;
+}
