@@ -1,8 +1,10 @@
 // af_grpo_advantage kernels: adv_i = (r_i - mean_g) / (std_g + eps) within each prompt's group.
 //
-// Contiguous groups (group_id == NULL): a block stages a run of whole groups in shared memory
-// with 128-bit loads, reduces each group with warp shuffles (two passes: mean, then squared
-// deviations), and writes the advantages back coalesced -- 4 B read + 4 B written per sample.
+// Contiguous groups (group_id == NULL), 4 B read + 4 B written per sample:
+//   G <= 32 (every GRPO workload here except the 64-wide store): one thread per group, registers;
+//   G <= 4096: a block stages a run of whole groups in shared memory with 128-bit loads, reduces
+//   each group with warp shuffles (two passes: mean, then squared deviations) and writes the
+//   advantages back coalesced;  larger groups: one block per group.
 // Arbitrary membership (group_id given): one block per group scans the id array; sums are taken
 // in a fixed thread/iteration order, so the result is reproducible without float atomics.
 #include "common.cuh"
@@ -32,6 +34,54 @@ __device__ __forceinline__ double inv_scale(double ssq, int64_t n, int ddof, flo
   const int64_t denom = n - ddof;
   const double sigma = denom > 0 ? sqrt(ssq / (double)denom) : 0.0;
   return 1.0 / (sigma + (double)eps);
+}
+
+// Small contiguous groups (G <= 32): one thread per group.  A thread reads its group's G
+// consecutive rewards into registers (128-bit loads when G % 4 == 0), takes the two sums in fp64
+// and writes G advantages back; adjacent threads own adjacent groups, so a warp covers one
+// contiguous 32*G*4-byte span -- no shared memory, no shuffles, no barriers.
+constexpr int kSmallG = 32;
+template <int kCap>  // kCap = 4, 8, 16 or 32 >= G: bounds the register array
+__global__ void __launch_bounds__(kThreads) advantage_small_group_kernel(
+    const float* __restrict__ reward, float* __restrict__ adv, int64_t n_groups, int G, float eps,
+    int ddof, int vec_ok) {
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < n_groups; g += stride) {
+    const float* src = reward + g * G;
+    float* dst = adv + g * G;
+    float r[kCap];
+    if (vec_ok) {
+#pragma unroll
+      for (int q = 0; q < kCap / 4; ++q) {
+        if (q * 4 < G) {
+          const float4 v = __ldg(reinterpret_cast<const float4*>(src) + q);
+          r[q * 4 + 0] = v.x; r[q * 4 + 1] = v.y; r[q * 4 + 2] = v.z; r[q * 4 + 3] = v.w;
+        }
+      }
+    } else {
+#pragma unroll
+      for (int k = 0; k < kCap; ++k) if (k < G) r[k] = __ldg(src + k);
+    }
+    double s = 0.0;
+#pragma unroll
+    for (int k = 0; k < kCap; ++k) if (k < G) s += (double)r[k];
+    const double mu = s / (double)G;
+    double q2 = 0.0;
+#pragma unroll
+    for (int k = 0; k < kCap; ++k) if (k < G) { const double dv = (double)r[k] - mu; q2 += dv * dv; }
+    const double inv = inv_scale(q2, G, ddof, eps);
+#pragma unroll
+    for (int k = 0; k < kCap; ++k) if (k < G) r[k] = (float)(((double)r[k] - mu) * inv);
+    if (vec_ok) {
+#pragma unroll
+      for (int q = 0; q < kCap / 4; ++q)
+        if (q * 4 < G)
+          reinterpret_cast<float4*>(dst)[q] = make_float4(r[q * 4 + 0], r[q * 4 + 1], r[q * 4 + 2], r[q * 4 + 3]);
+    } else {
+#pragma unroll
+      for (int k = 0; k < kCap; ++k) if (k < G) dst[k] = r[k];
+    }
+  }
 }
 
 // Groups of equal size G, G <= kStage: each block iteration owns `gpb` whole groups.
@@ -135,7 +185,20 @@ cudaError_t launch_advantage(const float* reward, const int32_t* group_id, int64
   if (N == 0 || n_groups == 0) return cudaSuccess;
   if (group_id == nullptr) {
     const int64_t G = N / n_groups;
-    if (G <= kStage && G >= 1) {
+    if (G >= 1 && G <= kSmallG) {
+      const int vec_ok = (G % 4 == 0) && ((reinterpret_cast<uintptr_t>(reward) & 15) == 0) &&
+                         ((reinterpret_cast<uintptr_t>(adv) & 15) == 0);
+      int64_t blocks = (n_groups + kThreads - 1) / kThreads;
+      if (blocks > (int64_t)sm_count * 8) blocks = (int64_t)sm_count * 8;
+      if (G <= 4)
+        advantage_small_group_kernel<4><<<(int)blocks, kThreads, 0, s>>>(reward, adv, n_groups, (int)G, eps_adv, ddof, vec_ok);
+      else if (G <= 8)
+        advantage_small_group_kernel<8><<<(int)blocks, kThreads, 0, s>>>(reward, adv, n_groups, (int)G, eps_adv, ddof, vec_ok);
+      else if (G <= 16)
+        advantage_small_group_kernel<16><<<(int)blocks, kThreads, 0, s>>>(reward, adv, n_groups, (int)G, eps_adv, ddof, vec_ok);
+      else
+        advantage_small_group_kernel<32><<<(int)blocks, kThreads, 0, s>>>(reward, adv, n_groups, (int)G, eps_adv, ddof, vec_ok);
+    } else if (G <= kStage && G >= 1) {
       int gpb = (int)(kStage / G);
       // keep every SM busy before making block iterations large
       const int64_t want = (n_groups + (int64_t)sm_count * 4 - 1) / ((int64_t)sm_count * 4);

@@ -273,7 +273,7 @@ af_status af_policy_loss(af_ctx* c, const float* logp, const float* old_logp, co
   if (!c || !params || !out || !cu_seqlens || B < 0 || T < 0) return AF_ERR_INVALID_ARG;
   if (T > 0 && (!logp || !old_logp || !ref_logp || !adv_seq || B < 1)) return AF_ERR_INVALID_ARG;
   if (params->agg_mode != 0 && params->agg_mode != 1) return AF_ERR_INVALID_ARG;
-  if (T >= ((int64_t)1 << 31)) return AF_ERR_SHAPE;
+  if (T > ((int64_t)1 << 31) - 65536) return AF_ERR_SHAPE;  // token indices are 32-bit in the kernel
   DeviceGuard guard(c->device);
   return launch_policy_loss(logp, old_logp, ref_logp, entropy, adv_seq, cu_seqlens, B, T, *params, out,
                             dlogp, c->loss_ws.p, c->d_err, c->sm_count,
