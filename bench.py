@@ -34,6 +34,12 @@ from paper_2507_01663_b200 import workloads as wl  # noqa: E402
 METRIC = "scored tokens/sec (logprob+GRPO loss) at Qwen-7B head; % dense-BF16 peak"
 UNIT = "tokens/s"
 KERNELS_PER_STEP = 6  # advantage, pack columns, pack rows, fused LM-head GEMM, partial merge, loss
+# DRAM bytes per scored token of the fused LM-head kernel (dram__bytes_read + dram__bytes_write of
+# one ncu capture at T = 65536, d = 3584, V = 152064: 15.812 GB + 10.5 MB; traffic grows with the
+# number of 37-row-tile waves, i.e. in proportion to T).  Valid for the 7B head shape only; set to
+# None whenever the kernel changes until it is captured again.
+GEMM_DRAM_BYTES_PER_TOKEN_7B = (15.812258e9 + 10.496e6) / 65536
+BWD_TOKEN_BLOCK = 9472  # the library's default backward block (3 GEMM launches per block + 2 transposes)
 
 
 # ------------------------------------------------------------------------------------------
@@ -99,6 +105,10 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def head_name(w) -> str:
+    return {(3584, 152064): "Qwen2.5-7B-shaped", (5120, 152064): "Qwen2.5-32B-shaped"}.get((w.d, w.V), "synthetic")
+
+
 def dist_env():
     return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
 
@@ -154,25 +164,79 @@ class ScoringJob:
         }
         self.logp, self.ent, self.lse, self.dlogp = (torch.empty(T, device=device) for _ in range(4))
         self.loss_out = B.new_loss_out(device)
-        self.ctx.reserve(T, w.N, w.d, w.V)
-        self.gemm_events = []
+        if w.backward:
+            self.d_hidden = torch.empty(T, w.d, dtype=torch.bfloat16, device=device)
+            self.d_W = torch.empty(w.V, w.d, device=device)
+        self.ctx.reserve(T, w.N, w.d, w.V, with_backward=w.backward)
+        self.gemm_events, self.pack_events, self.bwd_events = [], [], []
+        self.launches_per_step = KERNELS_PER_STEP + (2 + 3 * -(-T // BWD_TOKEN_BLOCK) if w.backward else 0)
 
     def step(self, time_gemm: bool = False):
         w, c = self.w, self.ctx
         c.grpo_advantage(self.reward, None, w.n_prompts, self.adv)
         store = {"tok_offset_host": self.off, "d": w.d, "adv": self.adv, **self.store}
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(6)] if time_gemm else None
+        if ev:
+            ev[0].record()
         T = c.pack_microbatch(store, self.idx, self.packed)
-        if time_gemm:
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
+        if ev:
+            ev[1].record()
+            ev[2].record()
         c.token_logprob(self.packed["hidden"], self.W, self.packed["target"], self.logp, self.ent, self.lse, T=T)
-        if time_gemm:
-            e1.record()
-            self.gemm_events.append((e0, e1))
+        if ev:
+            ev[3].record()
         c.policy_loss(self.logp, self.packed["old_logp"], self.packed["ref_logp"], self.packed["adv_seq"],
                       self.packed["cu_seqlens"], self.loss_out, self.dlogp, self.ent,
                       w.clip_eps, w.clip_eps, w.kl_coef, 0, 1.0, B=w.N, T=T)
+        if w.backward:
+            if ev:
+                ev[4].record()
+            c.policy_loss_backward(self.packed["hidden"], self.W, self.packed["target"], self.lse, self.dlogp,
+                                   self.d_hidden, self.d_W, False, T=T)
+            if ev:
+                ev[5].record()
+                self.bwd_events.append((ev[4], ev[5]))
+        if ev:
+            self.pack_events.append((ev[0], ev[1]))
+            self.gemm_events.append((ev[2], ev[3]))
         return T
+
+    def hbm_kernels_at_scale(self, peak_gbs: float) -> dict:
+        """Loss and advantage kernels at sizes where bandwidth, not launch latency, decides
+        (2^26 tokens / responses); the pack figure comes from the timed steps themselves."""
+        dev, c, B = self.dev, self.ctx, self.B
+        out = {}
+
+        def avg_ms(fn, n=10):
+            for _ in range(3):
+                fn()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(n):
+                fn()
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) / n
+
+        n = 1 << 26
+        seq = 1024
+        logp = wl.gen_surrogate_logp(self.w, 1 << 20, dev).repeat(n >> 20)
+        old, ref, ent = logp + 0.1, logp - 0.1, -logp
+        adv = wl.normal01(self.w.seed, wl.S_MISC, 0, n // seq, dev)
+        cu = torch.arange(n // seq + 1, device=dev, dtype=torch.int32) * seq
+        g, lo = torch.empty(n, device=dev), B.new_loss_out(dev)
+        ms = avg_ms(lambda: c.policy_loss(logp, old, ref, adv, cu, lo, g, ent))
+        gbs = 20.0 * n / ms / 1e6
+        out["policy_loss"] = {"tokens": n, "bytes_per_token": 20, "ms": ms, "gbs": gbs, "frac": gbs / peak_gbs}
+        del logp, old, ref, ent, g
+        r = wl.uniform01(self.w.seed, wl.S_REWARD, 0, 1 << 20, dev).repeat(n >> 20)
+        a = torch.empty(n, device=dev)
+        G = self.w.group_size if self.w.group_size <= 32 else 8
+        ms = avg_ms(lambda: c.grpo_advantage(r, None, n // G, a))
+        gbs = 8.0 * n / ms / 1e6
+        out["grpo_advantage"] = {"responses": n, "group_size": G, "bytes_per_response": 8, "ms": ms, "gbs": gbs,
+                                 "frac": gbs / peak_gbs}
+        return out
 
     # -- end-to-end: store columns start in pinned host memory ------------------------------
     def make_host_store(self):
@@ -257,6 +321,8 @@ def run_ours(args):
     ms_total = timed_loop(lambda: job.step(time_gemm=True), args.steps, world)
     clocks = sampler.stop() if rank == 0 else None
     gemm_ms = float(np.mean([a.elapsed_time(b) for a, b in job.gemm_events]))
+    pack_ms = float(np.mean([a.elapsed_time(b) for a, b in job.pack_events]))
+    bwd_ms = float(np.mean([a.elapsed_time(b) for a, b in job.bwd_events])) if job.bwd_events else None
     ms_step, tokens = reduce_over_ranks(ms_total / args.steps, job.T, world)
     flags = job.ctx.check_device_errors()
     if flags:
@@ -277,21 +343,35 @@ def run_ours(args):
         "metric": METRIC, "value": tokens / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": f"{args.workload}: Qwen2.5-7B-shaped head d={w.d} V={w.V}, {w.N} responses "
+        "config": {"workload": f"{args.workload}: {head_name(w)} head d={w.d} V={w.V}, {w.N} responses "
                                f"({w.n_prompts} prompts x {w.group_size}), {job.T} scored tokens per GPU, "
-                               "one arrival-ordered packed micro-batch",
+                               "one arrival-ordered packed micro-batch" + (", forward + backward (dH, dW)" if w.backward else ""),
                    "l2": "inputs (hidden states >> 126 MB L2) exceed L2; no flush needed",
                    "loss": {"clip_eps": w.clip_eps, "kl_coef": w.kl_coef, "agg": "seq-mean-token-mean"}},
         "roofline": {"bound": "tensor", "kernel": "fused LM-head GEMM + online log-softmax (af_token_logprob)",
                      "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
                      "peak_source": f"bf16_tflops_sustained, {peaks['source']}",
                      "frac_of_burst": achieved / peaks["bf16_tflops"], "frac_of_nominal_2250": achieved / 2250.0,
-                     "kernel_ms": gemm_ms, "traffic": None},
+                     "kernel_ms": gemm_ms,
+                     "traffic": (GEMM_DRAM_BYTES_PER_TOKEN_7B * job.T
+                                 if GEMM_DRAM_BYTES_PER_TOKEN_7B and (w.d, w.V) == (3584, 152064) else None)},
         "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": job.h2d_bytes,
                 "d2h_bytes_per_step": int(job.loss_out.numel()), "ms_per_step": ms_e2e},
-        "gpu_launches": KERNELS_PER_STEP * args.steps,
+        "gpu_launches": job.launches_per_step * args.steps,
         "clocks": clocks, "loss": loss,
     }
+    pack_bytes = 2.0 * job.T * (2 * w.d + 12) + 8.0 * w.N
+    pack_gbs = pack_bytes / (pack_ms * 1e-3) / 1e9
+    line["hbm_kernels"] = {"peak_gbs": peaks["hbm_gbs"], "peak_source": f"hbm_gbs, {peaks['source']}",
+                           "pack_microbatch": {"tokens": job.T, "bytes_per_token": 2 * (2 * w.d + 12), "ms": pack_ms,
+                                               "gbs": pack_gbs, "frac": pack_gbs / peaks["hbm_gbs"],
+                                               "where": "inside the timed steps (2 kernels + metadata copy)"}}
+    if bwd_ms is not None:
+        bflops = 6.0 * job.T * w.d * w.V
+        line["backward"] = {"ms": bwd_ms, "tflops": bflops / (bwd_ms * 1e-3) / 1e12, "flop_model": "6*T*d*V",
+                            "frac_of_sustained": bflops / (bwd_ms * 1e-3) / 1e12 / peak}
+    if rank == 0 and world == 1:
+        line["hbm_kernels"].update(job.hbm_kernels_at_scale(peaks["hbm_gbs"]))
     if rank == 0 and world == 1:
         n = args.cpu_sample
         rows = job.packed["hidden"][:n].cpu()
@@ -333,7 +413,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f64", "data": "synthetic",
-        "config": {"workload": f"{args.workload}: Qwen2.5-7B-shaped head d={w.d} V={w.V}; bounded sample: {sample}"},
+        "config": {"workload": f"{args.workload}: {head_name(w)} head d={w.d} V={w.V}; bounded sample: {sample}"},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,

@@ -205,8 +205,8 @@ af_status af_policy_loss(af_ctx* ctx, const float* logp, const float* old_logp,
  *   d_W[v,:]      = sum_t dZ_tv * hidden[t,:]     -> [V,d] fp32 (added to d_W if accumulate_dW)
  *
  * dZ is rounded to bf16 for the two tensor-core products (fp32 accumulation).  Tokens are
- * processed in blocks; the scratch (dZ of one block, transposed copies of W and hidden) lives
- * in the context's workspace and does not grow with T beyond the hidden copy.
+ * processed in blocks; the only scratch is the dZ of one block (token block x V bf16) in the
+ * context's workspace, independent of T.  No operand is transposed in memory.
  * Requirements: d % 8 == 0, V % 8 == 0, 16-byte aligned pointers, 0 <= T < 2^31.
  * ------------------------------------------------------------------------------------------- */
 af_status af_policy_loss_backward(af_ctx* ctx, const void* hidden, const void* W,

@@ -105,7 +105,7 @@ af_status af_destroy(af_ctx* c) {
   if (!c) return AF_ERR_INVALID_ARG;
   DeviceGuard guard(c->device);
   cudaDeviceSynchronize();
-  Buf* bufs[] = {&c->partial, &c->loss_ws, &c->pack_meta, &c->wt, &c->ht, &c->dz, &c->dzt};
+  Buf* bufs[] = {&c->partial, &c->loss_ws, &c->pack_meta, &c->dz};
   for (Buf* b : bufs) if (b->p) cudaFree(b->p);
   for (int i = 0; i < kPackRing; ++i) {
     if (c->pack_host[i]) cudaFreeHost(c->pack_host[i]);
@@ -118,8 +118,7 @@ af_status af_destroy(af_ctx* c) {
 
 int64_t af_workspace_bytes(const af_ctx* c) {
   if (!c) return 0;
-  return (int64_t)(c->partial.cap + c->loss_ws.cap + c->pack_meta.cap + c->wt.cap + c->ht.cap +
-                   c->dz.cap + c->dzt.cap);
+  return (int64_t)(c->partial.cap + c->loss_ws.cap + c->pack_meta.cap + c->dz.cap);
 }
 
 af_status af_set_tuning(af_ctx* c, int32_t v_splits, int32_t bwd_token_block) {

@@ -2,12 +2,17 @@
 //
 // Tokens are processed in blocks of Tc rows.  Per block, three tensor-core GEMMs built on the
 // same tcgen05 main loop:
-//   1. recompute  Z = H_blk W^T  and turn it, in the epilogue, into
-//        dZ = g_t (1{v = y_t} - exp(z - lse_t))   (bf16), written as dZ [Tc,V] and dZ^T [V,Tc];
-//   2. dH_blk = dZ  * W      ([Tc,V] x [V,d], K = V)  -> bf16, using W^T  [d,V] as the K-major B;
-//   3. dW    += dZ^T * H_blk ([V,Tc] x [Tc,d], K = Tc) -> fp32, using H^T [d,T] as the K-major B.
-// The scratch is one block of dZ (both orientations) plus transposed copies of W and H; [T,V] is
-// never materialised and the scratch does not grow with T (beyond the H^T copy).
+//   1. recompute  Z = H_blk W^T  (both operands K-major) and turn it, in the epilogue, into
+//        dZ = g_t (1{v = y_t} - exp(z - lse_t))   (bf16), written once as dZ [Tc, V];
+//   2. dH_blk = dZ * W        A = dZ [Tc,V] K-major,  B = W [V,d] read MN-major   -> bf16 [Tc, d];
+//   3. dW    += dZ^T * H_blk  A = dZ [Tc,V] and B = H_blk [Tc,d], both read MN-major -> fp32 [V, d].
+// No operand is ever transposed in memory.  The scratch is one block of dZ; [T,V] is never
+// materialised and the scratch does not grow with T.
+//
+// Epilogues hold one output row per lane (the TMEM load shape); storing that directly would write
+// 16 bytes to each of 32 different rows per instruction.  Each warp therefore passes its 32x32
+// chunk through a private, XOR-swizzled shared-memory buffer and stores whole 64/128-byte row
+// segments, four to eight rows per instruction.
 #include "common.cuh"
 #include "umma.cuh"
 
@@ -27,55 +32,43 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&h);
 }
 
-// ---- bf16 transpose: out[c, r] = in[r, c]; in [R, C] pitch ldi, out [C, R] pitch ldo ----------
-__global__ void __launch_bounds__(256) transpose_bf16_kernel(const __nv_bfloat16* __restrict__ in,
-                                                             __nv_bfloat16* __restrict__ out, int R,
-                                                             int C, int64_t ldi, int64_t ldo) {
-  __shared__ __nv_bfloat16 tile[64][66];
-  const int r0 = blockIdx.x * 64, c0 = blockIdx.y * 64;
-  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;  // 32 x 8
-  for (int i = ty; i < 64; i += 8) {
-    const int r = r0 + i, c = c0 + tx * 2;
-    __nv_bfloat16 a = __float2bfloat16(0.f), b = a;
-    if (r < R) {
-      if (c + 1 < C) {
-        const __nv_bfloat162 v = *reinterpret_cast<const __nv_bfloat162*>(in + (int64_t)r * ldi + c);
-        a = v.x; b = v.y;
-      } else if (c < C) {
-        a = in[(int64_t)r * ldi + c];
-      }
-    }
-    tile[i][tx * 2] = a; tile[i][tx * 2 + 1] = b;
+// Store a 32-row x 32-column bf16 chunk (lane L holds row L as 16 packed words) to a row-major
+// bf16 matrix: rows row0.., columns col0..; rows >= M and 8-column groups past N are skipped.
+// Staging layout: row r occupies 64 bytes = four 16-byte slots; slot q of row r lives at position
+// q ^ ((r >> 1) & 3), which makes both the row-per-lane writes and the 8-rows-per-instruction
+// reads free of bank conflicts.
+__device__ __forceinline__ void store_chunk_bf16(const uint32_t (&w)[16], uint8_t* stage, int lane,
+                                                 __nv_bfloat16* C, int64_t ldc, int row0, int col0,
+                                                 int M, int N) {
+  uint4* st = reinterpret_cast<uint4*>(stage);
+#pragma unroll
+  for (int q = 0; q < 4; ++q)
+    st[lane * 4 + (q ^ ((lane >> 1) & 3))] = make_uint4(w[q * 4 + 0], w[q * 4 + 1], w[q * 4 + 2], w[q * 4 + 3]);
+  __syncwarp();
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int r = i * 8 + (lane >> 2), c = lane & 3;
+    const uint4 v = st[r * 4 + (c ^ ((r >> 1) & 3))];
+    const int grow = row0 + r, gcol = col0 + c * 8;
+    if (grow < M && gcol + 8 <= N) *reinterpret_cast<uint4*>(C + (size_t)grow * ldc + gcol) = v;
   }
-  __syncthreads();
-  for (int i = ty; i < 64; i += 8) {
-    const int c = c0 + i, r = r0 + tx * 2;
-    if (c < C) {
-      if (r + 1 < R) {
-        __nv_bfloat162 v; v.x = tile[tx * 2][i]; v.y = tile[tx * 2 + 1][i];
-        *reinterpret_cast<__nv_bfloat162*>(out + (int64_t)c * ldo + r) = v;
-      } else if (r < R) {
-        out[(int64_t)c * ldo + r] = tile[tx * 2][i];
-      }
-    }
-  }
+  __syncwarp();
 }
 
-// ---- epilogue 1: logits tile -> dZ (both orientations) ----------------------------------------
+// ---- epilogue 1: logits tile -> dZ ----------------------------------------------------------------
 struct DzEpi {
   struct Params {
     const int32_t* target;  // [rows] of this block
     const float* lse;       // [rows]
     const float* g;         // [rows] dL/dlogp
     __nv_bfloat16* dz;      // [rows, V]
-    __nv_bfloat16* dzt;     // [V, ldzt]
     int rows, V;
-    int64_t ldzt;
   };
   struct State {
     float g, nl;
     int y;
   };
+  static constexpr bool kStaged = true;
   static __device__ __forceinline__ void unit_begin(State& st, const Params& p, int row, int, int) {
     if (row < p.rows) {
       st.g = __ldg(p.g + row);
@@ -86,8 +79,9 @@ struct DzEpi {
     }
   }
   static __device__ __forceinline__ void chunk(State& st, const Params& p, int row, int col0,
-                                               const uint32_t (&v)[32]) {
-    if (row >= p.rows || col0 >= p.V) return;
+                                               const uint32_t (&v)[32], uint8_t* stage) {
+    if (col0 >= p.V) return;                       // uniform across the warp
+    const int lane = threadIdx.x & 31;
     float dzv[32];
 #pragma unroll
     for (int j = 0; j < 32; ++j) {
@@ -99,29 +93,10 @@ struct DzEpi {
 #pragma unroll
       for (int j = 0; j < 32; ++j) if (j == yl) dzv[j] += st.g;
     }
-    __nv_bfloat16* drow = p.dz + (size_t)row * p.V + col0;
-    if (col0 + 32 <= p.V) {
+    uint32_t w[16];
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        uint4 w;
-        w.x = pack_bf16x2(dzv[q * 8 + 0], dzv[q * 8 + 1]);
-        w.y = pack_bf16x2(dzv[q * 8 + 2], dzv[q * 8 + 3]);
-        w.z = pack_bf16x2(dzv[q * 8 + 4], dzv[q * 8 + 5]);
-        w.w = pack_bf16x2(dzv[q * 8 + 6], dzv[q * 8 + 7]);
-        *reinterpret_cast<uint4*>(drow + q * 8) = w;
-      }
-#pragma unroll
-      for (int j = 0; j < 32; ++j) p.dzt[(size_t)(col0 + j) * p.ldzt + row] = __float2bfloat16_rn(dzv[j]);
-    } else {
-#pragma unroll
-      for (int j = 0; j < 32; ++j) {
-        if (col0 + j < p.V) {
-          const __nv_bfloat16 b = __float2bfloat16_rn(dzv[j]);
-          drow[j] = b;
-          p.dzt[(size_t)(col0 + j) * p.ldzt + row] = b;
-        }
-      }
-    }
+    for (int j = 0; j < 16; ++j) w[j] = pack_bf16x2(dzv[2 * j], dzv[2 * j + 1]);
+    store_chunk_bf16(w, stage, lane, p.dz, p.V, row - lane, col0, p.rows, p.V);
   }
   static __device__ __forceinline__ void unit_end(State&, const Params&, int, int) {}
 };
@@ -134,27 +109,22 @@ struct StoreBf16Epi {
     int M, N;
   };
   struct State {};
+  static constexpr bool kStaged = true;
   static __device__ __forceinline__ void unit_begin(State&, const Params&, int, int, int) {}
   static __device__ __forceinline__ void chunk(State&, const Params& p, int row, int col0,
-                                               const uint32_t (&v)[32]) {
-    if (row >= p.M || col0 >= p.N) return;
-    __nv_bfloat16* c = p.C + (size_t)row * p.ldc + col0;
+                                               const uint32_t (&v)[32], uint8_t* stage) {
+    if (col0 >= p.N) return;
+    const int lane = threadIdx.x & 31;
+    uint32_t w[16];
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      if (col0 + q * 8 + 8 <= p.N) {
-        uint4 w;
-        w.x = pack_bf16x2(__uint_as_float(v[q * 8 + 0]), __uint_as_float(v[q * 8 + 1]));
-        w.y = pack_bf16x2(__uint_as_float(v[q * 8 + 2]), __uint_as_float(v[q * 8 + 3]));
-        w.z = pack_bf16x2(__uint_as_float(v[q * 8 + 4]), __uint_as_float(v[q * 8 + 5]));
-        w.w = pack_bf16x2(__uint_as_float(v[q * 8 + 6]), __uint_as_float(v[q * 8 + 7]));
-        *reinterpret_cast<uint4*>(c + q * 8) = w;
-      }
-    }
+    for (int j = 0; j < 16; ++j) w[j] = pack_bf16x2(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
+    store_chunk_bf16(w, stage, lane, p.C, p.ldc, row - lane, col0, p.M, p.N);
   }
   static __device__ __forceinline__ void unit_end(State&, const Params&, int, int) {}
 };
 
 // ---- epilogue 3: accumulator tile -> fp32 matrix (store or add) ---------------------------------
+// Staging: row r = 128 bytes = eight 16-byte slots, slot q at position q ^ (r & 7).
 struct StoreF32Epi {
   struct Params {
     float* C;
@@ -163,47 +133,70 @@ struct StoreF32Epi {
     int accumulate;
   };
   struct State {};
+  static constexpr bool kStaged = true;
   static __device__ __forceinline__ void unit_begin(State&, const Params&, int, int, int) {}
   static __device__ __forceinline__ void chunk(State&, const Params& p, int row, int col0,
-                                               const uint32_t (&v)[32]) {
-    if (row >= p.M || col0 >= p.N) return;
-    float* c = p.C + (size_t)row * p.ldc + col0;
+                                               const uint32_t (&v)[32], uint8_t* stage) {
+    if (col0 >= p.N) return;
+    const int lane = threadIdx.x & 31;
+    const int row0 = row - lane;
+    uint4* st = reinterpret_cast<uint4*>(stage);
 #pragma unroll
-    for (int q = 0; q < 8; ++q) {
-      if (col0 + q * 4 + 4 <= p.N) {
-        float4 w = make_float4(__uint_as_float(v[q * 4 + 0]), __uint_as_float(v[q * 4 + 1]),
-                               __uint_as_float(v[q * 4 + 2]), __uint_as_float(v[q * 4 + 3]));
+    for (int q = 0; q < 8; ++q)
+      st[lane * 8 + (q ^ (lane & 7))] = make_uint4(v[q * 4 + 0], v[q * 4 + 1], v[q * 4 + 2], v[q * 4 + 3]);
+    __syncwarp();
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int r = i * 4 + (lane >> 3), c = lane & 7;
+      const uint4 u = st[r * 8 + (c ^ (r & 7))];
+      const int grow = row0 + r, gcol = col0 + c * 4;
+      if (grow < p.M && gcol + 4 <= p.N) {
+        float* dst = p.C + (size_t)grow * p.ldc + gcol;
+        float4 w = make_float4(__uint_as_float(u.x), __uint_as_float(u.y), __uint_as_float(u.z), __uint_as_float(u.w));
         if (p.accumulate) {
-          const float4 o = *reinterpret_cast<const float4*>(c + q * 4);
+          const float4 o = *reinterpret_cast<const float4*>(dst);
           w.x += o.x; w.y += o.y; w.z += o.z; w.w += o.w;
         }
-        *reinterpret_cast<float4*>(c + q * 4) = w;
+        *reinterpret_cast<float4*>(dst) = w;
       }
     }
+    __syncwarp();
   }
   static __device__ __forceinline__ void unit_end(State&, const Params&, int, int) {}
 };
 
-template <class E>
-af_status run_gemm(af_ctx* ctx, const void* A, uint64_t a_rows, uint64_t a_pitch, const void* B,
-                   uint64_t b_rows, uint64_t b_pitch, uint64_t K, int splits,
+// One operand of a GEMM launch: the matrix as it sits in memory.
+struct Operand {
+  const void* base;
+  uint64_t rows, cols;   // memory rows and (contiguous) columns
+  uint64_t pitch_bytes;
+};
+
+// C[M,N] = sum_k A(m,k) B(n,k).  A K-major operand is stored [M or N, K]; an MN-major operand is
+// stored [K, M or N].  Box: 64 contiguous elements wide; 128 / 256 rows for K-major A / B, 64
+// K-rows for MN-major.
+template <class E, bool kAMN, bool kBMN>
+af_status run_gemm(af_ctx* ctx, const Operand& A, const Operand& B, int splits,
                    const typename E::Params& ep, cudaStream_t s) {
   CUtensorMap ta, tb;
-  af_status st = encode_bf16_2d(ctx, &ta, A, a_rows, K, a_pitch, umma::kBM);
+  af_status st = encode_bf16_2d(ctx, &ta, A.base, A.rows, A.cols, A.pitch_bytes, kAMN ? 64 : umma::kBM);
   if (st != AF_OK) return st;
-  st = encode_bf16_2d(ctx, &tb, B, b_rows, K, b_pitch, umma::kBN);
+  st = encode_bf16_2d(ctx, &tb, B.base, B.rows, B.cols, B.pitch_bytes, kBMN ? 64 : umma::kBN);
   if (st != AF_OK) return st;
+  const uint64_t M = kAMN ? A.cols : A.rows, K = kAMN ? A.rows : A.cols;
+  const uint64_t N = kBMN ? B.cols : B.rows;
   umma::GemmShape g;
-  g.M = (int)a_rows; g.N = (int)b_rows; g.K = (int)K;
-  g.m_tiles = (int)((a_rows + umma::kBM - 1) / umma::kBM);
-  g.n_tiles = (int)((b_rows + umma::kBN - 1) / umma::kBN);
+  g.M = (int)M; g.N = (int)N; g.K = (int)K;
+  g.m_tiles = (int)((M + umma::kBM - 1) / umma::kBM);
+  g.n_tiles = (int)((N + umma::kBN - 1) / umma::kBN);
   g.splits = splits > 0 && splits < g.n_tiles ? splits : g.n_tiles;
   g.k_blocks = (int)((K + umma::kBK - 1) / umma::kBK);
-  if (cudaFuncSetAttribute(umma::gemm_kernel<E>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           umma::kSmemBytes) != cudaSuccess) return AF_ERR_CUDA;
+  constexpr int smem = E::kStaged ? umma::kSmemBytesStaged : umma::kSmemBytes;
+  if (cudaFuncSetAttribute(umma::gemm_kernel<E, kAMN, kBMN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           smem) != cudaSuccess) return AF_ERR_CUDA;
   const int64_t units = (int64_t)g.m_tiles * g.splits;
   const int grid = (int)(units < ctx->sm_count ? units : ctx->sm_count);
-  umma::gemm_kernel<E><<<grid, umma::kThreads, umma::kSmemBytes, s>>>(ta, tb, g, ep, ctx->d_err);
+  umma::gemm_kernel<E, kAMN, kBMN><<<grid, umma::kThreads, smem, s>>>(ta, tb, g, ep, ctx->d_err);
   return cudaGetLastError() == cudaSuccess ? AF_OK : AF_ERR_CUDA;
 }
 
@@ -215,13 +208,9 @@ af_status launch_backward(af_ctx* ctx, const void* hidden, const void* W, const 
   int64_t Tc = ctx->bwd_token_block > 0 ? ctx->bwd_token_block : kDefaultTokenBlock;
   const int64_t T_round = ((T + 127) / 128) * 128;
   if (Tc > T_round) Tc = T_round > 0 ? T_round : 128;
-  const int64_t T_pad = (T + 7) & ~(int64_t)7;
 
   af_status st;
-  if ((st = ws_grow(ctx->wt, (size_t)d * V * 2)) != AF_OK) return st;
-  if ((st = ws_grow(ctx->ht, (size_t)d * (T_pad > 0 ? T_pad : 8) * 2)) != AF_OK) return st;
   if ((st = ws_grow(ctx->dz, (size_t)Tc * V * 2)) != AF_OK) return st;
-  if ((st = ws_grow(ctx->dzt, (size_t)V * Tc * 2)) != AF_OK) return st;
   if (accumulate_dW < 0) return AF_OK;  // reserve only
 
   if (T == 0) {
@@ -229,36 +218,26 @@ af_status launch_backward(af_ctx* ctx, const void* hidden, const void* W, const 
     return AF_OK;
   }
   const __nv_bfloat16* H = static_cast<const __nv_bfloat16*>(hidden);
-  __nv_bfloat16* wt = static_cast<__nv_bfloat16*>(ctx->wt.p);
-  __nv_bfloat16* ht = static_cast<__nv_bfloat16*>(ctx->ht.p);
   __nv_bfloat16* dz = static_cast<__nv_bfloat16*>(ctx->dz.p);
-  __nv_bfloat16* dzt = static_cast<__nv_bfloat16*>(ctx->dzt.p);
-
-  {  // K-major copies of the two B operands
-    dim3 gw((V + 63) / 64, (d + 63) / 64);
-    transpose_bf16_kernel<<<gw, 256, 0, s>>>(static_cast<const __nv_bfloat16*>(W), wt, V, d, d, V);
-    dim3 gh((unsigned)((T + 63) / 64), (d + 63) / 64);
-    transpose_bf16_kernel<<<gh, 256, 0, s>>>(H, ht, (int)T, d, d, T_pad);
-    if (cudaGetLastError() != cudaSuccess) return AF_ERR_CUDA;
-  }
+  const uint64_t dB = (uint64_t)d * 2, vB = (uint64_t)V * 2;
 
   bool first = true;
   for (int64_t t0 = 0; t0 < T; t0 += Tc, first = false) {
-    const int64_t tc = (T - t0) < Tc ? (T - t0) : Tc;
-    // 1. dZ block
-    DzEpi::Params p1{target + t0, lse + t0, dlogp + t0, dz, dzt, (int)tc, V, Tc};
-    st = run_gemm<DzEpi>(ctx, H + t0 * d, (uint64_t)tc, (uint64_t)d * 2, W, (uint64_t)V, (uint64_t)d * 2,
-                         (uint64_t)d, logprob_pick_splits(tc, V, ctx->sm_count, ctx->v_splits), p1, s);
+    const uint64_t tc = (uint64_t)((T - t0) < Tc ? (T - t0) : Tc);
+    const Operand Hblk{H + t0 * d, tc, (uint64_t)d, dB};
+    const Operand Wop{W, (uint64_t)V, (uint64_t)d, dB};
+    const Operand dZop{dz, tc, (uint64_t)V, vB};
+    // 1. dZ block:  Z = H_blk W^T, both K-major
+    DzEpi::Params p1{target + t0, lse + t0, dlogp + t0, dz, (int)tc, V};
+    st = run_gemm<DzEpi, false, false>(ctx, Hblk, Wop, logprob_pick_splits((int64_t)tc, V, ctx->sm_count, ctx->v_splits), p1, s);
     if (st != AF_OK) return st;
-    // 2. dH block = dZ * W
+    // 2. dH block = dZ W:  A = dZ (K = v contiguous), B = W read MN-major (n = d contiguous, K = v rows)
     StoreBf16Epi::Params p2{static_cast<__nv_bfloat16*>(d_hidden) + t0 * d, d, (int)tc, d};
-    st = run_gemm<StoreBf16Epi>(ctx, dz, (uint64_t)tc, (uint64_t)V * 2, wt, (uint64_t)d, (uint64_t)V * 2,
-                                (uint64_t)V, 0, p2, s);
+    st = run_gemm<StoreBf16Epi, false, true>(ctx, dZop, Wop, 0, p2, s);
     if (st != AF_OK) return st;
-    // 3. dW += dZ^T * H block
+    // 3. dW += dZ^T H_blk:  A = dZ read MN-major (m = v contiguous, K = t rows), B = H_blk read MN-major
     StoreF32Epi::Params p3{d_W, d, V, d, (!first || accumulate_dW) ? 1 : 0};
-    st = run_gemm<StoreF32Epi>(ctx, dzt, (uint64_t)V, (uint64_t)Tc * 2, ht + t0, (uint64_t)d,
-                               (uint64_t)T_pad * 2, (uint64_t)tc, 0, p3, s);
+    st = run_gemm<StoreF32Epi, true, true>(ctx, dZop, Hblk, 0, p3, s);
     if (st != AF_OK) return st;
   }
   return AF_OK;

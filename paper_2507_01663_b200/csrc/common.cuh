@@ -39,10 +39,7 @@ struct af_ctx {
   af::Buf partial;    // [splits, T] float4 online-softmax partials
   af::Buf loss_ws;    // per-block partial sums + ticket of the loss reduction
   af::Buf pack_meta;  // per-call sequence table of af_pack_microbatch
-  af::Buf wt;         // W^T  [d, V]      bf16 (backward)
-  af::Buf ht;         // H^T  [d, T_pad]  bf16 (backward)
-  af::Buf dz;         // dZ   [Tc, V]     bf16 (backward, one token block)
-  af::Buf dzt;        // dZ^T [V, Tc]     bf16 (backward, one token block)
+  af::Buf dz;         // dZ [Tc, V] bf16 (backward, one token block)
 
   // pinned staging ring for pack metadata
   void* pack_host[af::kPackRing] = {};

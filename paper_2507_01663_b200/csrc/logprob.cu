@@ -33,12 +33,13 @@ struct LogprobEpi {
     float m, s, u, zy;
     int y;
   };
+  static constexpr bool kStaged = false;   // nothing is stored per tile: no staging buffer needed
   static __device__ __forceinline__ void unit_begin(State& st, const Params& p, int row, int, int) {
     st.m = -INFINITY; st.s = 0.f; st.u = 0.f; st.zy = -INFINITY;
     st.y = row < p.T ? __ldg(p.target + row) : -1;
   }
   static __device__ __forceinline__ void chunk(State& st, const Params& p, int, int col0,
-                                               const uint32_t (&v)[32]) {
+                                               const uint32_t (&v)[32], uint8_t*) {
     if (col0 >= p.V) return;
     float z[32];
 #pragma unroll

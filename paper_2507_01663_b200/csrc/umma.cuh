@@ -2,8 +2,10 @@
 // accumulators -- inline PTX only -- and the warp-specialised persistent GEMM main loop every
 // tensor-core kernel of the library is built on.
 //
-//   C[M,N] = A[M,K] * B[N,K]^T     A, B bf16, both K-major (row-major with K contiguous);
-//   fp32 accumulation in tensor memory; the epilogue functor consumes the accumulator tile.
+//   C[M,N] = sum_k A(m,k) * B(n,k)    A, B bf16; fp32 accumulation in tensor memory; the epilogue
+//   functor consumes the accumulator tile.  Each operand is either K-major (stored [rows, K], K
+//   contiguous) or MN-major (stored [K, rows], the M or N index contiguous), chosen at compile
+//   time, so products with a transposed operand need no transposed copy.
 //
 // CTA = 6 warps.  warp 0: TMA producer (one elected lane).  warp 1: allocates TMEM and issues
 // tcgen05.mma (one elected lane).  warps 2-5: epilogue, one TMEM lane (= output row) per thread.
@@ -34,7 +36,10 @@ constexpr int kStageBytes = kABytes + kBBytes;            // 48 KB
 constexpr int kTmemCols = 512;                            // 2 accumulators x 256 fp32 columns
 constexpr int kThreads = 192;
 constexpr int kEpiThreads = 128;
+constexpr int kMnBoxBytes = 64 * kBK * 2;                 // one 64 (MN) x 64 (K) box of an MN-major tile
+constexpr int kEpiStageBytes = 4096;                      // per epilogue warp: a 32 x 32 fp32 chunk
 constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int kSmemBytesStaged = kSmemBytes + 4 * kEpiStageBytes;
 constexpr unsigned long long kWaitLimitNs = 4000000000ull;
 constexpr unsigned int kWatchdogBit = 2u;                 // AF_DEVERR_WATCHDOG
 
@@ -150,10 +155,25 @@ __device__ __forceinline__ uint64_t smem_desc_k_sw128(uint32_t smem_addr) {
   d |= (uint64_t)2 << 61;                        // layout: 128-byte swizzle
   return d;
 }
-// Instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = 256.
-__host__ __device__ constexpr uint32_t instr_desc_bf16_f32(int m, int n) {
+// Descriptor for an MN-major bf16 tile: TMA writes it as boxes of 64 K-rows x 128 bytes (64
+// consecutive M or N indices), 128-byte swizzle, one box per 64 indices.  Inside a box, groups of
+// 8 K-rows are 1024 bytes apart (stride byte offset); boxes are kMnBoxBytes apart (leading byte
+// offset).  One MMA (K = 16) spans two 8-row groups, so the K step is 2048 bytes.
+__device__ __forceinline__ uint64_t smem_desc_mn_sw128(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)(kMnBoxBytes >> 4) << 16;       // leading byte offset: next 64 M/N indices
+  d |= (uint64_t)(1024 >> 4) << 32;              // stride byte offset: next 8 K-rows
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+// Instruction descriptor: D fp32, A and B bf16, M x N tile, each operand K-major or MN-major.
+__host__ __device__ constexpr uint32_t instr_desc_bf16_f32(int m, int n, bool a_mn = false, bool b_mn = false) {
   return (1u << 4)                         // D format: fp32
          | (1u << 7) | (1u << 10)          // A, B format: bf16
+         | ((a_mn ? 1u : 0u) << 15)        // A major: 0 = K, 1 = MN
+         | ((b_mn ? 1u : 0u) << 16)        // B major
          | ((uint32_t)(n >> 3) << 17)      // N / 8
          | ((uint32_t)(m >> 4) << 24);     // M / 16
 }
@@ -176,12 +196,16 @@ __device__ __forceinline__ int split_begin(const GemmShape& g, int s) {
 }
 
 // The epilogue functor E provides:
-//   struct Params;  struct State;
+//   struct Params;  struct State;  static constexpr bool kStaged;
 //   static __device__ void unit_begin(State&, const Params&, int row, int m_tile, int split);
-//   static __device__ void chunk(State&, const Params&, int row, int col0, const uint32_t (&v)[32]);
-//        -- 32 fp32 accumulator columns col0 .. col0+31 of output row `row` (bit patterns)
+//   static __device__ void chunk(State&, const Params&, int row, int col0, const uint32_t (&v)[32],
+//                                uint8_t* stage);
+//        -- 32 fp32 accumulator columns col0 .. col0+31 of output row `row` (bit patterns); called
+//           by all 32 lanes of an epilogue warp together (lane L holds row row0 + L).  `stage` is
+//           the warp's private kEpiStageBytes of shared memory (kStaged only, else null), used to
+//           turn row-per-lane data into coalesced global stores.
 //   static __device__ void unit_end(State&, const Params&, int row, int split);
-template <class E>
+template <class E, bool kAMN = false, bool kBMN = false>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
             const GemmShape g, const typename E::Params ep, unsigned int* d_err) {
@@ -195,6 +219,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
   auto tfull_bar = [&](int a) { return bars + 8u * (2 * kStages + a); };
   auto tempty_bar = [&](int a) { return bars + 8u * (2 * kStages + 2 + a); };
   const uint32_t tmem_slot = bars + 8u * (2 * kStages + 4);
+  uint8_t* const epi_stage_base = smem_raw + (bars + 256u - raw);   // behind the barrier block
   volatile uint32_t* tmem_slot_ptr =
       reinterpret_cast<volatile uint32_t*>(smem_raw + (tmem_slot - raw));
   __shared__ int abort_flag;
@@ -231,8 +256,20 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             if (!mbar_wait(empty_bar(stage), phase ^ 1u, &abort_flag)) { ok = false; break; }
             const uint32_t a_dst = tiles + stage * kStageBytes;
             mbar_arrive_expect_tx(full_bar(stage), kStageBytes);
-            tma_load_2d(a_dst, &tmap_a, full_bar(stage), kb * kBK, m_tile * kBM);
-            tma_load_2d(a_dst + kABytes, &tmap_b, full_bar(stage), kb * kBK, nt * kBN);
+            if constexpr (kAMN) {
+#pragma unroll
+              for (int b = 0; b < kBM / 64; ++b)
+                tma_load_2d(a_dst + b * kMnBoxBytes, &tmap_a, full_bar(stage), m_tile * kBM + b * 64, kb * kBK);
+            } else {
+              tma_load_2d(a_dst, &tmap_a, full_bar(stage), kb * kBK, m_tile * kBM);
+            }
+            if constexpr (kBMN) {
+#pragma unroll
+              for (int b = 0; b < kBN / 64; ++b)
+                tma_load_2d(a_dst + kABytes + b * kMnBoxBytes, &tmap_b, full_bar(stage), nt * kBN + b * 64, kb * kBK);
+            } else {
+              tma_load_2d(a_dst + kABytes, &tmap_b, full_bar(stage), kb * kBK, nt * kBN);
+            }
             if (++stage == kStages) { stage = 0; phase ^= 1u; }
           }
         }
@@ -242,7 +279,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
   } else if (warp == 1) {
     // ---------------------------------------------------------------- MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc = instr_desc_bf16_f32(kBM, kBN);
+      constexpr uint32_t idesc = instr_desc_bf16_f32(kBM, kBN, kAMN, kBMN);
+      // descriptor advance per K = 16 step, in 16-byte units: 32 bytes inside a swizzled K-major
+      // row, two 8-row groups (2048 bytes) for an MN-major tile
+      constexpr uint64_t a_step = kAMN ? (2048 >> 4) : 2, b_step = kBMN ? (2048 >> 4) : 2;
       int stage = 0; uint32_t phase = 0; uint32_t tile_count = 0; bool ok = true;
       for (int u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
         const int s = u % g.splits;
@@ -256,12 +296,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
             if (!mbar_wait(full_bar(stage), phase, &abort_flag)) { ok = false; break; }
             tc_fence_after();
             const uint32_t a_addr = tiles + stage * kStageBytes;
-            const uint64_t a_desc = smem_desc_k_sw128(a_addr);
-            const uint64_t b_desc = smem_desc_k_sw128(a_addr + kABytes);
+            const uint64_t a_desc = kAMN ? smem_desc_mn_sw128(a_addr) : smem_desc_k_sw128(a_addr);
+            const uint64_t b_desc = kBMN ? smem_desc_mn_sw128(a_addr + kABytes) : smem_desc_k_sw128(a_addr + kABytes);
 #pragma unroll
             for (int k = 0; k < kBK / kUmmaK; ++k) {
-              // advance both descriptors by k * 32 bytes inside the swizzle row (16-byte units)
-              mma_bf16_ss(d_tmem, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)(k * 2), idesc,
+              mma_bf16_ss(d_tmem, a_desc + (uint64_t)k * a_step, b_desc + (uint64_t)k * b_step, idesc,
                           (kb | k) != 0 ? 1u : 0u);
             }
             mma_commit(empty_bar(stage));  // smem slot reusable once these MMAs have read it
@@ -278,6 +317,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
     const int row_in_tile = quarter * 32 + lane;
     uint32_t tile_count = 0; bool ok = true;
     typename E::State st;
+    uint8_t* const stage = E::kStaged ? epi_stage_base + (warp - 2) * kEpiStageBytes : nullptr;
     for (int u = blockIdx.x; u < total_units && ok; u += gridDim.x) {
       const int m_tile = u / g.splits, s = u % g.splits;
       const int nb = split_begin(g, s), ne = split_begin(g, s + 1);
@@ -285,7 +325,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
       E::unit_begin(st, ep, row, m_tile, s);
       for (int nt = nb; nt < ne && ok; ++nt, ++tile_count) {
         const uint32_t acc = tile_count & 1u, acc_phase = (tile_count >> 1) & 1u;
-        if (!mbar_wait(tfull_bar(acc), acc_phase, &abort_flag)) { ok = false; break; }
+        // the lanes of a warp must leave together: chunk() may synchronise the warp
+        if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar(acc), acc_phase, &abort_flag))) { ok = false; break; }
         tc_fence_after();
         const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * kBN;
 #pragma unroll 1
@@ -293,7 +334,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
           uint32_t v[32];
           tmem_ld32(t_row + c * 32, v);
           tmem_ld_wait();
-          E::chunk(st, ep, row, nt * kBN + c * 32, v);
+          E::chunk(st, ep, row, nt * kBN + c * 32, v, stage);
         }
         tc_fence_before();
         mbar_arrive(tempty_bar(acc));
