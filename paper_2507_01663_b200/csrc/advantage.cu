@@ -1,7 +1,10 @@
 // af_grpo_advantage kernels: adv_i = (r_i - mean_g) / (std_g + eps) within each prompt's group.
 //
 // Contiguous groups (group_id == NULL), 4 B read + 4 B written per sample:
-//   G <= 32 (every GRPO workload here except the 64-wide store): one thread per group, registers;
+//   G a power of two in 4..128 (every GRPO workload here) and 16-byte aligned buffers: a thread
+//   owns 4 consecutive rewards (one 128-bit load), the G/4 adjacent lanes of a group combine
+//   their sums with shuffles, four independent loads are in flight per thread;
+//   other G <= 32: one thread per group, registers;
 //   G <= 4096: a block stages a run of whole groups in shared memory with 128-bit loads, reduces
 //   each group with warp shuffles (two passes: mean, then squared deviations) and writes the
 //   advantages back coalesced;  larger groups: one block per group.
@@ -80,6 +83,43 @@ __global__ void __launch_bounds__(kThreads) advantage_small_group_kernel(
     } else {
 #pragma unroll
       for (int k = 0; k < kCap; ++k) if (k < G) dst[k] = r[k];
+    }
+  }
+}
+
+// Power-of-two groups, 4 <= G <= 128.  Thread v of the flat index space owns rewards 4v .. 4v+3;
+// a group is `team` = G/4 adjacent lanes of one warp (teams never straddle a warp because the
+// warp's first index is a multiple of 32 and team divides 32).  Mean and deviations are taken in
+// fp64 (see inv_scale); the squared deviations, the root and the division run in fp32, whose
+// relative error of ~1e-7 is far inside the tolerance on an advantage of magnitude <= sqrt(G).
+constexpr int kRowUnroll = 4;
+__global__ void __launch_bounds__(kThreads) advantage_pow2_kernel(
+    const float4* __restrict__ reward, float4* __restrict__ adv, int64_t n_vec, int G, float eps, int ddof) {
+  const int team = G >> 2;
+  const double inv_g = 1.0 / (double)G;                    // exact: G is a power of two
+  const float inv_denom = G - ddof > 0 ? 1.f / (float)(G - ddof) : 0.f;
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  const int lane = threadIdx.x & 31;
+  const int64_t warp_first = (int64_t)blockIdx.x * blockDim.x + (threadIdx.x & ~31);
+  for (int64_t base = warp_first; base < n_vec; base += stride * kRowUnroll) {   // warp-uniform trip count
+    float4 r[kRowUnroll];
+#pragma unroll
+    for (int u = 0; u < kRowUnroll; ++u) {
+      const int64_t v = base + u * stride + lane;
+      r[u] = v < n_vec ? __ldg(reward + v) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int u = 0; u < kRowUnroll; ++u) {
+      const double x0 = r[u].x, x1 = r[u].y, x2 = r[u].z, x3 = r[u].w;
+      double s = (x0 + x1) + (x2 + x3);
+      for (int o = team >> 1; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+      const double mu = s * inv_g;
+      const float d0 = (float)(x0 - mu), d1 = (float)(x1 - mu), d2 = (float)(x2 - mu), d3 = (float)(x3 - mu);
+      float q = fmaf(d0, d0, fmaf(d1, d1, fmaf(d2, d2, d3 * d3)));
+      for (int o = team >> 1; o > 0; o >>= 1) q += __shfl_xor_sync(0xffffffffu, q, o);
+      const float inv = 1.f / (sqrtf(q * inv_denom) + eps);
+      const int64_t v = base + u * stride + lane;
+      if (v < n_vec) adv[v] = make_float4(d0 * inv, d1 * inv, d2 * inv, d3 * inv);
     }
   }
 }
@@ -185,7 +225,15 @@ cudaError_t launch_advantage(const float* reward, const int32_t* group_id, int64
   if (N == 0 || n_groups == 0) return cudaSuccess;
   if (group_id == nullptr) {
     const int64_t G = N / n_groups;
-    if (G >= 1 && G <= kSmallG) {
+    const bool aligned = ((reinterpret_cast<uintptr_t>(reward) | reinterpret_cast<uintptr_t>(adv)) & 15) == 0;
+    if (G >= 4 && G <= 128 && (G & (G - 1)) == 0 && aligned) {
+      const int64_t n_vec = N / 4;
+      int64_t blocks = (n_vec + (int64_t)kThreads * kRowUnroll - 1) / ((int64_t)kThreads * kRowUnroll);
+      if (blocks > (int64_t)sm_count * 8) blocks = (int64_t)sm_count * 8;
+      advantage_pow2_kernel<<<(int)blocks, kThreads, 0, s>>>(reinterpret_cast<const float4*>(reward),
+                                                             reinterpret_cast<float4*>(adv), n_vec, (int)G,
+                                                             eps_adv, ddof);
+    } else if (G >= 1 && G <= kSmallG) {
       const int vec_ok = (G % 4 == 0) && ((reinterpret_cast<uintptr_t>(reward) & 15) == 0) &&
                          ((reinterpret_cast<uintptr_t>(adv) & 15) == 0);
       int64_t blocks = (n_groups + kThreads - 1) / kThreads;

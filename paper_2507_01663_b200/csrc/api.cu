@@ -142,11 +142,12 @@ af_status af_check_device_errors(af_ctx* c, uint32_t* flags, void* stream) {
 }
 
 static size_t pack_meta_bytes(int32_t B) {
-  // [src_row int64 x B][cu int32 x (B+1)][idx int32 x B], each part 16-byte aligned
+  // [src_row int64 x B][cu int32 x (B+1)][idx int32 x B][chunk_cu int32 x (B+1)], each part
+  // 16-byte aligned
   size_t a = ((size_t)B * 8 + 15) & ~(size_t)15;
   size_t b = ((size_t)(B + 1) * 4 + 15) & ~(size_t)15;
   size_t c = ((size_t)B * 4 + 15) & ~(size_t)15;
-  return a + b + c + 16;
+  return a + b + c + b + 16;
 }
 
 af_status af_reserve(af_ctx* c, int64_t max_T, int32_t max_B, int32_t d, int32_t V,
@@ -156,10 +157,11 @@ af_status af_reserve(af_ctx* c, int64_t max_T, int32_t max_B, int32_t d, int32_t
   DeviceGuard guard(c->device);
   af_status st = AF_OK;
   if (max_T > 0) {
-    const int S = logprob_pick_splits(max_T, V, c->sm_count, c->v_splits);
-    // small batches pick more splits than large ones; reserve for the larger of both products
-    size_t need = (size_t)S * (size_t)max_T;
-    size_t small = (size_t)c->sm_count * 128 * 2;
+    const int S = logprob_pick_splits(max_T, d, V, c->sm_count, c->v_splits);
+    // smaller batches may pick up to 4 ranges whatever their size, and more than 4 only while
+    // there are at most 8 units per SM
+    size_t need = (size_t)(S > 4 ? S : 4) * (size_t)max_T;
+    size_t small = (size_t)c->sm_count * 8 * 128;
     if (need < small) need = small;
     st = ws_grow(c->partial, need * 16);
     if (st != AF_OK) return st;
@@ -212,8 +214,12 @@ af_status af_pack_microbatch(af_ctx* c, const af_store_view* store, const int32_
   int64_t* h_src = reinterpret_cast<int64_t*>(hb);
   int32_t* h_cu = reinterpret_cast<int32_t*>(hb + off_cu);
   int32_t* h_idx = reinterpret_cast<int32_t*>(hb + off_idx);
-  int64_t T = 0;
+  const size_t off_chunk = off_idx + (((size_t)B * 4 + 15) & ~(size_t)15);
+  int32_t* h_chunk = reinterpret_cast<int32_t*>(hb + off_chunk);
+  const int64_t rpc = store->hidden ? pack_rows_per_chunk(store->d) : 0;
+  int64_t T = 0, chunks = 0;
   h_cu[0] = 0;
+  h_chunk[0] = 0;
   for (int32_t j = 0; j < B; ++j) {
     const int64_t i = idx_host[j];
     if (i < 0 || i >= store->n_samples) return AF_ERR_INDEX;
@@ -224,6 +230,9 @@ af_status af_pack_microbatch(af_ctx* c, const af_store_view* store, const int32_
     T += hi - lo;
     if (T >= ((int64_t)1 << 31)) return AF_ERR_CAPACITY;
     h_cu[j + 1] = (int32_t)T;
+    if (rpc > 0) chunks += (hi - lo + rpc - 1) / rpc;
+    h_chunk[j + 1] = (int32_t)chunks;   // chunks <= T + B < 2^31 + 2^31: checked below
+    if (chunks >= ((int64_t)1 << 31)) return AF_ERR_CAPACITY;
   }
   if (T_out) *T_out = T;
   if (T > out->token_capacity) return AF_ERR_CAPACITY;
@@ -236,8 +245,9 @@ af_status af_pack_microbatch(af_ctx* c, const af_store_view* store, const int32_
   }
   if (cudaEventRecord(c->pack_evt[slot], s) != cudaSuccess) return AF_ERR_CUDA;
   PackSeqTable tab{reinterpret_cast<const int64_t*>(db), reinterpret_cast<const int32_t*>(db + off_cu),
-                   reinterpret_cast<const int32_t*>(db + off_idx)};
-  return launch_pack(*store, *out, tab, B, T, c->sm_count, s) == cudaSuccess ? AF_OK : AF_ERR_CUDA;
+                   reinterpret_cast<const int32_t*>(db + off_idx),
+                   reinterpret_cast<const int32_t*>(db + off_chunk), (int)chunks};
+  return launch_pack(*store, *out, tab, B, T, c->sm_count, c->d_err, s) == cudaSuccess ? AF_OK : AF_ERR_CUDA;
 }
 
 af_status af_token_logprob(af_ctx* c, const void* hidden, const void* W, const int32_t* target,

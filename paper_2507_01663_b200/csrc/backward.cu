@@ -229,7 +229,7 @@ af_status launch_backward(af_ctx* ctx, const void* hidden, const void* W, const 
     const Operand dZop{dz, tc, (uint64_t)V, vB};
     // 1. dZ block:  Z = H_blk W^T, both K-major
     DzEpi::Params p1{target + t0, lse + t0, dlogp + t0, dz, (int)tc, V};
-    st = run_gemm<DzEpi, false, false>(ctx, Hblk, Wop, logprob_pick_splits((int64_t)tc, V, ctx->sm_count, ctx->v_splits), p1, s);
+    st = run_gemm<DzEpi, false, false>(ctx, Hblk, Wop, logprob_pick_splits((int64_t)tc, d, V, ctx->sm_count, ctx->v_splits), p1, s);
     if (st != AF_OK) return st;
     // 2. dH block = dZ W:  A = dZ (K = v contiguous), B = W read MN-major (n = d contiguous, K = v rows)
     StoreBf16Epi::Params p2{static_cast<__nv_bfloat16*>(d_hidden) + t0 * d, d, (int)tc, d};

@@ -63,9 +63,13 @@ struct PackSeqTable {     // device views into ctx->pack_meta for one call
   const int64_t* src_row; // [B] first store row of sequence j
   const int32_t* cu;      // [B+1]
   const int32_t* idx;     // [B]
+  const int32_t* chunk_cu;// [B+1] first bulk-copy chunk of sequence j (hidden column)
+  int n_chunks;           // chunk_cu[B]
 };
+// Rows of the hidden column per bulk-copy chunk for hidden size d (0: rows too wide, no chunks).
+int pack_rows_per_chunk(int32_t d);
 cudaError_t launch_pack(const af_store_view& st, const af_packed& out, const PackSeqTable& tab,
-                        int32_t B, int64_t T, int sm_count, cudaStream_t s);
+                        int32_t B, int64_t T, int sm_count, unsigned int* d_err, cudaStream_t s);
 
 cudaError_t launch_advantage(const float* reward, const int32_t* group_id, int64_t N,
                              int32_t n_groups, float eps_adv, int32_t ddof, float* adv,
@@ -78,7 +82,7 @@ cudaError_t launch_policy_loss(const float* logp, const float* old_logp, const f
                                float* dlogp, void* ws, unsigned int* d_err, int sm_count,
                                cudaStream_t s);
 
-int logprob_pick_splits(int64_t T, int32_t V, int sm_count, int requested);
+int logprob_pick_splits(int64_t T, int32_t d, int32_t V, int sm_count, int requested);
 af_status launch_token_logprob(af_ctx* ctx, const void* hidden, const void* W,
                                const int32_t* target, int64_t T, int32_t d, int32_t V,
                                float* logp, float* entropy, float* lse, cudaStream_t s);

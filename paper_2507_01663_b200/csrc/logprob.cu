@@ -103,21 +103,41 @@ __global__ void __launch_bounds__(256) merge_partials_kernel(
 
 }  // namespace
 
-int logprob_pick_splits(int64_t T, int32_t V, int sm_count, int requested) {
-  const int m_tiles = (int)((T + umma::kBM - 1) / umma::kBM);
+// Number of vocabulary ranges S per row tile.  A CTA runs units b, b + grid, ..., each unit being
+// ceil(n_tiles / S) tiles long, so the launch lasts about ceil(m_tiles S / grid) * ceil(n_tiles / S)
+// tile times: S is chosen to minimise that product (wave quantisation decides it for small
+// batches).  The CTAs alive at one time sweep the vocabulary over ceil(grid / S) row tiles whose
+// hidden-state panels should stay L2-resident while W streams past once, which rules out small S
+// for wide hidden sizes.  Many ranges are only allowed while S * T stays small (partials buffer).
+int logprob_pick_splits(int64_t T, int32_t d, int32_t V, int sm_count, int requested) {
+  const int64_t m_tiles = (T + umma::kBM - 1) / umma::kBM;
   const int n_tiles = (V + umma::kBN - 1) / umma::kBN;
-  int S = requested > 0 ? requested : 4;
-  if (requested <= 0 && m_tiles * S < sm_count) S = (sm_count + m_tiles - 1) / (m_tiles > 0 ? m_tiles : 1);
-  if (S > n_tiles) S = n_tiles;
-  if (S < 1) S = 1;
-  return S;
+  if (requested > 0) return requested < n_tiles ? requested : n_tiles;
+  if (m_tiles < 1 || sm_count < 1) return 1;
+  constexpr int64_t kPanelBudget = 72ll << 20;        // bytes of hidden-state rows kept in L2
+  const int64_t max_units_many = (int64_t)sm_count * 8;
+  int best = 1;
+  double best_cost = 1e300;
+  for (int S = 1; S <= 32 && S <= n_tiles; ++S) {
+    const int64_t units = m_tiles * S;
+    if (S > 4 && units > max_units_many) break;
+    int64_t alive = (sm_count + S - 1) / S;
+    if (alive > m_tiles) alive = m_tiles;
+    const bool fits = alive * umma::kBM * (int64_t)d * 2 <= kPanelBudget;
+    const int64_t grid = units < sm_count ? units : sm_count;
+    double cost = (double)((units + grid - 1) / grid) * (double)((n_tiles + S - 1) / S);
+    cost *= 1.0 + 0.002 * S;                          // partials written and merged per range
+    if (!fits) cost *= 1.25;                          // W re-read from HBM by every row tile
+    if (cost < best_cost) { best_cost = cost; best = S; }
+  }
+  return best;
 }
 
 af_status launch_token_logprob(af_ctx* ctx, const void* hidden, const void* W,
                                const int32_t* target, int64_t T, int32_t d, int32_t V,
                                float* logp, float* entropy, float* lse, cudaStream_t s) {
   if (T == 0) return AF_OK;
-  const int S = logprob_pick_splits(T, V, ctx->sm_count, ctx->v_splits);
+  const int S = logprob_pick_splits(T, d, V, ctx->sm_count, ctx->v_splits);
   af_status st = ws_grow(ctx->partial, (size_t)S * (size_t)T * sizeof(float4));
   if (st != AF_OK) return st;
 
@@ -251,7 +271,7 @@ extern "C" af_status af_token_logprob_static(const void* hidden, const void* W, 
   if (d % 8 != 0 || (reinterpret_cast<uintptr_t>(hidden) & 15u) || (reinterpret_cast<uintptr_t>(W) & 15u))
     return AF_ERR_ALIGNMENT;
 
-  int S = logprob_pick_splits(T, V, st->sm_count, 0);
+  int S = logprob_pick_splits(T, d, V, st->sm_count, 0);
   if ((int64_t)S * T > kStaticPartialSlots) S = (int)(kStaticPartialSlots / T);
   unsigned int* err_word = device_flags ? device_flags : reinterpret_cast<unsigned int*>(st->scratch);
   float4* partial = reinterpret_cast<float4*>(st->scratch + kStaticHeaderBytes);

@@ -1,25 +1,40 @@
 // af_policy_loss kernel: clipped-ratio GRPO policy loss + k3 KL penalty, forward and dL/dlogp,
 // in one pass over the packed tokens (12-16 B read, 4 B written per token: HBM-bound).
 //
-// A block walks chunks of 1024-4096 tokens.  Per chunk, two warps locate the first and last
-// sequence it touches with a 32-way search over cu_seqlens and the block stages that window in
-// shared memory; token loads are issued before the lookup so both latencies overlap.  Each thread
-// owns 4 consecutive tokens (128-bit loads/stores).  Tokens of one sequence are contiguous, so a
+// A CTA owns a contiguous range of 2048-token chunks.  One thread feeds a ring of shared-memory
+// stages with bulk copies (TMA) of the chunk's logp / old / ref / entropy slices, up to three
+// chunks ahead, so the bytes in flight do not depend on how many threads are resident; each thread then
+// reads its 4 consecutive tokens from shared memory with one 128-bit load per column.  Warps run
+// free of one another inside the chunk loop: a "full" mbarrier per stage announces the data, an
+// "empty" mbarrier per stage (one arrival per warp) tells the feeding thread when the stage can
+// be refilled -- there is no block-wide barrier per chunk.
+//
+// The cu_seqlens entries (and advantages) of the sequences the CTA's tokens belong to are staged
+// in a shared-memory window, normally once per CTA; a thread finds its sequence by galloping
+// forward from where it was in the previous chunk.  The window is re-staged when a chunk runs
+// past it; a chunk that touches more sequences than a window holds (piles of empty sequences)
+// searches cu_seqlens in global memory instead.  Tokens of one sequence are contiguous, so a
 // thread sums its tokens run by run and scales each run by 1/L_i once (the per-sequence mean of
 // agg_mode 0); runs are combined with warp shuffles, per-block sums go to the workspace in fp64
 // and the last block to finish adds them in a fixed order -- no float atomics, so results are
-// bit-reproducible.
+// bit-reproducible.  Buffers that are not 16-byte aligned, and the last 1-3 tokens of a batch
+// whose length is not a multiple of 4, are read with plain loads instead.
 #include "common.cuh"
+#include "umma.cuh"
 
 namespace af {
 namespace {
 
-constexpr int kThreads = 256;
+constexpr int kThreads = 512;
+constexpr int kWarps = kThreads / 32;
 constexpr int kTokPerThread = 4;
-constexpr int kMaxSub = 4;                                // most passes of a block over one chunk
-constexpr int kPass = kThreads * kTokPerThread;           // tokens per pass
-constexpr int kMaxChunk = kPass * kMaxSub;                // most tokens per sequence-window lookup
+constexpr int kChunk = kThreads * kTokPerThread;          // tokens per chunk = per ring stage
+constexpr int kStages = 3;                                // ring depth: up to 3 chunks in flight
+constexpr int kColBytes = kChunk * 4;                     // one column slice of a stage
+constexpr int kStageBytes = 4 * kColBytes;                // logp | old | ref | entropy
+constexpr int kRingSmemBytes = kStages * kStageBytes + 128 /*alignment*/ + 64 /*barriers*/;
 constexpr int kNumSums = 4;  // pg, k3, entropy, clipped count
+constexpr int kWindow = 1025;  // cu_seqlens entries staged at a time (1024 sequences)
 
 struct LossWs {            // 64-byte header, then double partial[blocks][kNumSums]
   unsigned int ticket;
@@ -30,12 +45,20 @@ __device__ __forceinline__ double* ws_partial(LossWs* ws, int block) {
 }
 
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr int kWindow = kMaxChunk + 1;  // most cu_seqlens entries a chunk can touch unless empty sequences pile up
 
 __device__ __forceinline__ float ex2f(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               :: "r"(dst_smem), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ float4 lds128(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+  return v;
 }
 
 // largest j in [0, B) with cu[j] <= t  (cu non-decreasing, cu[0] = 0, t < cu[B])
@@ -65,14 +88,21 @@ __device__ __forceinline__ int find_seq_warp(const int32_t* __restrict__ cu, int
   return lo;
 }
 
-__global__ void __launch_bounds__(kThreads, 4) policy_loss_kernel(
+__global__ void __launch_bounds__(kThreads, 2) policy_loss_kernel(
     const float* __restrict__ logp, const float* __restrict__ old_logp,
     const float* __restrict__ ref_logp, const float* __restrict__ entropy,
     const float* __restrict__ adv_seq, const int32_t* __restrict__ cu, int B, int T,
     af_loss_params prm, af_loss_out* __restrict__ out, float* __restrict__ dlogp, LossWs* ws,
-    unsigned int* d_err, int vec_ok, int n_sub) {
-  __shared__ int s_cu[2][kWindow];
-  __shared__ int s_j0[2], s_j1[2];
+    unsigned int* d_err, int vec_ok) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ int s_win[kWindow];      // cu_seqlens[s_first .. s_first + s_count - 1]
+  __shared__ float s_adv[kWindow];    // adv_seq of the same sequences
+  __shared__ int s_first, s_count, s_cover;   // tokens < s_cover lie inside the staged window
+  __shared__ int abort_flag;
+  const uint32_t ring = (umma::smem_u32(smem_raw) + 127u) & ~127u;
+  const uint32_t bars = ring + kStages * kStageBytes;
+  auto full_bar = [&](int st) { return bars + 8u * st; };
+  auto empty_bar = [&](int st) { return bars + 8u * (kStages + st); };
   const float lo_b = 1.f - prm.clip_lo, hi_b = 1.f + prm.clip_hi;
   const float w_all = prm.agg_mode == 0 ? (B > 0 ? prm.loss_scale / (float)B : 0.f)
                                         : (T > 0 ? prm.loss_scale / (float)T : 0.f);
@@ -81,107 +111,170 @@ __global__ void __launch_bounds__(kThreads, 4) policy_loss_kernel(
   int acc_clip = 0;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 
-  const int kChunk = kPass * n_sub;   // tokens that share one sequence-window lookup
   const int n_chunks = (T + kChunk - 1) / kChunk;
-  int buf = 0;
-  for (int c = blockIdx.x; c < n_chunks; c += gridDim.x, buf ^= 1) {
-    const int c0 = c * kChunk;
-    const int c_last = (T - c0 > kChunk ? c0 + kChunk : T) - 1;   // last token of the chunk
-    // the chunk's window of cu_seqlens: entries j0 .. j1+1 (first and last sequence it touches)
-    if (warp == 0) {
-      const int j = find_seq_warp(cu, B, c0, lane);
-      if (lane == 0) s_j0[buf] = j;
-    } else if (warp == 1) {
-      const int j = find_seq_warp(cu, B, c_last, lane);
-      if (lane == 0) s_j1[buf] = j;
-    }
-    __syncthreads();
-    const int j0 = s_j0[buf];
-    const int nw = s_j1[buf] - j0 + 2;
-    const bool staged = nw <= kWindow;
-    int* win = s_cu[buf];
-    if (staged)
-      for (int i = threadIdx.x; i < nw; i += kThreads) win[i] = __ldg(cu + j0 + i);
-    __syncthreads();
+  const int c_begin = (int)(((int64_t)n_chunks * blockIdx.x) / gridDim.x);
+  const int n_mine = (int)(((int64_t)n_chunks * (blockIdx.x + 1)) / gridDim.x) - c_begin;
+  const int n_cols = entropy ? 4 : 3;
 
-#pragma unroll 1
-    for (int sub = 0; sub < n_sub; ++sub) {
-      const int t0 = c0 + sub * kPass + threadIdx.x * kTokPerThread;
-      const int n = t0 < T ? ((T - t0) < kTokPerThread ? (T - t0) : kTokPerThread) : 0;
-      float lp[4], ol[4], rf[4], en[4] = {0.f, 0.f, 0.f, 0.f}, g[4];
-      if (n == 4 && vec_ok) {
-        const float4 a = __ldg(reinterpret_cast<const float4*>(logp + t0));
-        const float4 b = __ldg(reinterpret_cast<const float4*>(old_logp + t0));
-        const float4 r = __ldg(reinterpret_cast<const float4*>(ref_logp + t0));
-        lp[0] = a.x; lp[1] = a.y; lp[2] = a.z; lp[3] = a.w;
-        ol[0] = b.x; ol[1] = b.y; ol[2] = b.z; ol[3] = b.w;
-        rf[0] = r.x; rf[1] = r.y; rf[2] = r.z; rf[3] = r.w;
-        if (entropy) {
-          const float4 e = __ldg(reinterpret_cast<const float4*>(entropy + t0));
-          en[0] = e.x; en[1] = e.y; en[2] = e.z; en[3] = e.w;
+  // feeding thread: bulk copies of chunk i's column slices into ring stage i % kStages.  A slice
+  // is copied up to its last whole group of 4 tokens (16 bytes).
+  auto issue = [&](int i) {
+    const int c0 = (c_begin + i) * kChunk;
+    const int ntok = T - c0 < kChunk ? T - c0 : kChunk;
+    const uint32_t nb = (uint32_t)(ntok & ~3) * 4u;
+    const uint32_t bar = full_bar(i % kStages);
+    if (nb == 0) { umma::mbar_arrive(bar); return; }
+    const uint32_t dst = ring + (i % kStages) * kStageBytes;
+    umma::mbar_arrive_expect_tx(bar, nb * n_cols);
+    bulk_load(dst, logp + c0, nb, bar);
+    bulk_load(dst + kColBytes, old_logp + c0, nb, bar);
+    bulk_load(dst + 2 * kColBytes, ref_logp + c0, nb, bar);
+    if (entropy) bulk_load(dst + 3 * kColBytes, entropy + c0, nb, bar);
+  };
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    s_first = 0; s_count = 0; s_cover = -1;
+    if (vec_ok) {
+      for (int s = 0; s < kStages; ++s) { umma::mbar_init(full_bar(s), 1); umma::mbar_init(empty_bar(s), kWarps); }
+      umma::fence_mbar_init();
+      for (int i = 0; i < kStages && i < n_mine; ++i) issue(i);
+    }
+  }
+  __syncthreads();
+
+  int hint = 0;        // this thread's position in the window at the previous chunk
+  bool ok = true;      // false once a wait ran out of time: the warp keeps the block-wide barriers
+                       // of the loop in step with the others but touches no more data
+  for (int i = 0; i < n_mine; ++i) {
+    const int c0 = (c_begin + i) * kChunk;
+    const int c_last = (T - c0 > kChunk ? c0 + kChunk : T) - 1;   // last token of the chunk
+    if (c_last >= s_cover) {
+      // (re)stage the window from the chunk's first sequence on; block-uniform and rare
+      __syncthreads();
+      if (warp == 0) {
+        const int j = find_seq_warp(cu, B, c0, lane);
+        if (lane == 0) {
+          const int cnt = B + 1 - j < kWindow ? B + 1 - j : kWindow;
+          s_first = j; s_count = cnt;
         }
-      } else {
-        for (int k = 0; k < n; ++k) {
+      }
+      __syncthreads();
+      const int j = s_first, cnt = s_count;
+      for (int q = threadIdx.x; q < cnt; q += kThreads) {
+        s_win[q] = __ldg(cu + j + q);
+        s_adv[q] = j + q < B ? __ldg(adv_seq + j + q) : 0.f;
+      }
+      if (threadIdx.x == 0) s_cover = __ldg(cu + j + cnt - 1);   // tokens below the last staged entry
+      hint = 0;
+      __syncthreads();
+    }
+    const int j0 = s_first, nw = s_count;
+    const bool staged = c_last < s_cover;
+    const int st = i % kStages;
+    if (vec_ok && ok) {
+      // the stage chunk i-1 used is refilled with chunk i + kStages - 1 once every warp has left it
+      if (threadIdx.x == 0 && i >= 1 && i + kStages - 1 < n_mine) {
+        if (umma::mbar_wait(empty_bar((i - 1) % kStages), (uint32_t)((i - 1) / kStages) & 1u, &abort_flag))
+          issue(i + kStages - 1);
+      }
+      ok = __all_sync(0xffffffffu, umma::mbar_wait(full_bar(st), (uint32_t)(i / kStages) & 1u, &abort_flag));
+    }
+    if (!ok) continue;
+
+    const int t0 = c0 + threadIdx.x * kTokPerThread;
+    const int n = t0 < T ? ((T - t0) < kTokPerThread ? (T - t0) : kTokPerThread) : 0;
+    float lp[4], ol[4], rf[4], en[4] = {0.f, 0.f, 0.f, 0.f}, g[4];
+    if (n == 4 && vec_ok) {
+      const uint32_t src = ring + st * kStageBytes + threadIdx.x * 16;
+      const float4 a = lds128(src), b = lds128(src + kColBytes), r = lds128(src + 2 * kColBytes);
+      lp[0] = a.x; lp[1] = a.y; lp[2] = a.z; lp[3] = a.w;
+      ol[0] = b.x; ol[1] = b.y; ol[2] = b.z; ol[3] = b.w;
+      rf[0] = r.x; rf[1] = r.y; rf[2] = r.z; rf[3] = r.w;
+      if (entropy) {
+        const float4 e = lds128(src + 3 * kColBytes);
+        en[0] = e.x; en[1] = e.y; en[2] = e.z; en[3] = e.w;
+      }
+    } else {
+#pragma unroll
+      for (int k = 0; k < kTokPerThread; ++k) {
+        if (k < n) {
           lp[k] = __ldg(logp + t0 + k); ol[k] = __ldg(old_logp + t0 + k); rf[k] = __ldg(ref_logp + t0 + k);
           if (entropy) en[k] = __ldg(entropy + t0 + k);
         }
       }
-      if (n > 0) {
-        int j, seq_beg, seq_end;
-        if (staged) {
-          int lo = 0, hi = nw - 1;  // win[lo] <= t0, and t0 < win[hi] unless cu_seqlens is malformed
-          while (hi - lo > 1) {
-            const int mid = (lo + hi) >> 1;
-            if (win[mid] <= t0) lo = mid; else hi = mid;
-          }
-          j = j0 + lo; seq_beg = win[lo]; seq_end = win[lo + 1];
-        } else {
-          j = find_seq(cu, B, t0); seq_beg = __ldg(cu + j); seq_end = __ldg(cu + j + 1);
+    }
+    if (vec_ok) {   // the values are in registers: this warp is done with the stage
+      __syncwarp();
+      if (lane == 0) umma::mbar_arrive(empty_bar(st));
+    }
+    if (n > 0) {
+      int j, seq_beg, seq_end;
+      if (staged) {
+        // gallop forward from the previous position, then bisect: s_win[lo] <= t0 < s_win[hi]
+        int lo = hint, hi, step = 1;
+        for (;;) {
+          hi = lo + step;
+          if (hi >= nw - 1) { hi = nw - 1; break; }
+          if (s_win[hi] > t0) break;
+          lo = hi; step <<= 1;
         }
-        const int j_max = staged ? j0 + nw - 2 : B - 1;   // last sequence this thread may step to
-        float A = __ldg(adv_seq + j);
-        float inv_len = prm.agg_mode == 0 ? __frcp_rn((float)(seq_end - seq_beg)) : 1.f;
-        float run_pg = 0.f, run_kl = 0.f;
+        while (hi - lo > 1) {
+          const int mid = (lo + hi) >> 1;
+          if (s_win[mid] <= t0) lo = mid; else hi = mid;
+        }
+        hint = lo;
+        j = j0 + lo; seq_beg = s_win[lo]; seq_end = s_win[lo + 1];
+      } else {
+        j = find_seq(cu, B, t0); seq_beg = __ldg(cu + j); seq_end = __ldg(cu + j + 1);
+      }
+      const int j_max = staged ? j0 + nw - 2 : B - 1;   // last sequence this thread may step to
+      float A = staged ? s_adv[j - j0] : __ldg(adv_seq + j);
+      float inv_len = prm.agg_mode == 0 ? __frcp_rn((float)(seq_end - seq_beg)) : 1.f;
+      float run_pg = 0.f, run_kl = 0.f;
 #pragma unroll
-        for (int k = 0; k < kTokPerThread; ++k) {
-          if (k < n) {
-            const int t = t0 + k;
-            if (t >= seq_end) {  // run of sequence j ends: scale it once, move to the next sequence
-              acc_pg += run_pg * inv_len; acc_kl += run_kl * inv_len;
-              run_pg = 0.f; run_kl = 0.f;
-              while (t >= seq_end && j < j_max) {
-                ++j;
-                seq_beg = seq_end;
-                seq_end = staged ? win[j - j0 + 1] : __ldg(cu + j + 1);
-              }
-              A = __ldg(adv_seq + j);
-              inv_len = prm.agg_mode == 0 ? __frcp_rn((float)(seq_end - seq_beg)) : 1.f;
+      for (int k = 0; k < kTokPerThread; ++k) {
+        if (k < n) {
+          const int t = t0 + k;
+          if (t >= seq_end) {  // run of sequence j ends: scale it once, move to the next sequence
+            acc_pg += run_pg * inv_len; acc_kl += run_kl * inv_len;
+            run_pg = 0.f; run_kl = 0.f;
+            while (t >= seq_end && j < j_max) {
+              ++j;
+              seq_beg = seq_end;
+              seq_end = staged ? s_win[j - j0 + 1] : __ldg(cu + j + 1);
             }
-            const float rho = ex2f((lp[k] - ol[k]) * kLog2e);
-            const float s1 = rho * A;
-            const float s2 = fminf(fmaxf(rho, lo_b), hi_b) * A;
-            const bool clipped = s2 < s1;
-            const float delta = rf[k] - lp[k];
-            const float em1 = ex2f(delta * kLog2e) - 1.f;   // exactly 0 when ref == logp
-            run_pg -= fminf(s1, s2);
-            run_kl += em1 - delta;
-            acc_ent += en[k];
-            acc_clip += clipped ? 1 : 0;
-            g[k] = (w_all * inv_len) * fmaf(nbeta, em1, clipped ? 0.f : -s1);
+            A = staged ? s_adv[j - j0] : __ldg(adv_seq + j);
+            inv_len = prm.agg_mode == 0 ? __frcp_rn((float)(seq_end - seq_beg)) : 1.f;
           }
+          const float rho = ex2f((lp[k] - ol[k]) * kLog2e);
+          const float s1 = rho * A;
+          const float s2 = fminf(fmaxf(rho, lo_b), hi_b) * A;
+          const bool clipped = s2 < s1;
+          const float delta = rf[k] - lp[k];
+          const float em1 = ex2f(delta * kLog2e) - 1.f;   // exactly 0 when ref == logp
+          run_pg -= fminf(s1, s2);
+          run_kl += em1 - delta;
+          acc_ent += en[k];
+          acc_clip += clipped ? 1 : 0;
+          g[k] = (w_all * inv_len) * fmaf(nbeta, em1, clipped ? 0.f : -s1);
         }
-        acc_pg += run_pg * inv_len; acc_kl += run_kl * inv_len;
-        if (dlogp) {
-          if (n == 4 && vec_ok) {
-            *reinterpret_cast<float4*>(dlogp + t0) = make_float4(g[0], g[1], g[2], g[3]);
-          } else {
-            for (int k = 0; k < n; ++k) dlogp[t0 + k] = g[k];
-          }
+      }
+      acc_pg += run_pg * inv_len; acc_kl += run_kl * inv_len;
+      if (dlogp) {
+        if (n == 4 && vec_ok) {
+          *reinterpret_cast<float4*>(dlogp + t0) = make_float4(g[0], g[1], g[2], g[3]);
+        } else {
+#pragma unroll
+          for (int k = 0; k < kTokPerThread; ++k) if (k < n) dlogp[t0 + k] = g[k];
         }
+      }
     }
-    }
-    // no barrier here: the next chunk uses the other window buffer, and its first barrier
-    // orders this chunk's reads before the chunk after it reuses this buffer
+  }
+
+  __syncthreads();
+  if (abort_flag) {   // a bulk copy did not arrive in time: flag it, let copies in flight land
+    if (threadIdx.x == 0) atomicOr(d_err, umma::kWatchdogBit);
+    __nanosleep(1000000);
   }
 
   // block reduction: warp shuffles, then fp64 across warps (fixed order)
@@ -244,17 +337,21 @@ cudaError_t launch_policy_loss(const float* logp, const float* old_logp, const f
                                int32_t B, int64_t T, const af_loss_params& p, af_loss_out* out,
                                float* dlogp, void* ws, unsigned int* d_err, int sm_count,
                                cudaStream_t s) {
-  // large batches amortise the sequence-window lookup over several passes; small ones keep one
-  // pass per block so that every SM has work
-  int n_sub = 1;
-  while (n_sub < kMaxSub && T / ((int64_t)kPass * n_sub * 2) >= (int64_t)sm_count * 4) n_sub *= 2;
-  const int64_t chunk = (int64_t)kPass * n_sub;
-  int64_t chunks = (T + chunk - 1) / chunk;
-  int blocks = (int)(chunks < 1 ? 1 : (chunks < (int64_t)sm_count * 8 ? chunks : (int64_t)sm_count * 8));
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(policy_loss_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         kRingSmemBytes);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  const int64_t chunks = (T + kChunk - 1) / kChunk;
+  // two CTAs per SM, each over a contiguous range of chunks (grid <= the workspace's 8 blocks per SM)
+  const int blocks = (int)(chunks < 1 ? 1 : (chunks < (int64_t)sm_count * 2 ? chunks : (int64_t)sm_count * 2));
   auto al = [](const void* q) { return (reinterpret_cast<uintptr_t>(q) & 15) == 0; };
   const int vec_ok = al(logp) && al(old_logp) && al(ref_logp) && al(entropy) && al(dlogp);
-  policy_loss_kernel<<<blocks, kThreads, 0, s>>>(logp, old_logp, ref_logp, entropy, adv_seq, cu, B,
-                                                 (int)T, p, out, dlogp, (LossWs*)ws, d_err, vec_ok, n_sub);
+  policy_loss_kernel<<<blocks, kThreads, kRingSmemBytes, s>>>(logp, old_logp, ref_logp, entropy, adv_seq, cu,
+                                                              B, (int)T, p, out, dlogp, (LossWs*)ws, d_err,
+                                                              vec_ok);
   return cudaGetLastError();
 }
 

@@ -1,11 +1,17 @@
 // af_pack_microbatch kernels: gather the token rows of the indexed samples into cu_seqlens-packed
 // tensors.  Pure data movement (HBM-bound): every payload byte is read once and written once,
-// as 16-byte words, so the result is bit-exact by construction.
+// untouched, so the result is bit-exact by construction.
 //
-// Layout: sample idx[j] owns the contiguous store rows src_row[j] .. src_row[j]+len-1, and the
-// packed rows cu[j] .. cu[j+1]-1.  A warp copies one token row (d*2 bytes) at a time; its
-// sequence is found by a binary search over cu (B+1 ints, L1/L2 resident).
+// Layout: sample idx[j] owns the contiguous store rows src_row[j] .. src_row[j]+len-1 and the
+// packed rows cu[j] .. cu[j+1]-1, so the hidden column of a sequence is ONE contiguous byte range
+// on both sides.  It is cut into chunks of whole rows (at most kChunkBytes) and every chunk moves
+// with two bulk-copy (TMA) instructions, global -> shared -> global, issued by a single thread
+// per CTA through a ring of shared-memory stages: no payload byte passes through a register, and
+// the number of bytes in flight does not depend on how many threads are resident.  Rows wider
+// than a chunk fall back to a warp-per-row copy with 128-bit loads and stores.  The 4-byte
+// columns are gathered by a second, small kernel (one thread per token).
 #include "common.cuh"
+#include "umma.cuh"
 
 namespace af {
 namespace {
@@ -48,16 +54,119 @@ __global__ void __launch_bounds__(256) pack_rows_kernel(const uint4* __restrict_
     const int64_t srow = __ldg(src_row + j) + (t - __ldg(cu + j));
     const uint4* s = src + srow * words;
     uint4* o = dst + t * (int64_t)words;
-    int w = lane;
-    for (; w + 32 * (kRowUnroll - 1) < words; w += 32 * kRowUnroll) {
+    for (int w = lane; w < words; w += 32 * kRowUnroll) {   // all loads of a batch before its stores
       uint4 v[kRowUnroll];
 #pragma unroll
-      for (int u = 0; u < kRowUnroll; ++u) v[u] = ld_stream(s + w + 32 * u);
+      for (int u = 0; u < kRowUnroll; ++u) if (w + 32 * u < words) v[u] = ld_stream(s + w + 32 * u);
 #pragma unroll
-      for (int u = 0; u < kRowUnroll; ++u) st_stream(o + w + 32 * u, v[u]);
+      for (int u = 0; u < kRowUnroll; ++u) if (w + 32 * u < words) st_stream(o + w + 32 * u, v[u]);
     }
-    for (; w < words; w += 32) st_stream(o + w, ld_stream(s + w));
   }
+}
+
+// ---- bulk-copy (TMA) path ---------------------------------------------------------------------
+constexpr int kChunkBytes = 32768;      // most bytes per bulk copy (whole rows)
+constexpr int kCopyStages = 6;          // shared-memory ring: 6 x 32 KB
+constexpr int kCopyAhead = 4;           // loads in flight ahead of the store being issued
+constexpr int kCopySmemBytes = kCopyStages * kChunkBytes + 128 /*alignment*/ + 64 /*barriers*/;
+
+__device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               :: "r"(dst_smem), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void bulk_store(void* dst, uint32_t src_smem, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+               :: "l"(dst), "r"(src_smem), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int kPending>
+__device__ __forceinline__ void bulk_wait_read() {   // at most kPending stores still reading shared memory
+  asm volatile("cp.async.bulk.wait_group.read %0;" :: "n"(kPending) : "memory");
+}
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
+// Walks the chunks of consecutive sequences: sequence j owns chunks chunk_cu[j] .. chunk_cu[j+1]-1,
+// each `rows_per_chunk` rows except the last one of the sequence.
+struct ChunkCursor {
+  const int64_t* src_row; const int32_t* cu; const int32_t* chunk_cu;
+  int B, rows_per_chunk;
+  int j, first_chunk, next_first, dst_row0, len;
+  int64_t src_row0;
+  __device__ void seek(int c) {   // largest j with chunk_cu[j] <= c (sequences without rows own no chunk)
+    int lo = 0, hi = B;
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (__ldg(chunk_cu + mid) <= c) lo = mid; else hi = mid;
+    }
+    j = lo;
+    load();
+  }
+  __device__ void load() {
+    first_chunk = __ldg(chunk_cu + j);
+    next_first = __ldg(chunk_cu + j + 1);
+    dst_row0 = __ldg(cu + j);
+    len = __ldg(cu + j + 1) - dst_row0;
+    src_row0 = __ldg(src_row + j);
+  }
+  // source row, packed row and row count of chunk c (c never decreases between calls)
+  __device__ void at(int c, int64_t& srow, int64_t& drow, int& rows) {
+    while (c >= next_first && j + 1 < B) { ++j; load(); }
+    const int r0 = (c - first_chunk) * rows_per_chunk;
+    rows = len - r0 < rows_per_chunk ? len - r0 : rows_per_chunk;
+    srow = src_row0 + r0;
+    drow = (int64_t)dst_row0 + r0;
+  }
+};
+
+// One CTA per SM, one working thread per CTA.  CTA b moves the contiguous chunk range
+// [n_chunks b / grid, n_chunks (b+1) / grid).
+__global__ void __launch_bounds__(32, 1) pack_rows_bulk_kernel(
+    const uint8_t* __restrict__ src, uint8_t* __restrict__ dst, const int64_t* __restrict__ src_row,
+    const int32_t* __restrict__ cu, const int32_t* __restrict__ chunk_cu, int B, int n_chunks,
+    int rows_per_chunk, int row_bytes, unsigned int* d_err) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ int abort_flag;
+  if (threadIdx.x != 0) return;
+  const uint32_t raw = umma::smem_u32(smem_raw);
+  const uint32_t ring = (raw + 127u) & ~127u;
+  const uint32_t bars = ring + kCopyStages * kChunkBytes;
+  abort_flag = 0;
+  for (int s = 0; s < kCopyStages; ++s) umma::mbar_init(bars + 8u * s, 1);
+  umma::fence_mbar_init();
+
+  const int c_begin = (int)(((int64_t)n_chunks * blockIdx.x) / gridDim.x);
+  const int c_end = (int)(((int64_t)n_chunks * (blockIdx.x + 1)) / gridDim.x);
+  const int n = c_end - c_begin;
+  if (n <= 0) return;
+
+  ChunkCursor lc{src_row, cu, chunk_cu, B, rows_per_chunk};   // cursor of the loads
+  ChunkCursor sc = lc;                                         // cursor of the stores
+  lc.seek(c_begin);
+  sc.seek(c_begin);
+  auto issue_load = [&](int i) {
+    int64_t srow, drow; int rows;
+    lc.at(c_begin + i, srow, drow, rows);
+    const int st = i % kCopyStages;
+    const uint32_t bytes = (uint32_t)rows * (uint32_t)row_bytes;
+    umma::mbar_arrive_expect_tx(bars + 8u * st, bytes);
+    bulk_load(ring + st * kChunkBytes, src + srow * row_bytes, bytes, bars + 8u * st);
+  };
+  for (int i = 0; i < kCopyAhead && i < n; ++i) issue_load(i);
+  for (int i = 0; i < n; ++i) {
+    const int st = i % kCopyStages;
+    if (!umma::mbar_wait(bars + 8u * st, (uint32_t)(i / kCopyStages) & 1u, &abort_flag)) break;
+    int64_t srow, drow; int rows;
+    sc.at(c_begin + i, srow, drow, rows);
+    bulk_store(dst + drow * row_bytes, ring + st * kChunkBytes, (uint32_t)rows * (uint32_t)row_bytes);
+    bulk_commit();
+    if (i + kCopyAhead < n) {
+      // the stage of load i + kCopyAhead was last read by store i + kCopyAhead - kCopyStages
+      bulk_wait_read<kCopyStages - kCopyAhead>();
+      issue_load(i + kCopyAhead);
+    }
+  }
+  bulk_wait_all();
+  if (abort_flag) atomicOr(d_err, umma::kWatchdogBit);
 }
 
 // One thread per packed token for the 4-byte columns; the first B threads also gather adv.
@@ -85,8 +194,13 @@ __global__ void __launch_bounds__(256) pack_cols_kernel(
 
 }  // namespace
 
+int pack_rows_per_chunk(int32_t d) {
+  const int64_t row_bytes = (int64_t)d * 2;
+  return row_bytes <= kChunkBytes ? (int)(kChunkBytes / row_bytes) : 0;
+}
+
 cudaError_t launch_pack(const af_store_view& st, const af_packed& out, const PackSeqTable& tab,
-                        int32_t B, int64_t T, int sm_count, cudaStream_t s) {
+                        int32_t B, int64_t T, int sm_count, unsigned int* d_err, cudaStream_t s) {
   {
     int64_t items = T > (int64_t)B + 1 ? T : (int64_t)B + 1;
     int blocks = (int)((items + 255) / 256);
@@ -97,11 +211,26 @@ cudaError_t launch_pack(const af_store_view& st, const af_packed& out, const Pac
                                             tab.idx, B, (int)T);
   }
   if (T > 0 && out.hidden) {
-    const int words = st.d / 8;
-    int64_t blocks = (T + 7) / 8;  // 8 warps per block
-    if (blocks > sm_count * 8) blocks = sm_count * 8;
-    pack_rows_kernel<<<(int)blocks, 256, 0, s>>>((const uint4*)st.hidden, (uint4*)out.hidden,
-                                                 tab.src_row, tab.cu, B, (int)T, words);
+    const int rpc = pack_rows_per_chunk(st.d);
+    if (rpc > 0 && tab.n_chunks > 0) {
+      static bool attr_set = false;
+      if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(pack_rows_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             kCopySmemBytes);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+      }
+      const int grid = tab.n_chunks < sm_count ? tab.n_chunks : sm_count;
+      pack_rows_bulk_kernel<<<grid, 32, kCopySmemBytes, s>>>(
+          (const uint8_t*)st.hidden, (uint8_t*)out.hidden, tab.src_row, tab.cu, tab.chunk_cu, B,
+          tab.n_chunks, rpc, st.d * 2, d_err);
+    } else {
+      const int words = st.d / 8;
+      int64_t blocks = (T + 7) / 8;  // 8 warps per block
+      if (blocks > sm_count * 8) blocks = sm_count * 8;
+      pack_rows_kernel<<<(int)blocks, 256, 0, s>>>((const uint4*)st.hidden, (uint4*)out.hidden,
+                                                   tab.src_row, tab.cu, B, (int)T, words);
+    }
   }
   return cudaGetLastError();
 }
