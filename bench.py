@@ -137,10 +137,11 @@ def reduce_over_ranks(ms_local: float, tokens_local: int, world: int):
 class ScoringJob:
     """Device buffers of one rank and the step function that runs the path through the C ABI."""
 
-    def __init__(self, w: wl.Workload, device: torch.device):
+    def __init__(self, w: wl.Workload, device: torch.device, gemm_pair: bool = False):
         from paper_2507_01663_b200 import binding as B
         self.B, self.w, self.dev = B, w, device
         self.ctx = B.Context(device.index or 0)
+        self.ctx.set_tuning(0, 0, gemm_pair)
         T = w.total_tokens
         self.T = T
         self.store = {
@@ -318,7 +319,7 @@ def run_ours(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
     w = rank_workload(args.workload, rank)
-    job = ScoringJob(w, dev)
+    job = ScoringJob(w, dev, args.gemm_pair)
     peaks = measured_peaks()
     hbm_alone = job.hbm_kernels_at_scale(peaks["hbm_gbs"]) if rank == 0 and world == 1 else {}
 
@@ -357,6 +358,7 @@ def run_ours(args):
                                f"({w.n_prompts} prompts x {w.group_size}), {job.T} scored tokens per GPU, "
                                "one arrival-ordered packed micro-batch" + (", forward + backward (dH, dW)" if w.backward else ""),
                    "l2": "inputs (hidden states >> 126 MB L2) exceed L2; no flush needed",
+                   "gemm": "CTA pairs (cta_group::2)" if args.gemm_pair else "one CTA per tile",
                    "loss": {"clip_eps": w.clip_eps, "kl_coef": w.kl_coef, "agg": "seq-mean-token-mean"}},
         "roofline": {"bound": "tensor", "kernel": "fused LM-head GEMM + online log-softmax (af_token_logprob)",
                      "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
@@ -439,6 +441,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2")
     ap.add_argument("--cpu-sample", type=int, default=1536, help="tokens in the CPU-oracle sample")
+    ap.add_argument("--gemm-pair", action="store_true",
+                    help="run the tensor-core GEMMs on CTA pairs (af_set_tuning gemm_pair = 1) instead of the default")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3

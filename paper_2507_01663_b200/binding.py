@@ -78,7 +78,7 @@ def load_library() -> C.CDLL:
     lib.af_reserve.argtypes = [vp, i64, i32, i32, i32, i32]
     lib.af_workspace_bytes.argtypes = [vp]
     lib.af_workspace_bytes.restype = i64
-    lib.af_set_tuning.argtypes = [vp, i32, i32]
+    lib.af_set_tuning.argtypes = [vp, i32, i32, i32]
     lib.af_check_device_errors.argtypes = [vp, C.POINTER(C.c_uint32), vp]
     lib.af_pack_microbatch.argtypes = [vp, C.POINTER(StoreView), vp, i32, C.POINTER(Packed),
                                        C.POINTER(i64), vp]
@@ -141,8 +141,8 @@ class Context:
     def workspace_bytes(self) -> int:
         return int(self.lib.af_workspace_bytes(self.handle))
 
-    def set_tuning(self, v_splits: int = 0, bwd_token_block: int = 0):
-        _check(self.lib.af_set_tuning(self.handle, v_splits, bwd_token_block), "af_set_tuning")
+    def set_tuning(self, v_splits: int = 0, bwd_token_block: int = 0, gemm_pair: bool = False):
+        _check(self.lib.af_set_tuning(self.handle, v_splits, bwd_token_block, int(gemm_pair)), "af_set_tuning")
 
     def check_device_errors(self, stream=None) -> int:
         """Synchronise the stream; return the device error bits (0 = none) and clear them."""

@@ -17,19 +17,6 @@ af_status ws_grow(Buf& b, size_t bytes) {
   return AF_OK;
 }
 
-af_status encode_bf16_2d(const af_ctx* ctx, CUtensorMap* map, const void* base, uint64_t rows,
-                         uint64_t cols, uint64_t pitch_bytes, uint32_t box_rows) {
-  cuuint64_t dims[2] = {cols, rows};
-  cuuint64_t strides[1] = {pitch_bytes};
-  cuuint32_t box[2] = {64, box_rows};
-  cuuint32_t estr[2] = {1, 1};
-  CUresult r = ctx->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims,
-                           strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS ? AF_OK : AF_ERR_CUDA;
-}
-
 namespace {
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -121,11 +108,12 @@ int64_t af_workspace_bytes(const af_ctx* c) {
   return (int64_t)(c->partial.cap + c->loss_ws.cap + c->pack_meta.cap + c->dz.cap);
 }
 
-af_status af_set_tuning(af_ctx* c, int32_t v_splits, int32_t bwd_token_block) {
-  if (!c || v_splits < 0 || bwd_token_block < 0) return AF_ERR_INVALID_ARG;
+af_status af_set_tuning(af_ctx* c, int32_t v_splits, int32_t bwd_token_block, int32_t gemm_pair) {
+  if (!c || v_splits < 0 || bwd_token_block < 0 || (gemm_pair != 0 && gemm_pair != 1)) return AF_ERR_INVALID_ARG;
   if (bwd_token_block % 128 != 0) return AF_ERR_SHAPE;
   c->v_splits = v_splits;
   c->bwd_token_block = bwd_token_block;
+  c->gemm_pair = gemm_pair;
   return AF_OK;
 }
 
@@ -157,7 +145,7 @@ af_status af_reserve(af_ctx* c, int64_t max_T, int32_t max_B, int32_t d, int32_t
   DeviceGuard guard(c->device);
   af_status st = AF_OK;
   if (max_T > 0) {
-    const int S = logprob_pick_splits(max_T, d, V, c->sm_count, c->v_splits);
+    const int S = logprob_pick_splits(max_T, d, V, c->sm_count, c->gemm_pair != 0, c->v_splits);
     // smaller batches may pick up to 4 ranges whatever their size, and more than 4 only while
     // there are at most 8 units per SM
     size_t need = (size_t)(S > 4 ? S : 4) * (size_t)max_T;

@@ -13,8 +13,7 @@
 // 16 bytes to each of 32 different rows per instruction.  Each warp therefore passes its 32x32
 // chunk through a private, XOR-swizzled shared-memory buffer and stores whole 64/128-byte row
 // segments, four to eight rows per instruction.
-#include "common.cuh"
-#include "umma.cuh"
+#include "gemm_launch.cuh"
 
 namespace af {
 namespace {
@@ -165,41 +164,6 @@ struct StoreF32Epi {
   static __device__ __forceinline__ void unit_end(State&, const Params&, int, int) {}
 };
 
-// One operand of a GEMM launch: the matrix as it sits in memory.
-struct Operand {
-  const void* base;
-  uint64_t rows, cols;   // memory rows and (contiguous) columns
-  uint64_t pitch_bytes;
-};
-
-// C[M,N] = sum_k A(m,k) B(n,k).  A K-major operand is stored [M or N, K]; an MN-major operand is
-// stored [K, M or N].  Box: 64 contiguous elements wide; 128 / 256 rows for K-major A / B, 64
-// K-rows for MN-major.
-template <class E, bool kAMN, bool kBMN>
-af_status run_gemm(af_ctx* ctx, const Operand& A, const Operand& B, int splits,
-                   const typename E::Params& ep, cudaStream_t s) {
-  CUtensorMap ta, tb;
-  af_status st = encode_bf16_2d(ctx, &ta, A.base, A.rows, A.cols, A.pitch_bytes, kAMN ? 64 : umma::kBM);
-  if (st != AF_OK) return st;
-  st = encode_bf16_2d(ctx, &tb, B.base, B.rows, B.cols, B.pitch_bytes, kBMN ? 64 : umma::kBN);
-  if (st != AF_OK) return st;
-  const uint64_t M = kAMN ? A.cols : A.rows, K = kAMN ? A.rows : A.cols;
-  const uint64_t N = kBMN ? B.cols : B.rows;
-  umma::GemmShape g;
-  g.M = (int)M; g.N = (int)N; g.K = (int)K;
-  g.m_tiles = (int)((M + umma::kBM - 1) / umma::kBM);
-  g.n_tiles = (int)((N + umma::kBN - 1) / umma::kBN);
-  g.splits = splits > 0 && splits < g.n_tiles ? splits : g.n_tiles;
-  g.k_blocks = (int)((K + umma::kBK - 1) / umma::kBK);
-  constexpr int smem = E::kStaged ? umma::kSmemBytesStaged : umma::kSmemBytes;
-  if (cudaFuncSetAttribute(umma::gemm_kernel<E, kAMN, kBMN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           smem) != cudaSuccess) return AF_ERR_CUDA;
-  const int64_t units = (int64_t)g.m_tiles * g.splits;
-  const int grid = (int)(units < ctx->sm_count ? units : ctx->sm_count);
-  umma::gemm_kernel<E, kAMN, kBMN><<<grid, umma::kThreads, smem, s>>>(ta, tb, g, ep, ctx->d_err);
-  return cudaGetLastError() == cudaSuccess ? AF_OK : AF_ERR_CUDA;
-}
-
 }  // namespace
 
 af_status launch_backward(af_ctx* ctx, const void* hidden, const void* W, const int32_t* target,
@@ -209,6 +173,7 @@ af_status launch_backward(af_ctx* ctx, const void* hidden, const void* W, const 
   const int64_t T_round = ((T + 127) / 128) * 128;
   if (Tc > T_round) Tc = T_round > 0 ? T_round : 128;
 
+  const GemmEnv env = gemm_env(ctx);
   af_status st;
   if ((st = ws_grow(ctx->dz, (size_t)Tc * V * 2)) != AF_OK) return st;
   if (accumulate_dW < 0) return AF_OK;  // reserve only
@@ -229,15 +194,16 @@ af_status launch_backward(af_ctx* ctx, const void* hidden, const void* W, const 
     const Operand dZop{dz, tc, (uint64_t)V, vB};
     // 1. dZ block:  Z = H_blk W^T, both K-major
     DzEpi::Params p1{target + t0, lse + t0, dlogp + t0, dz, (int)tc, V};
-    st = run_gemm<DzEpi, false, false>(ctx, Hblk, Wop, logprob_pick_splits((int64_t)tc, d, V, ctx->sm_count, ctx->v_splits), p1, s);
+    st = run_gemm<DzEpi, false, false>(env, Hblk, Wop,
+                                       logprob_pick_splits((int64_t)tc, d, V, ctx->sm_count, env.pair, ctx->v_splits), p1, s);
     if (st != AF_OK) return st;
     // 2. dH block = dZ W:  A = dZ (K = v contiguous), B = W read MN-major (n = d contiguous, K = v rows)
     StoreBf16Epi::Params p2{static_cast<__nv_bfloat16*>(d_hidden) + t0 * d, d, (int)tc, d};
-    st = run_gemm<StoreBf16Epi, false, true>(ctx, dZop, Wop, 0, p2, s);
+    st = run_gemm<StoreBf16Epi, false, true>(env, dZop, Wop, 0, p2, s);
     if (st != AF_OK) return st;
     // 3. dW += dZ^T H_blk:  A = dZ read MN-major (m = v contiguous, K = t rows), B = H_blk read MN-major
     StoreF32Epi::Params p3{d_W, d, V, d, (!first || accumulate_dW) ? 1 : 0};
-    st = run_gemm<StoreF32Epi, true, true>(ctx, dZop, Hblk, 0, p3, s);
+    st = run_gemm<StoreF32Epi, true, true>(env, dZop, Hblk, 0, p3, s);
     if (st != AF_OK) return st;
   }
   return AF_OK;

@@ -34,6 +34,7 @@ struct af_ctx {
   // tuning
   int v_splits = 0;         // 0 = automatic
   int bwd_token_block = 0;  // 0 = default
+  int gemm_pair = 0;        // 1 = CTA-pair GEMM variant
 
   // workspace (device)
   af::Buf partial;    // [splits, T] float4 online-softmax partials
@@ -52,11 +53,6 @@ struct af_ctx {
 namespace af {
 
 af_status ws_grow(Buf& b, size_t bytes);
-
-// Encode a 2-D bf16 tensor map: `rows` x `cols` elements, row pitch `pitch_bytes`, box of
-// `box_rows` x 64 elements, 128-byte swizzle, zero fill outside the tensor.
-af_status encode_bf16_2d(const af_ctx* ctx, CUtensorMap* map, const void* base, uint64_t rows,
-                         uint64_t cols, uint64_t pitch_bytes, uint32_t box_rows);
 
 // ---- launchers (each returns the cudaGetLastError of its launches) --------------------------
 struct PackSeqTable {     // device views into ctx->pack_meta for one call
@@ -82,7 +78,7 @@ cudaError_t launch_policy_loss(const float* logp, const float* old_logp, const f
                                float* dlogp, void* ws, unsigned int* d_err, int sm_count,
                                cudaStream_t s);
 
-int logprob_pick_splits(int64_t T, int32_t d, int32_t V, int sm_count, int requested);
+int logprob_pick_splits(int64_t T, int32_t d, int32_t V, int sm_count, bool pair, int requested);
 af_status launch_token_logprob(af_ctx* ctx, const void* hidden, const void* W,
                                const int32_t* target, int64_t T, int32_t d, int32_t V,
                                float* logp, float* entropy, float* lse, cudaStream_t s);

@@ -1,0 +1,78 @@
+// Host side of the tensor-core GEMMs: tensor-map encoding, work decomposition and the launch of
+// either variant of the main loop (one CTA per 128 x 256 tile, or a CTA pair per 256 x 256 tile).
+#pragma once
+
+#include "common.cuh"
+#include "umma.cuh"
+
+namespace af {
+
+// One operand of a GEMM launch: the matrix as it sits in memory.
+struct Operand {
+  const void* base;
+  uint64_t rows, cols;   // memory rows and (contiguous) columns
+  uint64_t pitch_bytes;
+};
+
+// What a launch needs from its surroundings (a context, or the context-free entry point).
+struct GemmEnv {
+  EncodeTiledFn encode;
+  int sm_count;
+  unsigned int* d_err;
+  bool pair;             // CTA-pair variant (cta_group::2)
+};
+
+inline af_status encode_operand(const GemmEnv& env, CUtensorMap* map, const Operand& op, uint32_t box_rows) {
+  cuuint64_t dims[2] = {op.cols, op.rows};
+  cuuint64_t strides[1] = {op.pitch_bytes};
+  cuuint32_t box[2] = {64, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = env.encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(op.base), dims, strides,
+                          box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? AF_OK : AF_ERR_CUDA;
+}
+
+// C[M,N] = sum_k A(m,k) B(n,k).  A K-major operand is stored [M or N, K]; an MN-major operand is
+// stored [K, M or N].  TMA box: 64 contiguous elements wide; K-major A 128 rows, K-major B 256
+// rows (128 per CTA of a pair), MN-major 64 K-rows.  `splits` <= 0 means one unit per B tile.
+template <class E, bool kAMN, bool kBMN>
+af_status run_gemm(const GemmEnv& env, const Operand& A, const Operand& B, int splits,
+                   const typename E::Params& ep, cudaStream_t s) {
+  CUtensorMap ta, tb;
+  af_status st = encode_operand(env, &ta, A, kAMN ? 64 : umma::kBM);
+  if (st != AF_OK) return st;
+  st = encode_operand(env, &tb, B, kBMN ? 64 : (env.pair ? umma::kBN / 2 : umma::kBN));
+  if (st != AF_OK) return st;
+  const uint64_t M = kAMN ? A.cols : A.rows, K = kAMN ? A.rows : A.cols;
+  const uint64_t N = kBMN ? B.cols : B.rows;
+  const int tile_rows = env.pair ? umma::kPairBM : umma::kBM;
+  umma::GemmShape g;
+  g.M = (int)M; g.N = (int)N; g.K = (int)K;
+  g.m_tiles = (int)((M + tile_rows - 1) / tile_rows);
+  g.n_tiles = (int)((N + umma::kBN - 1) / umma::kBN);
+  g.splits = splits > 0 && splits < g.n_tiles ? splits : g.n_tiles;
+  g.k_blocks = (int)((K + umma::kBK - 1) / umma::kBK);
+  const int64_t units = (int64_t)g.m_tiles * g.splits;
+  if (env.pair) {
+    constexpr int smem = E::kStaged ? umma::kPairSmemBytesStaged : umma::kPairSmemBytes;
+    if (cudaFuncSetAttribute(umma::gemm_pair_kernel<E, kAMN, kBMN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             smem) != cudaSuccess) return AF_ERR_CUDA;
+    const int pairs = env.sm_count / 2;
+    const int grid = 2 * (int)(units < pairs ? units : pairs);
+    umma::gemm_pair_kernel<E, kAMN, kBMN><<<grid, umma::kThreads, smem, s>>>(ta, tb, g, ep, env.d_err);
+  } else {
+    constexpr int smem = E::kStaged ? umma::kSmemBytesStaged : umma::kSmemBytes;
+    if (cudaFuncSetAttribute(umma::gemm_kernel<E, kAMN, kBMN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             smem) != cudaSuccess) return AF_ERR_CUDA;
+    const int grid = (int)(units < env.sm_count ? units : env.sm_count);
+    umma::gemm_kernel<E, kAMN, kBMN><<<grid, umma::kThreads, smem, s>>>(ta, tb, g, ep, env.d_err);
+  }
+  return cudaGetLastError() == cudaSuccess ? AF_OK : AF_ERR_CUDA;
+}
+
+inline GemmEnv gemm_env(const af_ctx* ctx) {
+  return GemmEnv{ctx->encode, ctx->sm_count, ctx->d_err, ctx->gemm_pair != 0};
+}
+
+}  // namespace af

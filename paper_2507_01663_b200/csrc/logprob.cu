@@ -8,8 +8,7 @@
 //   lse = M + log sum_i s_i e^{m_i - M},  logp = zy - lse,  entropy = lse - (sum_i u_i e^{m_i-M}) / S.
 #include <mutex>
 
-#include "common.cuh"
-#include "umma.cuh"
+#include "gemm_launch.cuh"
 
 namespace af {
 namespace {
@@ -103,28 +102,31 @@ __global__ void __launch_bounds__(256) merge_partials_kernel(
 
 }  // namespace
 
-// Number of vocabulary ranges S per row tile.  A CTA runs units b, b + grid, ..., each unit being
-// ceil(n_tiles / S) tiles long, so the launch lasts about ceil(m_tiles S / grid) * ceil(n_tiles / S)
-// tile times: S is chosen to minimise that product (wave quantisation decides it for small
-// batches).  The CTAs alive at one time sweep the vocabulary over ceil(grid / S) row tiles whose
-// hidden-state panels should stay L2-resident while W streams past once, which rules out small S
-// for wide hidden sizes.  Many ranges are only allowed while S * T stays small (partials buffer).
-int logprob_pick_splits(int64_t T, int32_t d, int32_t V, int sm_count, int requested) {
-  const int64_t m_tiles = (T + umma::kBM - 1) / umma::kBM;
+// Number of vocabulary ranges S per row tile.  A worker (a CTA, or a CTA pair) runs units w,
+// w + workers, ..., each unit being ceil(n_tiles / S) tiles long, so the launch lasts about
+// ceil(m_tiles S / workers) * ceil(n_tiles / S) tile times: S is chosen to minimise that product
+// (wave quantisation decides it for small batches).  The workers alive at one time sweep the
+// vocabulary over ceil(workers / S) row tiles whose hidden-state panels should stay L2-resident
+// while W streams past once, which rules out small S for wide hidden sizes.  Many ranges are only
+// allowed while S * T stays small (partials buffer).
+int logprob_pick_splits(int64_t T, int32_t d, int32_t V, int sm_count, bool pair, int requested) {
+  const int tile_rows = pair ? umma::kPairBM : umma::kBM;
+  const int workers = pair ? (sm_count / 2 > 0 ? sm_count / 2 : 1) : (sm_count > 0 ? sm_count : 1);
+  const int64_t m_tiles = (T + tile_rows - 1) / tile_rows;
   const int n_tiles = (V + umma::kBN - 1) / umma::kBN;
   if (requested > 0) return requested < n_tiles ? requested : n_tiles;
-  if (m_tiles < 1 || sm_count < 1) return 1;
+  if (m_tiles < 1) return 1;
   constexpr int64_t kPanelBudget = 72ll << 20;        // bytes of hidden-state rows kept in L2
-  const int64_t max_units_many = (int64_t)sm_count * 8;
+  const int64_t max_units_many = (int64_t)workers * 8;
   int best = 1;
   double best_cost = 1e300;
   for (int S = 1; S <= 32 && S <= n_tiles; ++S) {
     const int64_t units = m_tiles * S;
     if (S > 4 && units > max_units_many) break;
-    int64_t alive = (sm_count + S - 1) / S;
+    int64_t alive = (workers + S - 1) / S;
     if (alive > m_tiles) alive = m_tiles;
-    const bool fits = alive * umma::kBM * (int64_t)d * 2 <= kPanelBudget;
-    const int64_t grid = units < sm_count ? units : sm_count;
+    const bool fits = alive * tile_rows * (int64_t)d * 2 <= kPanelBudget;
+    const int64_t grid = units < workers ? units : workers;
     double cost = (double)((units + grid - 1) / grid) * (double)((n_tiles + S - 1) / S);
     cost *= 1.0 + 0.002 * S;                          // partials written and merged per range
     if (!fits) cost *= 1.25;                          // W re-read from HBM by every row tile
@@ -137,34 +139,15 @@ af_status launch_token_logprob(af_ctx* ctx, const void* hidden, const void* W,
                                const int32_t* target, int64_t T, int32_t d, int32_t V,
                                float* logp, float* entropy, float* lse, cudaStream_t s) {
   if (T == 0) return AF_OK;
-  const int S = logprob_pick_splits(T, d, V, ctx->sm_count, ctx->v_splits);
+  const GemmEnv env = gemm_env(ctx);
+  const int S = logprob_pick_splits(T, d, V, ctx->sm_count, env.pair, ctx->v_splits);
   af_status st = ws_grow(ctx->partial, (size_t)S * (size_t)T * sizeof(float4));
   if (st != AF_OK) return st;
-
-  CUtensorMap ta, tb;
-  st = encode_bf16_2d(ctx, &ta, hidden, (uint64_t)T, (uint64_t)d, (uint64_t)d * 2, umma::kBM);
-  if (st != AF_OK) return st;
-  st = encode_bf16_2d(ctx, &tb, W, (uint64_t)V, (uint64_t)d, (uint64_t)d * 2, umma::kBN);
-  if (st != AF_OK) return st;
-
-  umma::GemmShape g;
-  g.M = (int)T; g.N = V; g.K = d;
-  g.m_tiles = (int)((T + umma::kBM - 1) / umma::kBM);
-  g.n_tiles = (V + umma::kBN - 1) / umma::kBN;
-  g.splits = S;
-  g.k_blocks = (d + umma::kBK - 1) / umma::kBK;
+  const Operand Hop{hidden, (uint64_t)T, (uint64_t)d, (uint64_t)d * 2};
+  const Operand Wop{W, (uint64_t)V, (uint64_t)d, (uint64_t)d * 2};
   LogprobEpi::Params ep{target, (float4*)ctx->partial.p, (int)T, V};
-
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(umma::gemm_kernel<LogprobEpi>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             umma::kSmemBytes) != cudaSuccess) return AF_ERR_CUDA;
-    attr_set = true;
-  }
-  const int64_t units = (int64_t)g.m_tiles * S;
-  const int grid = (int)(units < ctx->sm_count ? units : ctx->sm_count);
-  umma::gemm_kernel<LogprobEpi><<<grid, umma::kThreads, umma::kSmemBytes, s>>>(ta, tb, g, ep, ctx->d_err);
-  if (cudaGetLastError() != cudaSuccess) return AF_ERR_CUDA;
+  st = run_gemm<LogprobEpi, false, false>(env, Hop, Wop, S, ep, s);
+  if (st != AF_OK) return st;
   merge_partials_kernel<<<(int)((T + 255) / 256), 256, 0, s>>>((const float4*)ctx->partial.p, target,
                                                               (int)T, V, S, logp, entropy, lse,
                                                               ctx->d_err);
@@ -203,7 +186,7 @@ EncodeTiledFn g_static_encode = nullptr;
 std::mutex g_static_mutex;
 
 // Once per device, with that device current: resolve the scratch address, read the SM count,
-// fetch the tensor-map encoder and raise the kernel's dynamic shared memory limit.
+// and fetch the tensor-map encoder.
 af_status static_setup(int dev, StaticDeviceState** out) {
   if (dev < 0 || dev >= kStaticMaxDevices) return AF_ERR_UNSUPPORTED_DEVICE;
   std::lock_guard<std::mutex> lock(g_static_mutex);
@@ -228,27 +211,12 @@ af_status static_setup(int dev, StaticDeviceState** out) {
         return AF_ERR_CUDA;
       g_static_encode = reinterpret_cast<EncodeTiledFn>(fn);
     }
-    if (cudaFuncSetAttribute(umma::gemm_kernel<LogprobEpi>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             umma::kSmemBytes) != cudaSuccess)
-      return AF_ERR_CUDA;
     st.scratch = static_cast<unsigned char*>(p);
     st.sm_count = sms;
     st.ready = true;
   }
   *out = &st;
   return AF_OK;
-}
-
-af_status static_encode_2d(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols,
-                           uint32_t box_rows) {
-  cuuint64_t dims[2] = {cols, rows};
-  cuuint64_t strides[1] = {cols * 2};
-  cuuint32_t box[2] = {64, box_rows};
-  cuuint32_t estr[2] = {1, 1};
-  return g_static_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides,
-                         box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                         CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS
-             ? AF_OK : AF_ERR_CUDA;
 }
 
 }  // namespace
@@ -271,26 +239,17 @@ extern "C" af_status af_token_logprob_static(const void* hidden, const void* W, 
   if (d % 8 != 0 || (reinterpret_cast<uintptr_t>(hidden) & 15u) || (reinterpret_cast<uintptr_t>(W) & 15u))
     return AF_ERR_ALIGNMENT;
 
-  int S = logprob_pick_splits(T, d, V, st->sm_count, 0);
+  int S = logprob_pick_splits(T, d, V, st->sm_count, false, 0);
   if ((int64_t)S * T > kStaticPartialSlots) S = (int)(kStaticPartialSlots / T);
   unsigned int* err_word = device_flags ? device_flags : reinterpret_cast<unsigned int*>(st->scratch);
   float4* partial = reinterpret_cast<float4*>(st->scratch + kStaticHeaderBytes);
 
-  CUtensorMap ta, tb;
-  if ((rc = static_encode_2d(&ta, hidden, (uint64_t)T, (uint64_t)d, umma::kBM)) != AF_OK) return rc;
-  if ((rc = static_encode_2d(&tb, W, (uint64_t)V, (uint64_t)d, umma::kBN)) != AF_OK) return rc;
-  umma::GemmShape g;
-  g.M = (int)T; g.N = V; g.K = d;
-  g.m_tiles = (int)((T + umma::kBM - 1) / umma::kBM);
-  g.n_tiles = (V + umma::kBN - 1) / umma::kBN;
-  g.splits = S;
-  g.k_blocks = (d + umma::kBK - 1) / umma::kBK;
+  const GemmEnv env{g_static_encode, st->sm_count, err_word, false};
+  const Operand Hop{hidden, (uint64_t)T, (uint64_t)d, (uint64_t)d * 2};
+  const Operand Wop{W, (uint64_t)V, (uint64_t)d, (uint64_t)d * 2};
   LogprobEpi::Params ep{target, partial, (int)T, V};
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  const int64_t units = (int64_t)g.m_tiles * S;
-  const int grid = (int)(units < st->sm_count ? units : st->sm_count);
-  umma::gemm_kernel<LogprobEpi><<<grid, umma::kThreads, umma::kSmemBytes, s>>>(ta, tb, g, ep, err_word);
-  if (cudaGetLastError() != cudaSuccess) return AF_ERR_CUDA;
+  if ((rc = run_gemm<LogprobEpi, false, false>(env, Hop, Wop, S, ep, s)) != AF_OK) return rc;
   merge_partials_kernel<<<(int)((T + 255) / 256), 256, 0, s>>>(partial, target, (int)T, V, S, logp, entropy,
                                                               lse, err_word);
   return cudaGetLastError() == cudaSuccess ? AF_OK : AF_ERR_CUDA;

@@ -354,5 +354,240 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
   }
 }
 
+
+// ==========================================================================================
+// CTA-pair variant (cta_group::2).  Two CTAs of a cluster, on the two SMs of one pair, compute a
+// 256 x 256 tile together: each holds 128 rows of A and 128 of the 256 rows of B in its own
+// shared memory and 128 rows of the fp32 accumulator in its own tensor memory; one thread of the
+// pair's first CTA (the leader) issues every MMA for both.  Per 128 x 256 x 64 block of work a SM
+// now stages 32 KB instead of 48 KB, which deepens the ring to 6 stages and takes a third off the
+// L2 -> shared-memory traffic.
+//
+// Barriers (same shared-memory offsets in both CTAs):
+//   full[s]   leader's copy only: one arrival (the leader's producer, with the byte count of both
+//             CTAs' copies); each CTA's TMA loads complete on it.
+//   empty[s]  per CTA: the leader's MMA thread commits to both copies at once.
+//   tfull[a]  per CTA: accumulator a complete (committed to both copies at once).
+//   tempty[a] leader's copy only: one arrival per epilogue warp of either CTA (8 in all).
+// No load is multicast; every CTA fetches its own operand halves.
+// ==========================================================================================
+constexpr int kPairBM = 256;                                  // rows of A per pair tile
+constexpr int kPairStages = 6;
+constexpr int kPairBBytes = (kBN / 2) * kBK * 2;              // this CTA's half of the B tile
+constexpr int kPairStageBytes = kABytes + kPairBBytes;        // 32 KB
+constexpr int kPairSmemBytes = kPairStages * kPairStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int kPairSmemBytesStaged = kPairSmemBytes + 4 * kEpiStageBytes;
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Arrive on the barrier at the same shared-memory offset in CTA `rank` of the cluster.
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar, uint32_t rank) {
+  asm volatile(
+      "{\n\t.reg .b32 ra;\n\t"
+      "mapa.shared::cluster.u32 ra, %0, %1;\n\t"
+      "mbarrier.arrive.release.cluster.shared::cluster.b64 _, [ra];\n\t}"
+      ::"r"(bar), "r"(rank) : "memory");
+}
+// Cluster-wide address of the shared-memory location `addr` of CTA `rank`.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+// TMA tile load of a CTA pair: data lands in this CTA's shared memory, the bytes are counted on
+// `leader_bar`, a barrier of the pair's leader given by its cluster-wide address.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst_smem, const CUtensorMap* map,
+                                                 uint32_t leader_bar, int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst_smem), "l"(map), "r"(leader_bar), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t dst_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+// D[tmem of both CTAs] (+)= A * B^T, 256 x 256 x 16 over the pair.
+__device__ __forceinline__ void mma_bf16_ss_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                                 uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// Arrive on `bar` in both CTAs of the pair once every MMA issued so far has completed.
+__device__ __forceinline__ void mma_commit_pair(uint32_t bar) {
+  asm volatile(
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+      ::"r"(bar), "h"((unsigned short)3) : "memory");
+}
+
+// Work decomposition of the pair kernel: a unit is one 256-row tile times a range of B tiles;
+// pair p processes units p, p + n_pairs, ...
+template <class E, bool kAMN = false, bool kBMN = false>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                 const GemmShape g, const typename E::Params ep, unsigned int* d_err) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t tiles = (raw + 1023u) & ~1023u;
+  const uint32_t bars = tiles + kPairStages * kPairStageBytes;
+  auto full_bar = [&](int s) { return bars + 8u * s; };
+  auto empty_bar = [&](int s) { return bars + 8u * (kPairStages + s); };
+  auto tfull_bar = [&](int a) { return bars + 8u * (2 * kPairStages + a); };
+  auto tempty_bar = [&](int a) { return bars + 8u * (2 * kPairStages + 2 + a); };
+  const uint32_t tmem_slot = bars + 8u * (2 * kPairStages + 4);
+  uint8_t* const epi_stage_base = smem_raw + (bars + 256u - raw);
+  volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(smem_raw + (tmem_slot - raw));
+  __shared__ int abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();          // 0 = leader
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    for (int s = 0; s < kPairStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 8); }
+    fence_mbar_init();
+    tma_prefetch_desc(&tmap_a);
+    tma_prefetch_desc(&tmap_b);
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(tmem_slot, kTmemCols);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();       // the peer's barriers exist before anything is signalled across CTAs
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot_ptr;
+
+  const int total_units = g.m_tiles * g.splits;     // m_tiles counts 256-row tiles here
+
+  if (warp == 0) {
+    // ---------------------------------------------------------------- TMA producer (both CTAs)
+    if (lane == 0) {
+      int stage = 0; uint32_t phase = 0; bool ok = true;
+      const uint32_t leader_full0 = map_to_cta(full_bar(0), 0);
+      for (int u = pair; u < total_units && ok; u += n_pairs) {
+        const int m_tile = u / g.splits, s = u % g.splits;
+        const int nb = split_begin(g, s), ne = split_begin(g, s + 1);
+        const int m0 = m_tile * kPairBM + (int)rank * kBM;          // this CTA's 128 rows of A
+        for (int nt = nb; nt < ne && ok; ++nt) {
+          const int n0 = nt * kBN + (int)rank * (kBN / 2);          // this CTA's 128 rows of B
+          for (int kb = 0; kb < g.k_blocks; ++kb) {
+            if (!mbar_wait(empty_bar(stage), phase ^ 1u, &abort_flag)) { ok = false; break; }
+            const uint32_t a_dst = tiles + stage * kPairStageBytes;
+            const uint32_t lbar = leader_full0 + 8u * stage;
+            if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), 2 * kPairStageBytes);
+            if constexpr (kAMN) {
+#pragma unroll
+              for (int b = 0; b < kBM / 64; ++b)
+                tma_load_2d_pair(a_dst + b * kMnBoxBytes, &tmap_a, lbar, m0 + b * 64, kb * kBK);
+            } else {
+              tma_load_2d_pair(a_dst, &tmap_a, lbar, kb * kBK, m0);
+            }
+            if constexpr (kBMN) {
+#pragma unroll
+              for (int b = 0; b < kBN / 128; ++b)
+                tma_load_2d_pair(a_dst + kABytes + b * kMnBoxBytes, &tmap_b, lbar, n0 + b * 64, kb * kBK);
+            } else {
+              tma_load_2d_pair(a_dst + kABytes, &tmap_b, lbar, kb * kBK, n0);
+            }
+            if (++stage == kPairStages) { stage = 0; phase ^= 1u; }
+          }
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ---------------------------------------------------------------- MMA issuer (leader only)
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = instr_desc_bf16_f32(kPairBM, kBN, kAMN, kBMN);
+      constexpr uint64_t a_step = kAMN ? (2048 >> 4) : 2, b_step = kBMN ? (2048 >> 4) : 2;
+      int stage = 0; uint32_t phase = 0; uint32_t tile_count = 0; bool ok = true;
+      for (int u = pair; u < total_units && ok; u += n_pairs) {
+        const int s = u % g.splits;
+        const int nb = split_begin(g, s), ne = split_begin(g, s + 1);
+        for (int nt = nb; nt < ne && ok; ++nt, ++tile_count) {
+          const uint32_t acc = tile_count & 1u, acc_phase = (tile_count >> 1) & 1u;
+          if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, &abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t d_tmem = tmem_base + acc * kBN;
+          for (int kb = 0; kb < g.k_blocks; ++kb) {
+            if (!mbar_wait(full_bar(stage), phase, &abort_flag)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t a_addr = tiles + stage * kPairStageBytes;
+            const uint64_t a_desc = kAMN ? smem_desc_mn_sw128(a_addr) : smem_desc_k_sw128(a_addr);
+            const uint64_t b_desc = kBMN ? smem_desc_mn_sw128(a_addr + kABytes) : smem_desc_k_sw128(a_addr + kABytes);
+#pragma unroll
+            for (int k = 0; k < kBK / kUmmaK; ++k) {
+              mma_bf16_ss_pair(d_tmem, a_desc + (uint64_t)k * a_step, b_desc + (uint64_t)k * b_step, idesc,
+                               (kb | k) != 0 ? 1u : 0u);
+            }
+            mma_commit_pair(empty_bar(stage));   // both CTAs' slots reusable once these MMAs have read them
+            if (++stage == kPairStages) { stage = 0; phase ^= 1u; }
+          }
+          if (ok) mma_commit_pair(tfull_bar(acc));  // accumulator complete in both CTAs
+        }
+      }
+    }
+    __syncwarp();
+  } else {
+    // ---------------------------------------------------------------- epilogue (warps 2..5, both CTAs)
+    const int quarter = warp & 3;
+    const int row_in_tile = (int)rank * kBM + quarter * 32 + lane;
+    uint32_t tile_count = 0; bool ok = true;
+    typename E::State st;
+    uint8_t* const stage = E::kStaged ? epi_stage_base + (warp - 2) * kEpiStageBytes : nullptr;
+    for (int u = pair; u < total_units && ok; u += n_pairs) {
+      const int m_tile = u / g.splits, s = u % g.splits;
+      const int nb = split_begin(g, s), ne = split_begin(g, s + 1);
+      const int row = m_tile * kPairBM + row_in_tile;
+      E::unit_begin(st, ep, row, m_tile, s);
+      for (int nt = nb; nt < ne && ok; ++nt, ++tile_count) {
+        const uint32_t acc = tile_count & 1u, acc_phase = (tile_count >> 1) & 1u;
+        if (!__all_sync(0xffffffffu, mbar_wait(tfull_bar(acc), acc_phase, &abort_flag))) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * kBN;
+#pragma unroll 1
+        for (int c = 0; c < kBN / 32; ++c) {
+          uint32_t v[32];
+          tmem_ld32(t_row + c * 32, v);
+          tmem_ld_wait();
+          E::chunk(st, ep, row, nt * kBN + c * 32, v, stage);
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(tempty_bar(acc), 0);   // one arrival per warp, on the leader
+      }
+      if (ok) E::unit_end(st, ep, row, s);
+    }
+  }
+
+  // ---------------------------------------------------------------- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && abort_flag) atomicOr(d_err, kWatchdogBit);
+  if (abort_flag) __nanosleep(1000000);  // let copies in flight land before the CTA retires
+  cluster_sync_all();   // neither CTA leaves while the other may still touch its memory or barriers
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc_pair(tmem_base, kTmemCols);
+  }
+}
+
 }  // namespace umma
 }  // namespace af

@@ -12,6 +12,19 @@ from gpu_util import GRAD_RTOL, device, f32, np_of
 pytestmark = pytest.mark.gpu
 
 
+PAIR = False   # which GEMM variant the helpers below select
+
+
+@pytest.fixture(autouse=True, params=[False, True], ids=["cta", "pair"])
+def gemm_variant(request):
+    """Every test of this module runs on both tensor-core main loops: one CTA per 128 x 256
+    tile (the default) and a CTA pair per 256 x 256 tile."""
+    global PAIR
+    PAIR = request.param
+    yield
+    PAIR = False
+
+
 @pytest.fixture(scope="module")
 def ctx():
     from paper_2507_01663_b200 import binding as B
@@ -35,7 +48,7 @@ def run_bwd(ctx, H, W, y, g, lse, token_block=0, accumulate=False, dW_init=None)
     V = W.shape[0]
     dH = torch.full((max(T, 1), d), 7.0, dtype=torch.bfloat16, device=dev)
     dW = torch.full((V, d), 7.0, device=dev) if dW_init is None else dW_init.clone()
-    ctx.set_tuning(0, token_block)
+    ctx.set_tuning(0, token_block, PAIR)
     ctx.policy_loss_backward(H.to(dev), W.to(dev), y.to(dev), f32(lse), g.to(dev), dH, dW, accumulate, T=T)
     flags = ctx.check_device_errors()
     ctx.set_tuning(0, 0)
@@ -82,6 +95,7 @@ def test_cfg4_mini_chain(ctx):
     # GPU chain
     Hd, Wd, yd = H.to(dev), W.to(dev), y.to(dev)
     logp_d, ent_d, lse_d, g_d = (torch.empty(T, device=dev) for _ in range(4))
+    ctx.set_tuning(0, 0, PAIR)
     ctx.token_logprob(Hd, Wd, yd, logp_d, ent_d, lse_d)
     out = B.new_loss_out(dev)
     ctx.policy_loss(logp_d, old.to(dev), ref.to(dev), f32(adv), torch.as_tensor(cu.astype(np.int32), device=dev), out,
@@ -89,6 +103,7 @@ def test_cfg4_mini_chain(ctx):
     dH = torch.empty(T, w.d, dtype=torch.bfloat16, device=dev)
     dW = torch.empty(w.V, w.d, device=dev)
     ctx.policy_loss_backward(Hd, Wd, yd, lse_d, g_d, dH, dW)
+    ctx.set_tuning(0, 0)
     res = B.read_loss_out(out)
     assert ctx.check_device_errors() == 0
     assert abs(res["loss"] - oref["loss"]) <= 1e-3 * abs(oref["loss"])
