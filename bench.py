@@ -154,53 +154,63 @@ class ScoringJob:
         self.store["ref_logp"] = centre + wl.gen_noise(w, wl.S_REF, T, device)
         del centre
         self.adv = torch.empty(w.N, device=device)
-        self.idx = wl.arrival_order(w)
+        # micro-batches: the whole arrival-ordered batch, or (streaming store) greedy arrival-ordered
+        # index lists under the workload's token budget, issued back to back on one stream
+        self.mbs = wl.microbatches(w)
+        self.idx = self.mbs[0]
         self.off = w.tok_offset
+        cap_T = max(int(w.lengths[m].sum()) for m in self.mbs)
+        cap_B = max(len(m) for m in self.mbs)
         self.packed = {
-            "cu_seqlens": torch.zeros(w.N + 1, dtype=torch.int32, device=device),
-            "hidden": torch.empty(T, w.d, dtype=torch.bfloat16, device=device),
-            "target": torch.empty(T, dtype=torch.int32, device=device),
-            "old_logp": torch.empty(T, device=device), "ref_logp": torch.empty(T, device=device),
-            "adv_seq": torch.empty(w.N, device=device),
+            "cu_seqlens": torch.zeros(cap_B + 1, dtype=torch.int32, device=device),
+            "hidden": torch.empty(cap_T, w.d, dtype=torch.bfloat16, device=device),
+            "target": torch.empty(cap_T, dtype=torch.int32, device=device),
+            "old_logp": torch.empty(cap_T, device=device), "ref_logp": torch.empty(cap_T, device=device),
+            "adv_seq": torch.empty(cap_B, device=device),
         }
-        self.logp, self.ent, self.lse, self.dlogp = (torch.empty(T, device=device) for _ in range(4))
-        self.loss_out = B.new_loss_out(device)
+        self.logp, self.ent, self.lse, self.dlogp = (torch.empty(cap_T, device=device) for _ in range(4))
+        self.loss_outs = [B.new_loss_out(device) for _ in self.mbs]
+        self.loss_out = self.loss_outs[-1]
         if w.backward:
-            self.d_hidden = torch.empty(T, w.d, dtype=torch.bfloat16, device=device)
+            self.d_hidden = torch.empty(cap_T, w.d, dtype=torch.bfloat16, device=device)
             self.d_W = torch.empty(w.V, w.d, device=device)
-        self.ctx.reserve(T, w.N, w.d, w.V, with_backward=w.backward)
+        self.ctx.reserve(cap_T, cap_B, w.d, w.V, with_backward=w.backward)
         self.gemm_events, self.pack_events, self.bwd_events = [], [], []
-        self.launches_per_step = KERNELS_PER_STEP + (3 * -(-T // BWD_TOKEN_BLOCK) if w.backward else 0)
+        per_mb = KERNELS_PER_STEP - 1 + (3 * -(-cap_T // BWD_TOKEN_BLOCK) if w.backward else 0)
+        self.launches_per_step = 1 + per_mb * len(self.mbs)
 
     def step(self, time_gemm: bool = False):
         w, c = self.w, self.ctx
         c.grpo_advantage(self.reward, None, w.n_prompts, self.adv)
         store = {"tok_offset_host": self.off, "d": w.d, "adv": self.adv, **self.store}
-        ev = [torch.cuda.Event(enable_timing=True) for _ in range(6)] if time_gemm else None
-        if ev:
-            ev[0].record()
-        T = c.pack_microbatch(store, self.idx, self.packed)
-        if ev:
-            ev[1].record()
-            ev[2].record()
-        c.token_logprob(self.packed["hidden"], self.W, self.packed["target"], self.logp, self.ent, self.lse, T=T)
-        if ev:
-            ev[3].record()
-        c.policy_loss(self.logp, self.packed["old_logp"], self.packed["ref_logp"], self.packed["adv_seq"],
-                      self.packed["cu_seqlens"], self.loss_out, self.dlogp, self.ent,
-                      w.clip_eps, w.clip_eps, w.kl_coef, 0, 1.0, B=w.N, T=T)
-        if w.backward:
+        total = 0
+        for mb, loss_out in zip(self.mbs, self.loss_outs):
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(6)] if time_gemm else None
             if ev:
-                ev[4].record()
-            c.policy_loss_backward(self.packed["hidden"], self.W, self.packed["target"], self.lse, self.dlogp,
-                                   self.d_hidden, self.d_W, False, T=T)
+                ev[0].record()
+            T = c.pack_microbatch(store, mb, self.packed)
             if ev:
-                ev[5].record()
-                self.bwd_events.append((ev[4], ev[5]))
-        if ev:
-            self.pack_events.append((ev[0], ev[1]))
-            self.gemm_events.append((ev[2], ev[3]))
-        return T
+                ev[1].record()
+                ev[2].record()
+            c.token_logprob(self.packed["hidden"], self.W, self.packed["target"], self.logp, self.ent, self.lse, T=T)
+            if ev:
+                ev[3].record()
+            c.policy_loss(self.logp, self.packed["old_logp"], self.packed["ref_logp"], self.packed["adv_seq"],
+                          self.packed["cu_seqlens"], loss_out, self.dlogp, self.ent,
+                          w.clip_eps, w.clip_eps, w.kl_coef, 0, 1.0, B=len(mb), T=T)
+            if w.backward:
+                if ev:
+                    ev[4].record()
+                c.policy_loss_backward(self.packed["hidden"], self.W, self.packed["target"], self.lse, self.dlogp,
+                                       self.d_hidden, self.d_W, False, T=T)
+                if ev:
+                    ev[5].record()
+                    self.bwd_events.append((ev[4], ev[5]))
+            if ev:
+                self.pack_events.append((ev[0], ev[1]))
+                self.gemm_events.append((ev[2], ev[3]))
+            total += T
+        return total
 
     def hbm_kernels_at_scale(self, peak_gbs: float) -> dict:
         """The memory-bound kernels timed alone, before the long GEMM loop heats the part (the
@@ -224,9 +234,10 @@ class ScoringJob:
         w = self.w
         store = {"tok_offset_host": self.off, "d": w.d, "adv": self.adv, **self.store}
         ms = avg_ms(lambda: c.pack_microbatch(store, self.idx, self.packed))
-        nbytes = 2.0 * self.T * (2 * w.d + 12) + 8.0 * w.N
+        t_mb = int(w.lengths[self.idx].sum())
+        nbytes = 2.0 * t_mb * (2 * w.d + 12) + 8.0 * len(self.idx)
         gbs = nbytes / ms / 1e6
-        out["pack_microbatch"] = {"tokens": self.T, "bytes_per_token": 2 * (2 * w.d + 12), "ms": ms, "gbs": gbs,
+        out["pack_microbatch"] = {"tokens": t_mb, "bytes_per_token": 2 * (2 * w.d + 12), "ms": ms, "gbs": gbs,
                                   "frac": gbs / peak_gbs, "where": "timed alone, 10 calls (2 kernels + metadata copy each)"}
         n = 1 << 26
         seq = 1024
@@ -241,7 +252,7 @@ class ScoringJob:
         del logp, old, ref, ent, g
         r = wl.uniform01(self.w.seed, wl.S_REWARD, 0, 1 << 20, dev).repeat(n >> 20)
         a = torch.empty(n, device=dev)
-        G = self.w.group_size if self.w.group_size <= 32 else 8
+        G = self.w.group_size
         ms = avg_ms(lambda: c.grpo_advantage(r, None, n // G, a))
         gbs = 8.0 * n / ms / 1e6
         out["grpo_advantage"] = {"responses": n, "group_size": G, "bytes_per_response": 8, "ms": ms, "gbs": gbs,
@@ -257,14 +268,15 @@ class ScoringJob:
         self.host["reward"].copy_(self.reward)
         torch.cuda.synchronize()
         self.h2d_bytes = sum(t.numel() * t.element_size() for t in self.host.values())
-        self.host_loss = torch.empty(self.loss_out.shape, dtype=torch.uint8, pin_memory=True)
+        self.host_loss = [torch.empty(lo.shape, dtype=torch.uint8, pin_memory=True) for lo in self.loss_outs]
 
     def step_e2e(self):
         for k, v in self.store.items():
             v.copy_(self.host[k], non_blocking=True)
         self.reward.copy_(self.host["reward"], non_blocking=True)
         T = self.step()
-        self.host_loss.copy_(self.loss_out, non_blocking=True)
+        for h, lo in zip(self.host_loss, self.loss_outs):
+            h.copy_(lo, non_blocking=True)
         return T
 
 
@@ -331,9 +343,10 @@ def run_ours(args):
         sampler.start()
     ms_total = timed_loop(lambda: job.step(time_gemm=True), args.steps, world)
     clocks = sampler.stop() if rank == 0 else None
-    gemm_ms = float(np.mean([a.elapsed_time(b) for a, b in job.gemm_events]))
-    pack_ms = float(np.mean([a.elapsed_time(b) for a, b in job.pack_events]))
-    bwd_ms = float(np.mean([a.elapsed_time(b) for a, b in job.bwd_events])) if job.bwd_events else None
+    # per step: summed over the step's micro-batches
+    gemm_ms = float(np.sum([a.elapsed_time(b) for a, b in job.gemm_events])) / args.steps
+    pack_ms = float(np.sum([a.elapsed_time(b) for a, b in job.pack_events])) / args.steps
+    bwd_ms = float(np.sum([a.elapsed_time(b) for a, b in job.bwd_events])) / args.steps if job.bwd_events else None
     ms_step, tokens = reduce_over_ranks(ms_total / args.steps, job.T, world)
     flags = job.ctx.check_device_errors()
     if flags:
@@ -356,7 +369,10 @@ def run_ours(args):
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": f"{args.workload}: {head_name(w)} head d={w.d} V={w.V}, {w.N} responses "
                                f"({w.n_prompts} prompts x {w.group_size}), {job.T} scored tokens per GPU, "
-                               "one arrival-ordered packed micro-batch" + (", forward + backward (dH, dW)" if w.backward else ""),
+                               + (f"{len(job.mbs)} arrival-ordered micro-batches of <= {w.token_budget} tokens, packed, "
+                                  "scored and loss-reduced back to back on one stream" if w.token_budget
+                                  else "one arrival-ordered packed micro-batch")
+                               + (", forward + backward (dH, dW)" if w.backward else ""),
                    "l2": "inputs (hidden states >> 126 MB L2) exceed L2; no flush needed",
                    "gemm": "CTA pairs (cta_group::2)" if args.gemm_pair else "one CTA per tile",
                    "loss": {"clip_eps": w.clip_eps, "kl_coef": w.kl_coef, "agg": "seq-mean-token-mean"}},
@@ -368,7 +384,7 @@ def run_ours(args):
                      "traffic": (GEMM_DRAM_BYTES_PER_TOKEN_7B * job.T
                                  if GEMM_DRAM_BYTES_PER_TOKEN_7B and (w.d, w.V) == (3584, 152064) else None)},
         "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": job.h2d_bytes,
-                "d2h_bytes_per_step": int(job.loss_out.numel()), "ms_per_step": ms_e2e},
+                "d2h_bytes_per_step": int(sum(lo.numel() for lo in job.loss_outs)), "ms_per_step": ms_e2e},
         "gpu_launches": job.launches_per_step * args.steps,
         "clocks": clocks, "loss": loss,
     }
@@ -377,8 +393,8 @@ def run_ours(args):
     line["hbm_kernels"] = {"peak_gbs": peaks["hbm_gbs"], "peak_source": f"hbm_gbs, {peaks['source']}",
                            "pack_microbatch_in_step": {"tokens": job.T, "bytes_per_token": 2 * (2 * w.d + 12),
                                                        "ms": pack_ms, "gbs": pack_gbs, "frac": pack_gbs / peaks["hbm_gbs"],
-                                                       "where": "inside the timed steps, right after the previous "
-                                                                "step's GEMM (part at its power cap)"}}
+                                                       "where": "inside the timed steps (all micro-batches of a step), "
+                                                                "each right after a GEMM (part at its power cap)"}}
     line["hbm_kernels"].update(hbm_alone)
     if bwd_ms is not None:
         bflops = 6.0 * job.T * w.d * w.V
