@@ -51,6 +51,7 @@ typedef enum {
 #define AF_DEVERR_TARGET_RANGE 1u /* a target id was outside [0, V): that token's outputs are NaN */
 #define AF_DEVERR_WATCHDOG 2u     /* a bounded wait inside a kernel ran out; results invalid      */
 #define AF_DEVERR_CU_SEQLENS 4u   /* cu_seqlens not non-decreasing from 0 to T                     */
+#define AF_DEVERR_SAMPLE_INDEX 8u /* af_controller_put met an index outside [0, N): entry skipped  */
 
 /* Create / destroy a context on CUDA device `device`.  af_create fails with
  * AF_ERR_UNSUPPORTED_DEVICE unless the device is compute capability 10.0.  af_destroy
@@ -217,6 +218,84 @@ af_status af_policy_loss_backward(af_ctx* ctx, const void* hidden, const void* W
                                   const int32_t* target, const float* lse, const float* dlogp,
                                   int64_t T, int32_t d, int32_t V, void* d_hidden, float* d_W,
                                   int32_t accumulate_dW, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * af_controller_put / af_controller_get / af_controller_clear -- the status table of the
+ * streaming store and one read request against it.
+ *
+ * The paper's TransferQueue controller keeps, per sample, a binary "written" indicator for every
+ * column and a consumption record per RL task; a `get` request builds the mask of the requested
+ * columns, finds the samples whose requested columns are all written and that the requesting
+ * task has not been handed yet, selects the required number of them, returns their metadata and
+ * marks them consumed; storage units report finished writes, which turns indicators on (Section
+ * 4.4 "Control Plane: Panoramic Data Admin" with its figure of the get procedure; Section 4.2).
+ * Here the table lives on the device next to the store it describes:
+ *   ready[i]    bit c set  <=>  column c of sample i has been written       (c in 0..31)
+ *   consumed[i] bit t set  <=>  sample i has been handed to task t           (t in 0..31)
+ *   length[i]   tokens of sample i (only needed for token budgets)
+ *
+ * put:   ready[idx[j]] |= column_bits for j in [0, n); idx is a DEVICE array (for instance the
+ *        out_idx of the get that handed the samples out).  An index outside [0, N) is skipped
+ *        and sets AF_DEVERR_SAMPLE_INDEX.
+ * get:   sample i is eligible iff (ready[i] & column_mask) == column_mask and
+ *        (consumed[i] & task_bit) == 0.  The paper does not say how "the required number" is
+ *        chosen; this call takes eligible samples in increasing index and returns the longest
+ *        prefix of them with at most max_samples entries and, when token_budget > 0, at most
+ *        token_budget tokens in total -- except that a first eligible sample longer than the
+ *        whole budget is returned alone.  out_idx[0 .. count) (device, capacity max_samples)
+ *        receives the indices in increasing order, *out (device) the record below, and the
+ *        returned samples get task_bit set in consumed.  The result is unique (integer work).
+ * clear: ready[i] &= ~column_bits, consumed[i] &= ~task_bits for every sample (a new iteration).
+ *
+ * All three enqueue on `stream` and return; read *out / out_idx after synchronising (or place
+ * them in mapped pinned memory).  Calls on one table must not overlap on the GPU.
+ * Errors: AF_ERR_INVALID_ARG for null pointers, negative sizes, max_samples < 0, a task_bit that
+ * is not a single bit, or token_budget > 0 without length; AF_ERR_SHAPE for N >= 2^31.
+ * ------------------------------------------------------------------------------------------- */
+typedef struct {
+  int64_t n_samples;        /* N                                       */
+  uint32_t* ready;          /* [N] dev                                 */
+  uint32_t* consumed;       /* [N] dev                                 */
+  const int32_t* length;    /* [N] dev, or NULL (no token budgets)     */
+} af_controller_view;
+
+typedef struct {
+  int32_t count;            /* samples returned                                         */
+  int32_t eligible;         /* eligible samples in the table when the request was made  */
+  int64_t tokens;           /* their token total (0 without length)                     */
+} af_get_result;
+
+af_status af_controller_put(af_ctx* ctx, const af_controller_view* table, const int32_t* idx,
+                            int64_t n, uint32_t column_bits, void* stream);
+af_status af_controller_get(af_ctx* ctx, const af_controller_view* table, uint32_t column_mask,
+                            uint32_t task_bit, int32_t max_samples, int64_t token_budget,
+                            int32_t* out_idx, af_get_result* out, void* stream);
+af_status af_controller_clear(af_ctx* ctx, const af_controller_view* table, uint32_t column_bits,
+                              uint32_t task_bits, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * af_balance_partitions -- token-balanced split of a batch over k groups (host call, no GPU).
+ *
+ * The controller's load balancing (Section 4.4, last paragraph): a one-dimensional bin-packing
+ * problem solved with the Karmarkar-Karp largest differencing method.  equal_size != 0 is the
+ * data-parallel variant (every group gets the same number of samples, up to one when k does not
+ * divide n, and the spread of token totals is minimised under that constraint); equal_size == 0
+ * is the pipeline-parallel variant (sample counts free).
+ *
+ * Method: partial solutions are lists of k groups in decreasing order of token sum.  Start with
+ * one per sample (equal_size: one per run of k consecutive samples in decreasing length, one
+ * sample per group); repeatedly merge the two partial solutions of largest spread (largest minus
+ * smallest sum), joining the j-th largest group of the first with the j-th smallest of the
+ * second, until one is left.  Ties: samples by (length descending, index ascending); equal
+ * spreads in order of creation; equal sums keep their order.  Group g of the result has the
+ * g-th largest token total.
+ *
+ * length_host [n] >= 0 (host) in; part_host [n] (host) out, values in [0, k);
+ * group_tokens_host [k] (host, nullable) out.  AF_ERR_INVALID_ARG for null pointers, n < 0,
+ * k < 1 or a negative length.
+ * ------------------------------------------------------------------------------------------- */
+af_status af_balance_partitions(const int32_t* length_host, int32_t n, int32_t k, int32_t equal_size,
+                                int32_t* part_host, int64_t* group_tokens_host);
 
 /* ---------------------------------------------------------------------------------------------
  * af_token_logprob_static -- af_token_logprob for callers that are not allowed to allocate.

@@ -48,7 +48,7 @@ def controller_get_ref(ready: np.ndarray, consumed: np.ndarray, length, column_m
 
     ready[i]    : bit c set when column c of sample i has been written
     consumed[i] : bit t set when sample i has been handed to task t (updated in place)
-    length[i]   : tokens of sample i (only read when token_budget > 0)
+    length[i]   : tokens of sample i (None: no lengths known; then token_budget must be <= 0)
     Returns (indices handed out, their token total, number of eligible samples seen).
     """
     n = ready.shape[0]
@@ -62,7 +62,7 @@ def controller_get_ref(ready: np.ndarray, consumed: np.ndarray, length, column_m
         eligible += 1
         if not open_:
             continue
-        L = int(length[i]) if token_budget > 0 else 0
+        L = int(length[i]) if length is not None else 0
         fits = len(chosen) < max_samples and (token_budget <= 0 or tokens + L <= token_budget or not chosen)
         if fits:
             chosen.append(i)

@@ -21,11 +21,12 @@ AF_OK = 0
 STATUS_NAMES = {0: "AF_OK", -1: "AF_ERR_INVALID_ARG", -2: "AF_ERR_SHAPE", -3: "AF_ERR_ALIGNMENT",
                 -4: "AF_ERR_CAPACITY", -5: "AF_ERR_INDEX", -6: "AF_ERR_WORKSPACE", -7: "AF_ERR_CUDA",
                 -8: "AF_ERR_UNSUPPORTED_DEVICE", -9: "AF_ERR_DEVICE_FLAGGED"}
-DEVERR_TARGET_RANGE, DEVERR_WATCHDOG, DEVERR_CU_SEQLENS = 1, 2, 4
+DEVERR_TARGET_RANGE, DEVERR_WATCHDOG, DEVERR_CU_SEQLENS, DEVERR_SAMPLE_INDEX = 1, 2, 4, 8
 
 EXPORTS = ["af_create", "af_destroy", "af_status_string", "af_reserve", "af_workspace_bytes",
            "af_set_tuning", "af_check_device_errors", "af_pack_microbatch", "af_token_logprob",
-           "af_grpo_advantage", "af_policy_loss", "af_policy_loss_backward", "af_token_logprob_static"]
+           "af_grpo_advantage", "af_policy_loss", "af_policy_loss_backward", "af_token_logprob_static",
+           "af_controller_put", "af_controller_get", "af_controller_clear", "af_balance_partitions"]
 
 
 class AfError(RuntimeError):
@@ -58,6 +59,14 @@ class LossOut(C.Structure):
                 ("n_tokens", C.c_int64)]
 
 
+class ControllerView(C.Structure):
+    _fields_ = [("n_samples", C.c_int64), ("ready", C.c_void_p), ("consumed", C.c_void_p), ("length", C.c_void_p)]
+
+
+class GetResult(C.Structure):
+    _fields_ = [("count", C.c_int32), ("eligible", C.c_int32), ("tokens", C.c_int64)]
+
+
 _lib = None
 
 
@@ -88,6 +97,11 @@ def load_library() -> C.CDLL:
                                    vp, vp]
     lib.af_policy_loss_backward.argtypes = [vp, vp, vp, vp, vp, vp, i64, i32, i32, vp, vp, i32, vp]
     lib.af_token_logprob_static.argtypes = [vp, vp, vp, i64, i32, i32, vp, vp, vp, vp, vp]
+    u32 = C.c_uint32
+    lib.af_controller_put.argtypes = [vp, C.POINTER(ControllerView), vp, i64, u32, vp]
+    lib.af_controller_get.argtypes = [vp, C.POINTER(ControllerView), u32, u32, i32, i64, vp, vp, vp]
+    lib.af_controller_clear.argtypes = [vp, C.POINTER(ControllerView), u32, u32, vp]
+    lib.af_balance_partitions.argtypes = [vp, i32, i32, i32, vp, vp]
     for name in EXPORTS:
         if name not in ("af_status_string", "af_workspace_bytes"):
             getattr(lib, name).restype = C.c_int
@@ -208,6 +222,58 @@ class Context:
                                                 _ptr(lse), _ptr(dlogp), T, d, V, _ptr(d_hidden),
                                                 _ptr(d_W), int(accumulate_dW), _stream(stream)),
                "af_policy_loss_backward")
+
+
+    # -- controller: status table of the streaming store ----------------------------------------
+    @staticmethod
+    def _table(table: dict) -> ControllerView:
+        """``table``: device tensors ready / consumed (int32 or uint32 bit masks, [N]) and
+        optionally length (int32 [N])."""
+        ready = table["ready"]
+        return ControllerView(n_samples=ready.shape[0], ready=_ptr(ready), consumed=_ptr(table["consumed"]),
+                              length=_ptr(table.get("length")))
+
+    def controller_put(self, table: dict, idx: torch.Tensor, column_bits: int, n=None, stream=None):
+        tv = self._table(table)
+        n = idx.shape[0] if n is None else n
+        _check(self.lib.af_controller_put(self.handle, C.byref(tv), _ptr(idx), n, column_bits, _stream(stream)),
+               "af_controller_put")
+
+    def controller_get(self, table: dict, column_mask: int, task_bit: int, max_samples: int, token_budget: int,
+                       out_idx: torch.Tensor, out: torch.Tensor, stream=None):
+        """``out_idx``: device int32 [>= max_samples]; ``out``: device uint8 buffer of
+        ``ctypes.sizeof(GetResult)`` bytes (see read_get_result)."""
+        tv = self._table(table)
+        _check(self.lib.af_controller_get(self.handle, C.byref(tv), column_mask, task_bit, max_samples,
+                                          token_budget, _ptr(out_idx), _ptr(out), _stream(stream)),
+               "af_controller_get")
+
+    def controller_clear(self, table: dict, column_bits: int, task_bits: int, stream=None):
+        tv = self._table(table)
+        _check(self.lib.af_controller_clear(self.handle, C.byref(tv), column_bits, task_bits, _stream(stream)),
+               "af_controller_clear")
+
+
+def balance_partitions(length, k: int, equal_size: bool):
+    """``af_balance_partitions`` (host): returns (part [n] int32, group token totals [k] int64)."""
+    lib = load_library()
+    L = np.ascontiguousarray(length, dtype=np.int32)
+    part = np.empty(L.shape[0], dtype=np.int32)
+    sums = np.zeros(k, dtype=np.int64)
+    _check(lib.af_balance_partitions(C.c_void_p(L.ctypes.data) if L.size else None, L.shape[0], k, int(equal_size),
+                                     C.c_void_p(part.ctypes.data) if L.size else None,
+                                     C.c_void_p(sums.ctypes.data)), "af_balance_partitions")
+    return part, sums
+
+
+def new_get_result(device) -> torch.Tensor:
+    return torch.zeros(C.sizeof(GetResult), dtype=torch.uint8, device=device)
+
+
+def read_get_result(buf: torch.Tensor) -> dict:
+    """Copy the device ``af_get_result`` to the host (synchronises) and return it as a dict."""
+    o = GetResult.from_buffer_copy(buf.cpu().numpy().tobytes())
+    return {"count": o.count, "eligible": o.eligible, "tokens": o.tokens}
 
 
 def new_loss_out(device) -> torch.Tensor:

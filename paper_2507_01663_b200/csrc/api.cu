@@ -83,6 +83,7 @@ af_status af_create(af_ctx** out, int device) {
   }
   af_status st = ws_grow(c->loss_ws, loss_workspace_bytes(c->sm_count));
   if (st == AF_OK && cudaMemset(c->loss_ws.p, 0, c->loss_ws.cap) != cudaSuccess) st = AF_ERR_CUDA;
+  if (st == AF_OK) st = ws_grow(c->ctrl_ws, controller_workspace_bytes(c->sm_count));
   if (st != AF_OK) { af_destroy(c); return st; }
   *out = c;
   return AF_OK;
@@ -92,7 +93,7 @@ af_status af_destroy(af_ctx* c) {
   if (!c) return AF_ERR_INVALID_ARG;
   DeviceGuard guard(c->device);
   cudaDeviceSynchronize();
-  Buf* bufs[] = {&c->partial, &c->loss_ws, &c->pack_meta, &c->dz};
+  Buf* bufs[] = {&c->partial, &c->loss_ws, &c->pack_meta, &c->dz, &c->ctrl_ws};
   for (Buf* b : bufs) if (b->p) cudaFree(b->p);
   for (int i = 0; i < kPackRing; ++i) {
     if (c->pack_host[i]) cudaFreeHost(c->pack_host[i]);
@@ -105,7 +106,7 @@ af_status af_destroy(af_ctx* c) {
 
 int64_t af_workspace_bytes(const af_ctx* c) {
   if (!c) return 0;
-  return (int64_t)(c->partial.cap + c->loss_ws.cap + c->pack_meta.cap + c->dz.cap);
+  return (int64_t)(c->partial.cap + c->loss_ws.cap + c->pack_meta.cap + c->dz.cap + c->ctrl_ws.cap);
 }
 
 af_status af_set_tuning(af_ctx* c, int32_t v_splits, int32_t bwd_token_block, int32_t gemm_pair) {
@@ -290,6 +291,40 @@ af_status af_policy_loss_backward(af_ctx* c, const void* hidden, const void* W, 
   DeviceGuard guard(c->device);
   return launch_backward(c, hidden, W, target, lse, dlogp, T, d, V, d_hidden, d_W,
                          accumulate_dW ? 1 : 0, static_cast<cudaStream_t>(stream));
+}
+
+static bool table_ok(const af_controller_view* t) {
+  return t && t->n_samples >= 0 && (t->n_samples == 0 || (t->ready && t->consumed));
+}
+
+af_status af_controller_put(af_ctx* c, const af_controller_view* table, const int32_t* idx, int64_t n,
+                            uint32_t column_bits, void* stream) {
+  if (!c || !table_ok(table) || n < 0 || (n > 0 && !idx)) return AF_ERR_INVALID_ARG;
+  if (table->n_samples >= ((int64_t)1 << 31)) return AF_ERR_SHAPE;
+  DeviceGuard guard(c->device);
+  return launch_controller_put(*table, idx, n, column_bits, c->d_err, c->sm_count,
+                               static_cast<cudaStream_t>(stream)) == cudaSuccess ? AF_OK : AF_ERR_CUDA;
+}
+
+af_status af_controller_get(af_ctx* c, const af_controller_view* table, uint32_t column_mask, uint32_t task_bit,
+                            int32_t max_samples, int64_t token_budget, int32_t* out_idx, af_get_result* out,
+                            void* stream) {
+  if (!c || !table_ok(table) || !out || max_samples < 0 || (max_samples > 0 && !out_idx)) return AF_ERR_INVALID_ARG;
+  if (task_bit == 0 || (task_bit & (task_bit - 1)) != 0) return AF_ERR_INVALID_ARG;
+  if (token_budget > 0 && !table->length && table->n_samples > 0) return AF_ERR_INVALID_ARG;
+  if (table->n_samples >= ((int64_t)1 << 31)) return AF_ERR_SHAPE;
+  DeviceGuard guard(c->device);
+  return launch_controller_get(*table, column_mask, task_bit, max_samples, token_budget, out_idx, out,
+                               c->ctrl_ws.p, c->sm_count, static_cast<cudaStream_t>(stream)) == cudaSuccess
+             ? AF_OK : AF_ERR_CUDA;
+}
+
+af_status af_controller_clear(af_ctx* c, const af_controller_view* table, uint32_t column_bits, uint32_t task_bits,
+                              void* stream) {
+  if (!c || !table_ok(table)) return AF_ERR_INVALID_ARG;
+  DeviceGuard guard(c->device);
+  return launch_controller_clear(*table, column_bits, task_bits, c->sm_count,
+                                 static_cast<cudaStream_t>(stream)) == cudaSuccess ? AF_OK : AF_ERR_CUDA;
 }
 
 }  // extern "C"

@@ -41,6 +41,7 @@ struct af_ctx {
   af::Buf loss_ws;    // per-block partial sums + ticket of the loss reduction
   af::Buf pack_meta;  // per-call sequence table of af_pack_microbatch
   af::Buf dz;         // dZ [Tc, V] bf16 (backward, one token block)
+  af::Buf ctrl_ws;    // per-block aggregates of af_controller_get
 
   // pinned staging ring for pack metadata
   void* pack_host[af::kPackRing] = {};
@@ -77,6 +78,15 @@ cudaError_t launch_policy_loss(const float* logp, const float* old_logp, const f
                                int32_t B, int64_t T, const af_loss_params& p, af_loss_out* out,
                                float* dlogp, void* ws, unsigned int* d_err, int sm_count,
                                cudaStream_t s);
+
+size_t controller_workspace_bytes(int sm_count);
+cudaError_t launch_controller_put(const af_controller_view& v, const int32_t* idx, int64_t n, uint32_t bits,
+                                  unsigned int* d_err, int sm_count, cudaStream_t s);
+cudaError_t launch_controller_clear(const af_controller_view& v, uint32_t column_bits, uint32_t task_bits,
+                                    int sm_count, cudaStream_t s);
+cudaError_t launch_controller_get(const af_controller_view& v, uint32_t mask, uint32_t task_bit, int32_t max_samples,
+                                  int64_t token_budget, int32_t* out_idx, af_get_result* out, void* ws,
+                                  int sm_count, cudaStream_t s);
 
 int logprob_pick_splits(int64_t T, int32_t d, int32_t V, int sm_count, bool pair, int requested);
 af_status launch_token_logprob(af_ctx* ctx, const void* hidden, const void* W,
