@@ -257,7 +257,48 @@ class ScoringJob:
         gbs = 8.0 * n / ms / 1e6
         out["grpo_advantage"] = {"responses": n, "group_size": G, "bytes_per_response": 8, "ms": ms, "gbs": gbs,
                                  "frac": gbs / peak_gbs}
+        del r, a
+        # controller: one read request against a 2^26-sample status table (12 B read per sample:
+        # ready, consumed, length) that hands out the first 4096 eligible samples
+        tab = {"ready": torch.ones(n, dtype=torch.int32, device=dev),
+               "consumed": torch.zeros(n, dtype=torch.int32, device=dev),
+               "length": torch.full((n,), 300, dtype=torch.int32, device=dev)}
+        tab["ready"][: n - 100000] = 0          # the eligible samples sit at the far end of the table
+        out_idx, res = torch.empty(4096, dtype=torch.int32, device=dev), B.new_get_result(dev)
+
+        def get_once():
+            c.controller_get(tab, 1, 1, 4096, 1 << 20, out_idx, res)
+            c.controller_clear(tab, 0, 1)       # hand the same samples out again next time
+
+        ms_pair = avg_ms(get_once)
+        ms_clear = avg_ms(lambda: c.controller_clear(tab, 0, 1))
+        ms = ms_pair - ms_clear
+        gbs = 12.0 * n / ms / 1e6
+        out["controller_get"] = {"samples": n, "bytes_per_sample": 12, "ms": ms, "gbs": gbs, "frac": gbs / peak_gbs,
+                                 "returned": B.read_get_result(res)["count"],
+                                 "where": "2 launches (count, select); time of a get + clear pair minus a clear"}
         return out
+
+    def balance_report(self) -> dict:
+        """Token balancing of the workload's responses over 8 data-parallel groups (host call):
+        spread of the groups' token totals against dealing the responses out in arrival order."""
+        w, B = self.w, self.B
+        L = w.lengths.astype(np.int32)
+        k = 8
+        t0 = time.perf_counter()
+        part, sums = B.balance_partitions(L, k, True)
+        ms_dp = 1e3 * (time.perf_counter() - t0)
+        t0 = time.perf_counter()
+        _, sums_pp = B.balance_partitions(L, k, False)
+        ms_pp = 1e3 * (time.perf_counter() - t0)
+        order = wl.arrival_order(w)
+        rr = np.zeros(k, dtype=np.int64)
+        np.add.at(rr, np.arange(w.N) % k, w.lengths[order])
+        return {"groups": k, "samples": int(w.N), "host_ms_equal_counts": ms_dp, "host_ms_free_counts": ms_pp,
+                "token_spread_arrival_order": int(rr.max() - rr.min()),
+                "token_spread_equal_counts": int(sums.max() - sums.min()),
+                "token_spread_free_counts": int(sums_pp.max() - sums_pp.min()),
+                "mean_tokens_per_group": float(sums.mean())}
 
     # -- end-to-end: store columns start in pinned host memory ------------------------------
     def make_host_store(self):
@@ -396,6 +437,8 @@ def run_ours(args):
                                                        "where": "inside the timed steps (all micro-batches of a step), "
                                                                 "each right after a GEMM (part at its power cap)"}}
     line["hbm_kernels"].update(hbm_alone)
+    if rank == 0:
+        line["balance"] = job.balance_report()
     if bwd_ms is not None:
         bflops = 6.0 * job.T * w.d * w.V
         line["backward"] = {"ms": bwd_ms, "tflops": bflops / (bwd_ms * 1e-3) / 1e12, "flop_model": "6*T*d*V",

@@ -5,14 +5,19 @@
 //   1. recompute  Z = H_blk W^T  (both operands K-major) and turn it, in the epilogue, into
 //        dZ = g_t (1{v = y_t} - exp(z - lse_t))   (bf16), written once as dZ [Tc, V];
 //   2. dH_blk = dZ * W        A = dZ [Tc,V] K-major,  B = W [V,d] read MN-major   -> bf16 [Tc, d];
-//   3. dW    += dZ^T * H_blk  A = dZ [Tc,V] and B = H_blk [Tc,d], both read MN-major -> fp32 [V, d].
+//   3. dW^T  += H_blk^T * dZ  A = H_blk [Tc,d] and B = dZ [Tc,V], both read MN-major; the tile is
+//                             computed as [d, V] and stored transposed into fp32 dW [V, d].
 // No operand is ever transposed in memory.  The scratch is one block of dZ; [T,V] is never
 // materialised and the scratch does not grow with T.
 //
 // Epilogues hold one output row per lane (the TMEM load shape); storing that directly would write
-// 16 bytes to each of 32 different rows per instruction.  Each warp therefore passes its 32x32
-// chunk through a private, XOR-swizzled shared-memory buffer and stores whole 64/128-byte row
-// segments, four to eight rows per instruction.
+// 16 bytes to each of 32 different rows per instruction.  The dZ and dH epilogues therefore pass
+// their 32x32 chunk through a private, XOR-swizzled shared-memory buffer and store whole 64-byte
+// row segments, eight rows per instruction.  The dW product is laid out the other way round: its
+// accumulator rows run along d, the contiguous dimension of dW, so 32 lanes holding the same
+// vocabulary row write 128 consecutive bytes without any staging.  That orientation also gives the
+// product the forward's memory behaviour: the H_blk panels (68 MB at the 7B head) stay in L2 and
+// dZ streams through exactly once.
 #include "gemm_launch.cuh"
 
 namespace af {
@@ -122,44 +127,44 @@ struct StoreBf16Epi {
   static __device__ __forceinline__ void unit_end(State&, const Params&, int, int) {}
 };
 
-// ---- epilogue 3: accumulator tile -> fp32 matrix (store or add) ---------------------------------
-// Staging: row r = 128 bytes = eight 16-byte slots, slot q at position q ^ (r & 7).
-struct StoreF32Epi {
+// ---- epilogue 3: accumulator tile [m, n] -> fp32 matrix C[n, m] (store or add) ------------------
+// Lane L holds row m = row0 + L; for a fixed column n the 32 lanes address 32 consecutive floats of
+// C's row n: one coalesced 128-byte access per column.
+struct StoreF32TransposedEpi {
   struct Params {
-    float* C;
-    int64_t ldc;
+    float* C;          // [N, M] row-major
+    int64_t ldc;       // elements between consecutive n
     int M, N;
     int accumulate;
   };
   struct State {};
-  static constexpr bool kStaged = true;
+  static constexpr bool kStaged = false;
   static __device__ __forceinline__ void unit_begin(State&, const Params&, int, int, int) {}
   static __device__ __forceinline__ void chunk(State&, const Params& p, int row, int col0,
-                                               const uint32_t (&v)[32], uint8_t* stage) {
-    if (col0 >= p.N) return;
-    const int lane = threadIdx.x & 31;
-    const int row0 = row - lane;
-    uint4* st = reinterpret_cast<uint4*>(stage);
+                                               const uint32_t (&v)[32], uint8_t*) {
+    if (col0 >= p.N || row >= p.M) return;
+    float* dst = p.C + (size_t)col0 * p.ldc + row;
+    if (col0 + 32 <= p.N) {
+      if (p.accumulate) {
+        float o[32];
 #pragma unroll
-    for (int q = 0; q < 8; ++q)
-      st[lane * 8 + (q ^ (lane & 7))] = make_uint4(v[q * 4 + 0], v[q * 4 + 1], v[q * 4 + 2], v[q * 4 + 3]);
-    __syncwarp();
+        for (int j = 0; j < 32; ++j) o[j] = dst[(size_t)j * p.ldc];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const int r = i * 4 + (lane >> 3), c = lane & 7;
-      const uint4 u = st[r * 8 + (c ^ (r & 7))];
-      const int grow = row0 + r, gcol = col0 + c * 4;
-      if (grow < p.M && gcol + 4 <= p.N) {
-        float* dst = p.C + (size_t)grow * p.ldc + gcol;
-        float4 w = make_float4(__uint_as_float(u.x), __uint_as_float(u.y), __uint_as_float(u.z), __uint_as_float(u.w));
-        if (p.accumulate) {
-          const float4 o = *reinterpret_cast<const float4*>(dst);
-          w.x += o.x; w.y += o.y; w.z += o.z; w.w += o.w;
+        for (int j = 0; j < 32; ++j) dst[(size_t)j * p.ldc] = o[j] + __uint_as_float(v[j]);
+      } else {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) dst[(size_t)j * p.ldc] = __uint_as_float(v[j]);
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        if (col0 + j < p.N) {
+          float w = __uint_as_float(v[j]);
+          if (p.accumulate) w += dst[(size_t)j * p.ldc];
+          dst[(size_t)j * p.ldc] = w;
         }
-        *reinterpret_cast<float4*>(dst) = w;
       }
     }
-    __syncwarp();
   }
   static __device__ __forceinline__ void unit_end(State&, const Params&, int, int) {}
 };
@@ -201,9 +206,13 @@ af_status launch_backward(af_ctx* ctx, const void* hidden, const void* W, const 
     StoreBf16Epi::Params p2{static_cast<__nv_bfloat16*>(d_hidden) + t0 * d, d, (int)tc, d};
     st = run_gemm<StoreBf16Epi, false, true>(env, dZop, Wop, 0, p2, s);
     if (st != AF_OK) return st;
-    // 3. dW += dZ^T H_blk:  A = dZ read MN-major (m = v contiguous, K = t rows), B = H_blk read MN-major
-    StoreF32Epi::Params p3{d_W, d, V, d, (!first || accumulate_dW) ? 1 : 0};
-    st = run_gemm<StoreF32Epi, true, true>(env, dZop, Hblk, 0, p3, s);
+    // 3. dW^T += H_blk^T dZ:  A = H_blk read MN-major (m = d contiguous, K = t rows), B = dZ read
+    //    MN-major (n = v contiguous); tile [d, v] stored transposed into dW [V, d].  Vocabulary ranges
+    //    are chosen as in the forward: the H_blk panels stay in L2, dZ streams past once.
+    StoreF32TransposedEpi::Params p3{d_W, d, d, V, (!first || accumulate_dW) ? 1 : 0};
+    st = run_gemm<StoreF32TransposedEpi, true, true>(env, Hblk, dZop,
+                                                     logprob_pick_splits((int64_t)d, (int32_t)tc, V, ctx->sm_count, env.pair, 0),
+                                                     p3, s);
     if (st != AF_OK) return st;
   }
   return AF_OK;
