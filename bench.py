@@ -9,7 +9,8 @@ fused LM-head log-prob / entropy -> clipped policy loss + k3 KL (with dL/dlogp).
 
 Prints ONE JSON line (rank 0).  ``value`` is scored tokens/s over all ranks with the inputs
 resident in HBM; ``e2e`` is the same metric with the store columns starting in pinned host
-memory (host->device copies and the device->host read of the loss inside the timed region).
+memory: every step's host->device copies (on a second stream, into the device copy the previous
+step is not reading) and the device->host read of the loss are inside the timed region.
 ``--impl reference`` times the fp64 CPU oracle on a bounded sample of the same workload.
 """
 from __future__ import annotations
@@ -131,15 +132,25 @@ def reduce_over_ranks(ms_local: float, tokens_local: int, world: int):
     return float(t.item()), int(n.item())
 
 
+def allreduce_sum_(t: torch.Tensor, world: int) -> torch.Tensor:
+    """Actor update under data parallelism: every rank scores its own prompts with
+    loss_scale = B_rank / B_global, so the weight gradients of the ranks ADD UP to the gradient of
+    the global batch; the one exchange of the path is this sum (NCCL on GPUs, gloo in CPU tests)."""
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return t
+
+
 # ------------------------------------------------------------------------------------------
 # the CUDA arm
 # ------------------------------------------------------------------------------------------
 class ScoringJob:
     """Device buffers of one rank and the step function that runs the path through the C ABI."""
 
-    def __init__(self, w: wl.Workload, device: torch.device, gemm_pair: bool = False):
+    def __init__(self, w: wl.Workload, device: torch.device, gemm_pair: bool = False, world: int = 1):
         from paper_2507_01663_b200 import binding as B
-        self.B, self.w, self.dev = B, w, device
+        self.B, self.w, self.dev, self.world = B, w, device, world
         self.ctx = B.Context(device.index or 0)
         self.ctx.set_tuning(0, 0, gemm_pair)
         T = w.total_tokens
@@ -179,10 +190,10 @@ class ScoringJob:
         per_mb = KERNELS_PER_STEP - 1 + (3 * -(-cap_T // BWD_TOKEN_BLOCK) if w.backward else 0)
         self.launches_per_step = 1 + per_mb * len(self.mbs)
 
-    def step(self, time_gemm: bool = False):
+    def step(self, time_gemm: bool = False, store_cols=None, reward=None):
         w, c = self.w, self.ctx
-        c.grpo_advantage(self.reward, None, w.n_prompts, self.adv)
-        store = {"tok_offset_host": self.off, "d": w.d, "adv": self.adv, **self.store}
+        c.grpo_advantage(self.reward if reward is None else reward, None, w.n_prompts, self.adv)
+        store = {"tok_offset_host": self.off, "d": w.d, "adv": self.adv, **(self.store if store_cols is None else store_cols)}
         total = 0
         for mb, loss_out in zip(self.mbs, self.loss_outs):
             ev = [torch.cuda.Event(enable_timing=True) for _ in range(6)] if time_gemm else None
@@ -197,7 +208,7 @@ class ScoringJob:
                 ev[3].record()
             c.policy_loss(self.logp, self.packed["old_logp"], self.packed["ref_logp"], self.packed["adv_seq"],
                           self.packed["cu_seqlens"], loss_out, self.dlogp, self.ent,
-                          w.clip_eps, w.clip_eps, w.kl_coef, 0, 1.0, B=len(mb), T=T)
+                          w.clip_eps, w.clip_eps, w.kl_coef, 0, 1.0 / self.world, B=len(mb), T=T)
             if w.backward:
                 if ev:
                     ev[4].record()
@@ -206,6 +217,7 @@ class ScoringJob:
                 if ev:
                     ev[5].record()
                     self.bwd_events.append((ev[4], ev[5]))
+                allreduce_sum_(self.d_W, self.world)    # equal batches per rank: loss_scale = 1 / world
             if ev:
                 self.pack_events.append((ev[0], ev[1]))
                 self.gemm_events.append((ev[2], ev[3]))
@@ -302,20 +314,38 @@ class ScoringJob:
 
     # -- end-to-end: store columns start in pinned host memory ------------------------------
     def make_host_store(self):
+        """Pinned host copies of the store columns and rewards, a second device copy of the store
+        and a copy stream: the host->device copies of step k+1 run while step k computes."""
         self.host = {k: torch.empty(v.shape, dtype=v.dtype, pin_memory=True) for k, v in self.store.items()}
         self.host["reward"] = torch.empty(self.reward.shape, dtype=self.reward.dtype, pin_memory=True)
         for k, v in self.store.items():
             self.host[k].copy_(v)
         self.host["reward"].copy_(self.reward)
+        self.dev_store = [self.store, {k: torch.empty_like(v) for k, v in self.store.items()}]
+        self.dev_reward = [self.reward, torch.empty_like(self.reward)]
+        self.copy_stream = torch.cuda.Stream()
+        self.buf_ready = [torch.cuda.Event() for _ in range(2)]
+        self.buf_free = [torch.cuda.Event() for _ in range(2)]
         torch.cuda.synchronize()
+        for e in self.buf_free:
+            e.record()
+        self.e2e_steps = 0
         self.h2d_bytes = sum(t.numel() * t.element_size() for t in self.host.values())
         self.host_loss = [torch.empty(lo.shape, dtype=torch.uint8, pin_memory=True) for lo in self.loss_outs]
 
     def step_e2e(self):
-        for k, v in self.store.items():
-            v.copy_(self.host[k], non_blocking=True)
-        self.reward.copy_(self.host["reward"], non_blocking=True)
-        T = self.step()
+        b = self.e2e_steps & 1
+        self.e2e_steps += 1
+        main = torch.cuda.current_stream()
+        with torch.cuda.stream(self.copy_stream):
+            self.copy_stream.wait_event(self.buf_free[b])       # the step that last read this copy is done
+            for k, v in self.dev_store[b].items():
+                v.copy_(self.host[k], non_blocking=True)
+            self.dev_reward[b].copy_(self.host["reward"], non_blocking=True)
+            self.buf_ready[b].record(self.copy_stream)
+        main.wait_event(self.buf_ready[b])
+        T = self.step(store_cols=self.dev_store[b], reward=self.dev_reward[b])
+        self.buf_free[b].record(main)
         for h, lo in zip(self.host_loss, self.loss_outs):
             h.copy_(lo, non_blocking=True)
         return T
@@ -372,7 +402,7 @@ def run_ours(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
     w = rank_workload(args.workload, rank)
-    job = ScoringJob(w, dev, args.gemm_pair)
+    job = ScoringJob(w, dev, args.gemm_pair, world)
     peaks = measured_peaks()
     hbm_alone = job.hbm_kernels_at_scale(peaks["hbm_gbs"]) if rank == 0 and world == 1 else {}
 

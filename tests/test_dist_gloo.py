@@ -1,6 +1,7 @@
 """World-size-2 checks of the data-parallel host logic on CPU (gloo): prompts are split into
-whole groups, rank results concatenate to the single-rank result, and bench.py's reduction takes
-the max step time and the token sum over ranks."""
+whole groups, rank results concatenate to the single-rank result, bench.py's reduction takes the
+max step time and the token sum over ranks, and the weight gradients of the ranks' batches, each
+scored with loss_scale = B_rank / B_global, sum to the gradient of the global batch."""
 import os
 import socket
 
@@ -53,3 +54,64 @@ def test_two_rank_sharding(tmp_path):
     port = _free_port()
     mp.start_processes(_worker, args=(2, port, str(tmp_path)), nprocs=2, join=True, start_method="spawn")
     assert open(tmp_path / "ok").read() == "1"
+
+
+def _grad_worker(rank, world, port, out_dir):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    import bench
+    w = wl.make_workload("cfg1")
+    H, W, y = wl.bf16_bits(wl.gen_hidden(w)), wl.bf16_bits(wl.gen_weight(w)), wl.gen_target(w).numpy()
+    r = wl.gen_reward(w).numpy()
+    adv = O.grpo_advantage_ref(r, w.group_id, w.n_prompts)
+    off = w.tok_offset
+
+    def actor_update(samples, scale):
+        """Oracle forward + loss + backward over the given samples (packed in that order)."""
+        packed = O.pack_microbatch_ref(off, samples, {"hidden": H, "target": y}, adv)
+        lp, _, lse = O.token_logprob_ref(packed["hidden"], W, packed["target"])
+        T = lp.shape[0]
+        old = lp + 0.1 * np.sin(np.arange(T))            # any fixed perturbation, the same on every path
+        ref = lp - 0.05 * np.cos(np.arange(T))
+        res = O.policy_loss_ref(lp, old, ref, packed["adv_seq"], packed["cu_seqlens"], loss_scale=scale)
+        _, dW = O.policy_loss_backward_ref(packed["hidden"], W, packed["target"], lse, res["dlogp"])
+        return res["loss"], dW
+
+    prompts = wl.shard_prompts(w.n_prompts, world, rank)
+    mine = np.concatenate([np.arange(p * w.group_size, (p + 1) * w.group_size) for p in prompts])
+    loss_local, dW_local = actor_update(mine, len(mine) / w.N)
+    dW_sum = bench.allreduce_sum_(torch.from_numpy(dW_local.copy()), world).numpy()
+    loss_sum = bench.allreduce_sum_(torch.tensor([loss_local], dtype=torch.float64), world).item()
+    if rank == 0:
+        # old / ref perturbations depend on the position inside the rank's batch: replay both
+        # ranks' batches on one process and add them, which is what the global batch means here
+        total_loss, total_dW = 0.0, 0.0
+        for rk in range(world):
+            pr = wl.shard_prompts(w.n_prompts, world, rk)
+            idx = np.concatenate([np.arange(p * w.group_size, (p + 1) * w.group_size) for p in pr])
+            l, g = actor_update(idx, len(idx) / w.N)
+            total_loss, total_dW = total_loss + l, total_dW + g
+        ok = np.allclose(dW_sum, total_dW, rtol=0, atol=1e-12 * np.abs(total_dW).max()) and abs(loss_sum - total_loss) < 1e-14
+        # and the scaled per-rank losses add up to the global-batch loss when the inputs agree:
+        # with old = ref = logp every token's loss is -A, so L = -(1/B) sum_i A_i on any split
+        packed = O.pack_microbatch_ref(off, np.arange(w.N), {"hidden": H, "target": y}, adv)
+        lp, _, _ = O.token_logprob_ref(packed["hidden"], W, packed["target"])
+        full = O.policy_loss_ref(lp, lp, lp, packed["adv_seq"], packed["cu_seqlens"])["loss"]
+        parts = 0.0
+        for rk in range(world):
+            pr = wl.shard_prompts(w.n_prompts, world, rk)
+            idx = np.concatenate([np.arange(p * w.group_size, (p + 1) * w.group_size) for p in pr])
+            pk = O.pack_microbatch_ref(off, idx, {"hidden": H, "target": y}, adv)
+            lpr, _, _ = O.token_logprob_ref(pk["hidden"], W, pk["target"])
+            parts += O.policy_loss_ref(lpr, lpr, lpr, pk["adv_seq"], pk["cu_seqlens"], loss_scale=len(idx) / w.N)["loss"]
+        ok = ok and abs(parts - full) < 1e-12
+        with open(os.path.join(out_dir, "ok_grad"), "w") as f:
+            f.write("1" if ok else "0")
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_two_rank_gradient_sum(tmp_path):
+    port = _free_port()
+    mp.start_processes(_grad_worker, args=(2, port, str(tmp_path)), nprocs=2, join=True, start_method="spawn")
+    assert open(tmp_path / "ok_grad").read() == "1"
