@@ -34,7 +34,7 @@ from paper_2507_01663_b200 import workloads as wl  # noqa: E402
 
 METRIC = "scored tokens/sec (logprob+GRPO loss) at Qwen-7B head; % dense-BF16 peak"
 UNIT = "tokens/s"
-KERNELS_PER_STEP = 6  # advantage, pack columns, pack rows (bulk copy), fused LM-head GEMM, partial merge, loss
+KERNELS_PER_STEP = 7  # advantage, pack table fetch, pack columns, pack rows (bulk copy), fused LM-head GEMM, partial merge, loss
 # DRAM bytes per scored token of the fused LM-head kernel (dram__bytes_read + dram__bytes_write of
 # one ncu capture at T = 65536, d = 3584, V = 152064; traffic grows with the number of waves of
 # row tiles, i.e. in proportion to T).  Valid for the 7B head shape only; None whenever the kernel
@@ -148,11 +148,11 @@ def allreduce_sum_(t: torch.Tensor, world: int) -> torch.Tensor:
 class ScoringJob:
     """Device buffers of one rank and the step function that runs the path through the C ABI."""
 
-    def __init__(self, w: wl.Workload, device: torch.device, gemm_pair: bool = False, world: int = 1):
+    def __init__(self, w: wl.Workload, device: torch.device, gemm_variant: int = 0, world: int = 1):
         from paper_2507_01663_b200 import binding as B
         self.B, self.w, self.dev, self.world = B, w, device, world
         self.ctx = B.Context(device.index or 0)
-        self.ctx.set_tuning(0, 0, gemm_pair)
+        self.ctx.set_tuning(0, 0, gemm_variant)
         T = w.total_tokens
         self.T = T
         self.store = {
@@ -402,7 +402,7 @@ def run_ours(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
     w = rank_workload(args.workload, rank)
-    job = ScoringJob(w, dev, args.gemm_pair, world)
+    job = ScoringJob(w, dev, {"default": 0, "single": 1, "pair": 2}[args.gemm], world)
     peaks = measured_peaks()
     hbm_alone = job.hbm_kernels_at_scale(peaks["hbm_gbs"]) if rank == 0 and world == 1 else {}
 
@@ -445,7 +445,7 @@ def run_ours(args):
                                   else "one arrival-ordered packed micro-batch")
                                + (", forward + backward (dH, dW)" if w.backward else ""),
                    "l2": "inputs (hidden states >> 126 MB L2) exceed L2; no flush needed",
-                   "gemm": "CTA pairs (cta_group::2)" if args.gemm_pair else "one CTA per tile",
+                   "gemm": "one CTA per 128x256 tile" if args.gemm == "single" else "CTA pairs (cta_group::2), 256x256 tiles",
                    "loss": {"clip_eps": w.clip_eps, "kl_coef": w.kl_coef, "agg": "seq-mean-token-mean"}},
         "roofline": {"bound": "tensor", "kernel": "fused LM-head GEMM + online log-softmax (af_token_logprob)",
                      "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
@@ -530,8 +530,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2")
     ap.add_argument("--cpu-sample", type=int, default=1536, help="tokens in the CPU-oracle sample")
-    ap.add_argument("--gemm-pair", action="store_true",
-                    help="run the tensor-core GEMMs on CTA pairs (af_set_tuning gemm_pair = 1) instead of the default")
+    ap.add_argument("--gemm", default="default", choices=["default", "single", "pair"],
+                    help="main loop of the tensor-core GEMMs (af_set_tuning gemm_variant): CTA pairs (the default) "
+                         "or one CTA per tile")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3

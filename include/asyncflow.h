@@ -71,12 +71,12 @@ int64_t af_workspace_bytes(const af_ctx* ctx);
 
 /* Tuning knobs of the fused LM-head kernels (0 keeps the default): `v_splits` = number of
  * vocabulary ranges one token tile is split into across CTAs; `bwd_token_block` = tokens per
- * backward block, a multiple of 128 (scratch is proportional to it); `gemm_pair` = 1 runs every
- * tensor-core GEMM of the context on CTA pairs (two SMs share one 256 x 256 tile, each staging
- * half of the weight tile) instead of one CTA per 128 x 256 tile.  Pairs finish short launches
- * sooner; under the board's power limit the single-CTA default sustains the higher rate.
+ * backward block, a multiple of 128 (scratch is proportional to it); `gemm_variant` selects the
+ * main loop of every tensor-core GEMM of the context: 2 (and 0, the default) = CTA pairs -- two
+ * SMs share one 256 x 256 tile, each staging half of the weight tile, and the pairs pace one
+ * another so that a weight tile fetched once serves them all; 1 = one CTA per 128 x 256 tile.
  * Results agree within the stated tolerances either way. */
-af_status af_set_tuning(af_ctx* ctx, int32_t v_splits, int32_t bwd_token_block, int32_t gemm_pair);
+af_status af_set_tuning(af_ctx* ctx, int32_t v_splits, int32_t bwd_token_block, int32_t gemm_variant);
 
 /* Synchronise `stream`, read and clear the sticky device error word.  Returns AF_OK when it was
  * zero, else AF_ERR_DEVICE_FLAGGED with the bits in *flags (nullable). */

@@ -155,8 +155,9 @@ class Context:
     def workspace_bytes(self) -> int:
         return int(self.lib.af_workspace_bytes(self.handle))
 
-    def set_tuning(self, v_splits: int = 0, bwd_token_block: int = 0, gemm_pair: bool = False):
-        _check(self.lib.af_set_tuning(self.handle, v_splits, bwd_token_block, int(gemm_pair)), "af_set_tuning")
+    def set_tuning(self, v_splits: int = 0, bwd_token_block: int = 0, gemm_variant: int = 0):
+        """gemm_variant: 0 = default (CTA pairs), 1 = one CTA per tile, 2 = CTA pairs."""
+        _check(self.lib.af_set_tuning(self.handle, v_splits, bwd_token_block, gemm_variant), "af_set_tuning")
 
     def check_device_errors(self, stream=None) -> int:
         """Synchronise the stream; return the device error bits (0 = none) and clear them."""

@@ -69,6 +69,7 @@ af_status af_create(af_ctx** out, int device) {
   if (!c) return AF_ERR_WORKSPACE;
   c->device = device;
   c->sm_count = prop.multiProcessorCount;
+  c->gemm_pair = c->sm_count >= 2 ? 1 : 0;
   void* fn = nullptr;
   cudaDriverEntryPointQueryResult qres;
   if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
@@ -109,12 +110,12 @@ int64_t af_workspace_bytes(const af_ctx* c) {
   return (int64_t)(c->partial.cap + c->loss_ws.cap + c->pack_meta.cap + c->dz.cap + c->ctrl_ws.cap);
 }
 
-af_status af_set_tuning(af_ctx* c, int32_t v_splits, int32_t bwd_token_block, int32_t gemm_pair) {
-  if (!c || v_splits < 0 || bwd_token_block < 0 || (gemm_pair != 0 && gemm_pair != 1)) return AF_ERR_INVALID_ARG;
+af_status af_set_tuning(af_ctx* c, int32_t v_splits, int32_t bwd_token_block, int32_t gemm_variant) {
+  if (!c || v_splits < 0 || bwd_token_block < 0 || gemm_variant < 0 || gemm_variant > 2) return AF_ERR_INVALID_ARG;
   if (bwd_token_block % 128 != 0) return AF_ERR_SHAPE;
   c->v_splits = v_splits;
   c->bwd_token_block = bwd_token_block;
-  c->gemm_pair = gemm_pair;
+  c->gemm_pair = gemm_variant == 1 ? 0 : (c->sm_count >= 2 ? 1 : 0);
   return AF_OK;
 }
 
@@ -227,7 +228,7 @@ af_status af_pack_microbatch(af_ctx* c, const af_store_view* store, const int32_
   if (T > out->token_capacity) return AF_ERR_CAPACITY;
 
   char* db = static_cast<char*>(c->pack_meta.p);
-  if (cudaMemcpyAsync(db, hb, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return AF_ERR_CUDA;
+  if (launch_pack_meta_fetch(db, hb, bytes, s) != cudaSuccess) return AF_ERR_CUDA;
   if (!c->pack_evt_live[slot]) {
     if (cudaEventCreateWithFlags(&c->pack_evt[slot], cudaEventDisableTiming) != cudaSuccess) return AF_ERR_CUDA;
     c->pack_evt_live[slot] = true;

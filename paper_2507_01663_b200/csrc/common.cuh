@@ -12,6 +12,7 @@
 namespace af {
 
 constexpr int kPackRing = 8;  // pinned staging slots for af_pack_microbatch metadata
+constexpr int kTileClockWord = 16;  // word of the context's 256-byte device block used as the GEMM tile clock
 
 struct Buf {
   void* p = nullptr;
@@ -29,12 +30,12 @@ struct af_ctx {
   int device = 0;
   int sm_count = 0;
   af::EncodeTiledFn encode = nullptr;
-  unsigned int* d_err = nullptr;  // sticky device error word
+  unsigned int* d_err = nullptr;  // 256-byte device block: word 0 = sticky error word, word kTileClockWord = tile clock
 
   // tuning
   int v_splits = 0;         // 0 = automatic
   int bwd_token_block = 0;  // 0 = default
-  int gemm_pair = 0;        // 1 = CTA-pair GEMM variant
+  int gemm_pair = 1;        // 1 = CTA-pair GEMM variant (the default), 0 = one CTA per tile
 
   // workspace (device)
   af::Buf partial;    // [splits, T] float4 online-softmax partials
@@ -63,6 +64,8 @@ struct PackSeqTable {     // device views into ctx->pack_meta for one call
   const int32_t* chunk_cu;// [B+1] first bulk-copy chunk of sequence j (hidden column)
   int n_chunks;           // chunk_cu[B]
 };
+// Copy `bytes` (rounded up to 16) from pinned, device-mapped host memory to the device with a kernel.
+cudaError_t launch_pack_meta_fetch(void* dst_dev, const void* src_pinned, size_t bytes, cudaStream_t s);
 // Rows of the hidden column per bulk-copy chunk for hidden size d (0: rows too wide, no chunks).
 int pack_rows_per_chunk(int32_t d);
 cudaError_t launch_pack(const af_store_view& st, const af_packed& out, const PackSeqTable& tab,

@@ -120,7 +120,14 @@ __global__ void __launch_bounds__(kThreads) controller_count_kernel(
   int64_t q0, q1;
   segment_of(N, blockIdx.x, gridDim.x, q0, q1);
   int c = 0; long long t = 0;
-  for (int64_t q = q0 + threadIdx.x; q < q1; q += kThreads) {
+  int64_t q = q0 + threadIdx.x;
+  for (; q + kThreads < q1; q += 2 * kThreads) {          // two independent quads in flight per thread
+    const Quad v0 = load_quad(ready, consumed, length, q * kQuad, N, mask, task_bit, vec_ok != 0);
+    const Quad v1 = load_quad(ready, consumed, length, (q + kThreads) * kQuad, N, mask, task_bit, vec_ok != 0);
+#pragma unroll
+    for (int k = 0; k < kQuad; ++k) { c += v0.elig[k] + v1.elig[k]; t += v0.len[k] + v1.len[k]; }
+  }
+  for (; q < q1; q += kThreads) {
     const Quad v = load_quad(ready, consumed, length, q * kQuad, N, mask, task_bit, vec_ok != 0);
 #pragma unroll
     for (int k = 0; k < kQuad; ++k) { c += v.elig[k]; t += v.len[k]; }
@@ -159,8 +166,10 @@ __global__ void __launch_bounds__(kThreads) controller_select_kernel(
       block_scan((int)all_c, 0, d0, d1, all_tot, d2, s_c, s_t);
       if (threadIdx.x == 0) out->eligible = all_tot;
     }
-    // the prefix has ended before this segment: nothing here can be selected
+    // the prefix has ended before this segment, or the segment holds no eligible sample:
+    // nothing here can be selected (block-uniform)
     if (base_c >= max_samples || (token_budget > 0 && base_c > 0 && base_t > token_budget)) return;
+    if (agg[blockIdx.x].count == 0) return;
   }
   int64_t q0, q1;
   segment_of(N, blockIdx.x, gridDim.x, q0, q1);

@@ -20,6 +20,7 @@ struct GemmEnv {
   int sm_count;
   unsigned int* d_err;
   bool pair;             // CTA-pair variant (cta_group::2)
+  unsigned int* tile_clock;  // device word the pair variant paces itself with (zeroed per launch), or null
 };
 
 inline af_status encode_operand(const GemmEnv& env, CUtensorMap* map, const Operand& op, uint32_t box_rows) {
@@ -60,7 +61,9 @@ af_status run_gemm(const GemmEnv& env, const Operand& A, const Operand& B, int s
                              smem) != cudaSuccess) return AF_ERR_CUDA;
     const int pairs = env.sm_count / 2;
     const int grid = 2 * (int)(units < pairs ? units : pairs);
-    umma::gemm_pair_kernel<E, kAMN, kBMN><<<grid, umma::kThreads, smem, s>>>(ta, tb, g, ep, env.d_err);
+    unsigned int* clock = env.tile_clock;
+    if (clock && cudaMemsetAsync(clock, 0, sizeof(unsigned int), s) != cudaSuccess) return AF_ERR_CUDA;
+    umma::gemm_pair_kernel<E, kAMN, kBMN><<<grid, umma::kThreads, smem, s>>>(ta, tb, g, ep, env.d_err, clock);
   } else {
     constexpr int smem = E::kStaged ? umma::kSmemBytesStaged : umma::kSmemBytes;
     if (cudaFuncSetAttribute(umma::gemm_kernel<E, kAMN, kBMN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -72,7 +75,7 @@ af_status run_gemm(const GemmEnv& env, const Operand& A, const Operand& B, int s
 }
 
 inline GemmEnv gemm_env(const af_ctx* ctx) {
-  return GemmEnv{ctx->encode, ctx->sm_count, ctx->d_err, ctx->gemm_pair != 0};
+  return GemmEnv{ctx->encode, ctx->sm_count, ctx->d_err, ctx->gemm_pair != 0, ctx->d_err + kTileClockWord};
 }
 
 }  // namespace af

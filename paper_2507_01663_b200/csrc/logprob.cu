@@ -244,7 +244,7 @@ extern "C" af_status af_token_logprob_static(const void* hidden, const void* W, 
   unsigned int* err_word = device_flags ? device_flags : reinterpret_cast<unsigned int*>(st->scratch);
   float4* partial = reinterpret_cast<float4*>(st->scratch + kStaticHeaderBytes);
 
-  const GemmEnv env{g_static_encode, st->sm_count, err_word, false};
+  const GemmEnv env{g_static_encode, st->sm_count, err_word, false, nullptr};
   const Operand Hop{hidden, (uint64_t)T, (uint64_t)d, (uint64_t)d * 2};
   const Operand Wop{W, (uint64_t)V, (uint64_t)d, (uint64_t)d * 2};
   LogprobEpi::Params ep{target, partial, (int)T, V};

@@ -194,6 +194,31 @@ __global__ void __launch_bounds__(256) pack_cols_kernel(
 
 }  // namespace
 
+// Brings the per-call sequence table from pinned host memory to the device with a kernel (the
+// pinned buffer is mapped into the device's address space) instead of a host-to-device memcpy:
+// a memcpy would queue on the copy engine, behind whatever bulk transfers the application has in
+// flight (weights, the next batch of the store), and stall the whole micro-batch behind them.
+namespace {
+__global__ void __launch_bounds__(256) pack_meta_fetch_kernel(uint4* __restrict__ dst,
+                                                             const uint4* __restrict__ src_pinned, int n_words) {
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n_words; i += gridDim.x * blockDim.x) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(src_pinned + i));
+    dst[i] = v;
+  }
+}
+}  // namespace
+
+cudaError_t launch_pack_meta_fetch(void* dst_dev, const void* src_pinned, size_t bytes, cudaStream_t s) {
+  const int n_words = (int)((bytes + 15) / 16);
+  if (n_words == 0) return cudaSuccess;
+  int blocks = (n_words + 255) / 256;
+  if (blocks > 64) blocks = 64;
+  pack_meta_fetch_kernel<<<blocks, 256, 0, s>>>(static_cast<uint4*>(dst_dev), static_cast<const uint4*>(src_pinned), n_words);
+  return cudaGetLastError();
+}
+
 int pack_rows_per_chunk(int32_t d) {
   const int64_t row_bytes = (int64_t)d * 2;
   return row_bytes <= kChunkBytes ? (int)(kChunkBytes / row_bytes) : 0;

@@ -369,10 +369,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
 //   empty[s]  per CTA: the leader's MMA thread commits to both copies at once.
 //   tfull[a]  per CTA: accumulator a complete (committed to both copies at once).
 //   tempty[a] leader's copy only: one arrival per epilogue warp of either CTA (8 in all).
-// No load is multicast; every CTA fetches its own operand halves.
+// No load is multicast; every CTA fetches its own operand halves.  The leaders' producers pace
+// one another with a tile clock in global memory (a counter the host zeroes before the launch).
 // ==========================================================================================
 constexpr int kPairBM = 256;                                  // rows of A per pair tile
 constexpr int kPairStages = 6;
+constexpr unsigned int kClockWindow = 1;                      // tiles a pair may start ahead of the slowest pair
+constexpr unsigned long long kClockPatienceNs = 200000ull;    // longest wait on the tile clock before leaving it,
+constexpr unsigned long long kClockPatiencePerKBlockNs = 2000ull;  // plus this per K block of a tile (~5 tile times)
 constexpr int kPairBBytes = (kBN / 2) * kBK * 2;              // this CTA's half of the B tile
 constexpr int kPairStageBytes = kABytes + kPairBBytes;        // 32 KB
 constexpr int kPairSmemBytes = kPairStages * kPairStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
@@ -439,7 +443,7 @@ __device__ __forceinline__ void mma_commit_pair(uint32_t bar) {
 template <class E, bool kAMN = false, bool kBMN = false>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-                 const GemmShape g, const typename E::Params ep, unsigned int* d_err) {
+                 const GemmShape g, const typename E::Params ep, unsigned int* d_err, unsigned int* tile_clock) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles = (raw + 1023u) & ~1023u;
@@ -481,12 +485,38 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     if (lane == 0) {
       int stage = 0; uint32_t phase = 0; bool ok = true;
       const uint32_t leader_full0 = map_to_cta(full_bar(0), 0);
+      unsigned int my_tiles = 0;                                    // tiles this pair has started
+      bool clock_on = tile_clock != nullptr && rank == 0;
+      const unsigned long long patience = kClockPatienceNs + kClockPatiencePerKBlockNs * (unsigned long long)g.k_blocks;
+      // most tiles any pair starts in this launch
+      const unsigned int clock_most = (unsigned int)((total_units + n_pairs - 1) / n_pairs) *
+                                      (unsigned int)((g.n_tiles + g.splits - 1) / g.splits);
       for (int u = pair; u < total_units && ok; u += n_pairs) {
         const int m_tile = u / g.splits, s = u % g.splits;
         const int nb = split_begin(g, s), ne = split_begin(g, s + 1);
         const int m0 = m_tile * kPairBM + (int)rank * kBM;          // this CTA's 128 rows of A
         for (int nt = nb; nt < ne && ok; ++nt) {
           const int n0 = nt * kBN + (int)rank * (kBN / 2);          // this CTA's 128 rows of B
+          if (clock_on) {
+            // Tile clock: stay within kClockWindow tiles of the slowest pair, so that a B tile
+            // fetched by the first pair is still in L2 when the last one asks for it.  The clock
+            // counts tile starts over all pairs.  It is a pacing hint, not a dependency: a pair
+            // that waits longer than kClockPatienceNs (pairs not co-resident, say) leaves the
+            // clock for the rest of the launch, counting as finished so that nobody waits for it.
+            if (my_tiles >= kClockWindow) {
+              const unsigned int need = (unsigned int)n_pairs * (my_tiles - kClockWindow + 1);
+              const unsigned long long t0 = globaltimer_ns();
+              unsigned int seen;
+              for (;;) {
+                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(tile_clock) : "memory");
+                if (seen >= need) break;
+                if (globaltimer_ns() - t0 > patience) { clock_on = false; break; }
+                __nanosleep(100);
+              }
+            }
+            if (clock_on) { atomicAdd(tile_clock, 1u); ++my_tiles; }
+            else if (clock_most > my_tiles) atomicAdd(tile_clock, clock_most - my_tiles);
+          }
           for (int kb = 0; kb < g.k_blocks; ++kb) {
             if (!mbar_wait(empty_bar(stage), phase ^ 1u, &abort_flag)) { ok = false; break; }
             const uint32_t a_dst = tiles + stage * kPairStageBytes;
@@ -510,6 +540,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
           }
         }
       }
+      // a pair that runs out of work counts as having started every remaining tile
+      if (clock_on && clock_most > my_tiles) atomicAdd(tile_clock, clock_most - my_tiles);
     }
     __syncwarp();
   } else if (warp == 1) {

@@ -12,17 +12,17 @@ from gpu_util import GRAD_RTOL, device, f32, np_of
 pytestmark = pytest.mark.gpu
 
 
-PAIR = False   # which GEMM variant the helpers below select
+VARIANT = 0    # which GEMM variant the helpers below select (0 = library default)
 
 
-@pytest.fixture(autouse=True, params=[False, True], ids=["cta", "pair"])
+@pytest.fixture(autouse=True, params=[1, 2], ids=["cta", "pair"])
 def gemm_variant(request):
     """Every test of this module runs on both tensor-core main loops: one CTA per 128 x 256
-    tile (the default) and a CTA pair per 256 x 256 tile."""
-    global PAIR
-    PAIR = request.param
+    tile and a CTA pair per 256 x 256 tile (the default)."""
+    global VARIANT
+    VARIANT = request.param
     yield
-    PAIR = False
+    VARIANT = 0
 
 
 @pytest.fixture(scope="module")
@@ -48,7 +48,7 @@ def run_bwd(ctx, H, W, y, g, lse, token_block=0, accumulate=False, dW_init=None)
     V = W.shape[0]
     dH = torch.full((max(T, 1), d), 7.0, dtype=torch.bfloat16, device=dev)
     dW = torch.full((V, d), 7.0, device=dev) if dW_init is None else dW_init.clone()
-    ctx.set_tuning(0, token_block, PAIR)
+    ctx.set_tuning(0, token_block, VARIANT)
     ctx.policy_loss_backward(H.to(dev), W.to(dev), y.to(dev), f32(lse), g.to(dev), dH, dW, accumulate, T=T)
     flags = ctx.check_device_errors()
     ctx.set_tuning(0, 0)
@@ -95,7 +95,7 @@ def test_cfg4_mini_chain(ctx):
     # GPU chain
     Hd, Wd, yd = H.to(dev), W.to(dev), y.to(dev)
     logp_d, ent_d, lse_d, g_d = (torch.empty(T, device=dev) for _ in range(4))
-    ctx.set_tuning(0, 0, PAIR)
+    ctx.set_tuning(0, 0, VARIANT)
     ctx.token_logprob(Hd, Wd, yd, logp_d, ent_d, lse_d)
     out = B.new_loss_out(dev)
     ctx.policy_loss(logp_d, old.to(dev), ref.to(dev), f32(adv), torch.as_tensor(cu.astype(np.int32), device=dev), out,

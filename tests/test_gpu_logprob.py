@@ -12,17 +12,17 @@ from gpu_util import LOGP_TOL, device, np_of
 pytestmark = pytest.mark.gpu
 
 
-PAIR = False   # which GEMM variant the helpers below select
+VARIANT = 0    # which GEMM variant the helpers below select (0 = library default)
 
 
-@pytest.fixture(autouse=True, params=[False, True], ids=["cta", "pair"])
+@pytest.fixture(autouse=True, params=[1, 2], ids=["cta", "pair"])
 def gemm_variant(request):
     """Every test of this module runs on both tensor-core main loops: one CTA per 128 x 256
-    tile (the default) and a CTA pair per 256 x 256 tile."""
-    global PAIR
-    PAIR = request.param
+    tile and a CTA pair per 256 x 256 tile (the default)."""
+    global VARIANT
+    VARIANT = request.param
     yield
-    PAIR = False
+    VARIANT = 0
 
 
 @pytest.fixture(scope="module")
@@ -38,7 +38,7 @@ def run_case(ctx, H, W, y, splits=0):
     T = H.shape[0]
     Hd, Wd, yd = H.to(dev), W.to(dev), y.to(dev)
     logp, ent, lse = (torch.full((T,), 9.0, device=dev) for _ in range(3))
-    ctx.set_tuning(splits, 0, PAIR)
+    ctx.set_tuning(splits, 0, VARIANT)
     ctx.token_logprob(Hd, Wd, yd, logp, ent, lse)
     flags = ctx.check_device_errors()
     ctx.set_tuning(0, 0)
