@@ -36,10 +36,10 @@ METRIC = "scored tokens/sec (logprob+GRPO loss) at Qwen-7B head; % dense-BF16 pe
 UNIT = "tokens/s"
 KERNELS_PER_STEP = 7  # advantage, pack table fetch, pack columns, pack rows (bulk copy), fused LM-head GEMM, partial merge, loss
 # DRAM bytes per scored token of the fused LM-head kernel (dram__bytes_read + dram__bytes_write of
-# one ncu capture at T = 65536, d = 3584, V = 152064; traffic grows with the number of waves of
-# row tiles, i.e. in proportion to T).  Valid for the 7B head shape only; None whenever the kernel
+# one ncu capture of the CTA-pair kernel at T = 65536, d = 3584, V = 152064: 35.605 GB + 10.1 MB;
+# traffic grows with the number of waves of row tiles, i.e. in proportion to T).  Valid for the 7B head shape only; None whenever the kernel
 # or its work decomposition has changed since the counters were taken.
-GEMM_DRAM_BYTES_PER_TOKEN_7B = None
+GEMM_DRAM_BYTES_PER_TOKEN_7B = (35.605443e9 + 10.11e6) / 65536
 BWD_TOKEN_BLOCK = 9472  # the library's default backward block (3 GEMM launches per block)
 
 
@@ -453,7 +453,8 @@ def run_ours(args):
                      "frac_of_burst": achieved / peaks["bf16_tflops"], "frac_of_nominal_2250": achieved / 2250.0,
                      "kernel_ms": gemm_ms,
                      "traffic": (GEMM_DRAM_BYTES_PER_TOKEN_7B * job.T
-                                 if GEMM_DRAM_BYTES_PER_TOKEN_7B and (w.d, w.V) == (3584, 152064) else None)},
+                                 if GEMM_DRAM_BYTES_PER_TOKEN_7B and (w.d, w.V) == (3584, 152064)
+                                 and args.gemm != "single" and not w.token_budget else None)},
         "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": job.h2d_bytes,
                 "d2h_bytes_per_step": int(sum(lo.numel() for lo in job.loss_outs)), "ms_per_step": ms_e2e},
         "gpu_launches": job.launches_per_step * args.steps,
