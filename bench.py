@@ -36,10 +36,11 @@ METRIC = "scored tokens/sec (logprob+GRPO loss) at Qwen-7B head; % dense-BF16 pe
 UNIT = "tokens/s"
 KERNELS_PER_STEP = 7  # advantage, pack table fetch, pack columns, pack rows (bulk copy), fused LM-head GEMM, partial merge, loss
 # DRAM bytes per scored token of the fused LM-head kernel (dram__bytes_read + dram__bytes_write of
-# one ncu capture of the CTA-pair kernel at T = 65536, d = 3584, V = 152064: 35.605 GB + 10.1 MB;
-# traffic grows with the number of waves of row tiles, i.e. in proportion to T).  Valid for the 7B head shape only; None whenever the kernel
+# one ncu capture of the CTA-pair kernel at T = 65536, d = 3584, V = 152064 with the three
+# vocabulary ranges the library picks at the bench size: 13.655 GB + 8.4 MB; traffic grows with the
+# number of waves of row tiles, i.e. in proportion to T).  Valid for the 7B head shape only; None whenever the kernel
 # or its work decomposition has changed since the counters were taken.
-GEMM_DRAM_BYTES_PER_TOKEN_7B = (35.605443e9 + 10.11e6) / 65536
+GEMM_DRAM_BYTES_PER_TOKEN_7B = (13.654645e9 + 8.38e6) / 65536
 BWD_TOKEN_BLOCK = 9472  # the library's default backward block (3 GEMM launches per block)
 
 
@@ -148,11 +149,11 @@ def allreduce_sum_(t: torch.Tensor, world: int) -> torch.Tensor:
 class ScoringJob:
     """Device buffers of one rank and the step function that runs the path through the C ABI."""
 
-    def __init__(self, w: wl.Workload, device: torch.device, gemm_variant: int = 0, world: int = 1):
+    def __init__(self, w: wl.Workload, device: torch.device, gemm_variant: int = 0, world: int = 1, v_splits: int = 0):
         from paper_2507_01663_b200 import binding as B
         self.B, self.w, self.dev, self.world = B, w, device, world
         self.ctx = B.Context(device.index or 0)
-        self.ctx.set_tuning(0, 0, gemm_variant)
+        self.ctx.set_tuning(v_splits, 0, gemm_variant)
         T = w.total_tokens
         self.T = T
         self.store = {
@@ -312,6 +313,47 @@ class ScoringJob:
                 "token_spread_free_counts": int(sums_pp.max() - sums_pp.min()),
                 "mean_tokens_per_group": float(sums.mean())}
 
+    # -- delayed parameter update: new weights arrive while scoring goes on -----------------
+    def make_weight_refresh(self):
+        """A pinned host copy of the LM-head weight (the "received new parameters"), a standby
+        device buffer and a copy stream.  Scoring keeps using the old weight while the new one is
+        loaded; the buffers are swapped at the first micro-batch boundary after the load."""
+        self.W_host = torch.empty(self.W.shape, dtype=self.W.dtype, pin_memory=True)
+        self.W_host.copy_(self.W)
+        self.W_standby = torch.empty_like(self.W)
+        self.w_stream = torch.cuda.Stream()
+        self.w_loaded = torch.cuda.Event()
+        self.w_released = torch.cuda.Event()      # last kernel that read the standby buffer has run
+        torch.cuda.synchronize()
+        self.w_released.record()
+        self.w_swaps = 0
+
+    def step_with_weight_refresh(self):
+        w, c = self.w, self.ctx
+        main = torch.cuda.current_stream()
+        with torch.cuda.stream(self.w_stream):
+            self.w_stream.wait_event(self.w_released)
+            self.W_standby.copy_(self.W_host, non_blocking=True)
+            self.w_loaded.record(self.w_stream)
+        pending = True
+        c.grpo_advantage(self.reward, None, w.n_prompts, self.adv)
+        store = {"tok_offset_host": self.off, "d": w.d, "adv": self.adv, **self.store}
+        total = 0
+        for i, (mb, loss_out) in enumerate(zip(self.mbs, self.loss_outs)):
+            if pending and (self.w_loaded.query() or i == len(self.mbs) - 1):
+                main.wait_event(self.w_loaded)                 # no-op when the load has finished
+                self.W, self.W_standby = self.W_standby, self.W
+                self.w_released.record(main)                   # kernels enqueued so far read the old buffer
+                self.w_swaps += 1
+                pending = False
+            T = c.pack_microbatch(store, mb, self.packed)
+            c.token_logprob(self.packed["hidden"], self.W, self.packed["target"], self.logp, self.ent, self.lse, T=T)
+            c.policy_loss(self.logp, self.packed["old_logp"], self.packed["ref_logp"], self.packed["adv_seq"],
+                          self.packed["cu_seqlens"], loss_out, self.dlogp, self.ent,
+                          w.clip_eps, w.clip_eps, w.kl_coef, 0, 1.0 / self.world, B=len(mb), T=T)
+            total += T
+        return total
+
     # -- end-to-end: store columns start in pinned host memory ------------------------------
     def make_host_store(self):
         """Pinned host copies of the store columns and rewards, a second device copy of the store
@@ -402,7 +444,7 @@ def run_ours(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
     w = rank_workload(args.workload, rank)
-    job = ScoringJob(w, dev, {"default": 0, "single": 1, "pair": 2}[args.gemm], world)
+    job = ScoringJob(w, dev, {"default": 0, "single": 1, "pair": 2}[args.gemm], world, args.v_splits)
     peaks = measured_peaks()
     hbm_alone = job.hbm_kernels_at_scale(peaks["hbm_gbs"]) if rank == 0 and world == 1 else {}
 
@@ -431,6 +473,18 @@ def run_ours(args):
     ms_e2e_total = timed_loop(job.step_e2e, args.steps, world)
     ms_e2e, _ = reduce_over_ranks(ms_e2e_total / args.steps, job.T, world)
 
+    refresh = None
+    if args.weight_refresh and not w.backward:
+        job.make_weight_refresh()
+        for _ in range(2):
+            job.step_with_weight_refresh()
+        ms_r_total = timed_loop(job.step_with_weight_refresh, args.steps, world)
+        ms_r, _ = reduce_over_ranks(ms_r_total / args.steps, job.T, world)
+        refresh = {"value": tokens / (ms_r * 1e-3), "unit": UNIT, "ms_per_step": ms_r,
+                   "h2d_bytes_per_step": int(job.W.numel() * job.W.element_size()), "swaps": job.w_swaps,
+                   "what": "every step a new LM-head weight is loaded from pinned host memory on a second stream "
+                           "while scoring continues with the old one; swapped at a micro-batch boundary"}
+
     flops = 2.0 * job.T * w.d * w.V
     achieved = flops / (gemm_ms * 1e-3) / 1e12
     peak = peaks["bf16_tflops_sustained"]
@@ -454,7 +508,7 @@ def run_ours(args):
                      "kernel_ms": gemm_ms,
                      "traffic": (GEMM_DRAM_BYTES_PER_TOKEN_7B * job.T
                                  if GEMM_DRAM_BYTES_PER_TOKEN_7B and (w.d, w.V) == (3584, 152064)
-                                 and args.gemm != "single" and not w.token_budget else None)},
+                                 and args.gemm != "single" and args.v_splits == 0 and not w.token_budget else None)},
         "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": job.h2d_bytes,
                 "d2h_bytes_per_step": int(sum(lo.numel() for lo in job.loss_outs)), "ms_per_step": ms_e2e},
         "gpu_launches": job.launches_per_step * args.steps,
@@ -468,6 +522,8 @@ def run_ours(args):
                                                        "where": "inside the timed steps (all micro-batches of a step), "
                                                                 "each right after a GEMM (part at its power cap)"}}
     line["hbm_kernels"].update(hbm_alone)
+    if refresh is not None:
+        line["weight_refresh"] = refresh
     if rank == 0:
         line["balance"] = job.balance_report()
     if bwd_ms is not None:
@@ -531,6 +587,10 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2")
     ap.add_argument("--cpu-sample", type=int, default=1536, help="tokens in the CPU-oracle sample")
+    ap.add_argument("--v-splits", type=int, default=0,
+                    help="vocabulary ranges per row tile of the fused GEMM (af_set_tuning v_splits); 0 = the library's choice")
+    ap.add_argument("--weight-refresh", action="store_true",
+                    help="also time the steps while a new LM-head weight is loaded and swapped in every step")
     ap.add_argument("--gemm", default="default", choices=["default", "single", "pair"],
                     help="main loop of the tensor-core GEMMs (af_set_tuning gemm_variant): CTA pairs (the default) "
                          "or one CTA per tile")

@@ -116,7 +116,9 @@ int logprob_pick_splits(int64_t T, int32_t d, int32_t V, int sm_count, bool pair
   const int n_tiles = (V + umma::kBN - 1) / umma::kBN;
   if (requested > 0) return requested < n_tiles ? requested : n_tiles;
   if (m_tiles < 1) return 1;
-  constexpr int64_t kPanelBudget = 72ll << 20;        // bytes of hidden-state rows kept in L2
+  // bytes of hidden-state rows kept in L2: pairs sharing a row tile may sit on different dies, each
+  // of which then caches the panel in its own half of L2, so pairs get the smaller budget
+  const int64_t kPanelBudget = pair ? (48ll << 20) : (72ll << 20);
   const int64_t max_units_many = (int64_t)workers * 8;
   int best = 1;
   double best_cost = 1e300;
