@@ -148,9 +148,9 @@ af_status af_reserve(af_ctx* c, int64_t max_T, int32_t max_B, int32_t d, int32_t
   af_status st = AF_OK;
   if (max_T > 0) {
     const int S = logprob_pick_splits(max_T, d, V, c->sm_count, c->gemm_pair != 0, c->v_splits);
-    // smaller batches may pick up to 4 ranges whatever their size, and more than 4 only while
-    // there are at most 8 units per SM
-    size_t need = (size_t)(S > 4 ? S : 4) * (size_t)max_T;
+    // smaller batches may pick up to 8 ranges whatever their size, and more than 8 only while
+    // there are at most 8 units per worker
+    size_t need = (size_t)(S > 8 ? S : 8) * (size_t)max_T;
     size_t small = (size_t)c->sm_count * 8 * 128;
     if (need < small) need = small;
     st = ws_grow(c->partial, need * 16);

@@ -107,8 +107,8 @@ __global__ void __launch_bounds__(256) merge_partials_kernel(
 // ceil(m_tiles S / workers) * ceil(n_tiles / S) tile times: S is chosen to minimise that product
 // (wave quantisation decides it for small batches).  The workers alive at one time sweep the
 // vocabulary over ceil(workers / S) row tiles whose hidden-state panels should stay L2-resident
-// while W streams past once, which rules out small S for wide hidden sizes.  Many ranges are only
-// allowed while S * T stays small (partials buffer).
+// while W streams past once, which rules out small S for wide hidden sizes.  More than 8 ranges are
+// only allowed while S * T stays small (partials buffer).
 int logprob_pick_splits(int64_t T, int32_t d, int32_t V, int sm_count, bool pair, int requested) {
   const int tile_rows = pair ? umma::kPairBM : umma::kBM;
   const int workers = pair ? (sm_count / 2 > 0 ? sm_count / 2 : 1) : (sm_count > 0 ? sm_count : 1);
@@ -124,7 +124,7 @@ int logprob_pick_splits(int64_t T, int32_t d, int32_t V, int sm_count, bool pair
   double best_cost = 1e300;
   for (int S = 1; S <= 32 && S <= n_tiles; ++S) {
     const int64_t units = m_tiles * S;
-    if (S > 4 && units > max_units_many) break;
+    if (S > 8 && units > max_units_many) break;
     int64_t alive = (workers + S - 1) / S;
     if (alive > m_tiles) alive = m_tiles;
     const bool fits = alive * tile_rows * (int64_t)d * 2 <= kPanelBudget;

@@ -337,12 +337,11 @@ cudaError_t launch_policy_loss(const float* logp, const float* old_logp, const f
                                int32_t B, int64_t T, const af_loss_params& p, af_loss_out* out,
                                float* dlogp, void* ws, unsigned int* d_err, int sm_count,
                                cudaStream_t s) {
-  static bool attr_set = false;
-  if (!attr_set) {
+  // set on every launch: the attribute is per device, and a process may drive several
+  {
     cudaError_t e = cudaFuncSetAttribute(policy_loss_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          kRingSmemBytes);
     if (e != cudaSuccess) return e;
-    attr_set = true;
   }
   const int64_t chunks = (T + kChunk - 1) / kChunk;
   // two CTAs per SM, each over a contiguous range of chunks (grid <= the workspace's 8 blocks per SM)

@@ -238,12 +238,11 @@ cudaError_t launch_pack(const af_store_view& st, const af_packed& out, const Pac
   if (T > 0 && out.hidden) {
     const int rpc = pack_rows_per_chunk(st.d);
     if (rpc > 0 && tab.n_chunks > 0) {
-      static bool attr_set = false;
-      if (!attr_set) {
+      // set on every launch: the attribute is per device, and a process may drive several
+      {
         cudaError_t e = cudaFuncSetAttribute(pack_rows_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              kCopySmemBytes);
         if (e != cudaSuccess) return e;
-        attr_set = true;
       }
       const int grid = tab.n_chunks < sm_count ? tab.n_chunks : sm_count;
       pack_rows_bulk_kernel<<<grid, 32, kCopySmemBytes, s>>>(

@@ -157,3 +157,41 @@ def test_bitwise_reproducible(ctx):
     b = run_case(ctx, H, W, y)
     for x, z in zip(a[:3], b[:3]):
         assert x.tobytes() == z.tobytes()
+
+
+def test_weights_swapped_between_microbatches(ctx):
+    """Delayed parameter update: while micro-batches are scored with the old LM-head weight, the
+    new one is loaded into a standby buffer on a second stream; after the swap at a micro-batch
+    boundary the results are those of the new weight, before it those of the old one, bit for bit
+    (the load does not disturb the scoring in flight)."""
+    dev = device()
+    H, W0, y = random_case(640, 256, 4104, seed=21)
+    _, W1, _ = random_case(640, 256, 4104, seed=22)
+    Hd, yd = H.to(dev), y.to(dev)
+    ctx.set_tuning(0, 0, VARIANT)
+
+    def score(Wd, rows):
+        out = torch.empty(rows.stop - rows.start, device=dev)
+        ctx.token_logprob(Hd[rows], Wd, yd[rows], out)
+        return out
+
+    ref0 = [score(W0.to(dev), r) for r in (slice(0, 300), slice(300, 640))]
+    ref1 = [score(W1.to(dev), r) for r in (slice(0, 300), slice(300, 640))]
+    torch.cuda.synchronize()
+    active, standby = W0.to(dev), torch.empty_like(W0, device=dev)
+    W1_host = W1.pin_memory()
+    side, loaded = torch.cuda.Stream(), torch.cuda.Event()
+    with torch.cuda.stream(side):
+        standby.copy_(W1_host, non_blocking=True)          # arrives while micro-batch 0 is scored
+        loaded.record(side)
+    got0 = score(active, slice(0, 300))
+    torch.cuda.current_stream().wait_event(loaded)
+    active, standby = standby, active                      # swap at the micro-batch boundary
+    got1 = score(active, slice(300, 640))
+    torch.cuda.synchronize()
+    ctx.set_tuning(0, 0)
+    assert torch.equal(got0, ref0[0]) and torch.equal(got1, ref1[1])
+    assert not torch.equal(got1, ref0[1])
+    lp_ref, _, _ = O.token_logprob_ref(wl.bf16_bits(H[300:]), wl.bf16_bits(W1), y[300:].numpy())
+    assert np.abs(np_of(got1) - lp_ref).max() <= LOGP_TOL
+    assert ctx.check_device_errors() == 0
