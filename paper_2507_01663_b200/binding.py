@@ -71,13 +71,18 @@ _lib = None
 
 
 def load_library() -> C.CDLL:
-    """dlopen the in-tree library; fail loudly if it has not been built."""
+    """dlopen the in-tree library.  A missing library is compiled first when nvcc is at hand (a
+    fresh checkout); otherwise this fails loudly: there is no fallback implementation."""
     global _lib
     if _lib is not None:
         return _lib
     if not os.path.exists(LIB_PATH):
-        raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2507_01663_b200.build` "
-                          "(there is no fallback implementation)")
+        try:
+            from . import build as _build
+            _build.build()
+        except Exception as exc:
+            raise ImportError(f"{LIB_PATH} is missing and could not be built ({exc}): run "
+                              "`python -m paper_2507_01663_b200.build` (there is no fallback implementation)")
     lib = C.CDLL(LIB_PATH)
     vp, i32, i64, f32 = C.c_void_p, C.c_int32, C.c_int64, C.c_float
     lib.af_create.argtypes = [C.POINTER(vp), C.c_int]
