@@ -195,3 +195,58 @@ def test_weights_swapped_between_microbatches(ctx):
     lp_ref, _, _ = O.token_logprob_ref(wl.bf16_bits(H[300:]), wl.bf16_bits(W1), y[300:].numpy())
     assert np.abs(np_of(got1) - lp_ref).max() <= LOGP_TOL
     assert ctx.check_device_errors() == 0
+
+
+def test_two_contexts_on_two_streams_do_not_disturb_each_other(ctx):
+    """Two scoring calls of full-grid size in flight at once (two contexts, two streams): the
+    CTAs of the second cannot all be resident while the first runs, which is the situation the
+    pacing of the CTA pairs has to give way in.  Results equal those of the calls made one
+    after the other, bit for bit."""
+    from paper_2507_01663_b200 import binding as B
+    dev = device()
+    other = B.Context(0)
+    try:
+        cases = [random_case(19000, 256, 4104, seed=31), random_case(18000, 320, 4104, seed=32)]
+        dev_in = [(H.to(dev), W.to(dev), y.to(dev)) for H, W, y in cases]
+        ctxs, streams = [ctx, other], [torch.cuda.Stream(), torch.cuda.Stream()]
+        for c in ctxs:
+            c.set_tuning(0, 0, VARIANT)
+        ref = []
+        for c, (H, W, y) in zip(ctxs, dev_in):
+            out = [torch.empty(H.shape[0], device=dev) for _ in range(3)]
+            c.token_logprob(H, W, y, *out)
+            ref.append(out)
+        torch.cuda.synchronize()
+        for rep in range(3):
+            got = []
+            for c, s, (H, W, y) in zip(ctxs, streams, dev_in):
+                out = [torch.empty(H.shape[0], device=dev) for _ in range(3)]
+                with torch.cuda.stream(s):
+                    c.token_logprob(H, W, y, *out, stream=s)
+                got.append(out)
+            torch.cuda.synchronize()
+            for g, r in zip(got, ref):
+                assert all(torch.equal(a, b) for a, b in zip(g, r))
+        assert ctx.check_device_errors() == 0 and other.check_device_errors() == 0
+    finally:
+        ctx.set_tuning(0, 0)
+        other.close()
+
+
+def test_reserved_workspace_does_not_grow(ctx):
+    """After af_reserve for the largest batch, scoring calls of that size and smaller ones (which
+    pick other numbers of vocabulary ranges) allocate nothing more."""
+    dev = device()
+    T, d, V = 6000, 128, 8200
+    ctx.set_tuning(0, 0, VARIANT)
+    ctx.reserve(T, 64, d, V)
+    held = ctx.workspace_bytes()
+    H, W, y = random_case(T, d, V, seed=41)
+    Hd, Wd, yd = H.to(dev), W.to(dev), y.to(dev)
+    out = torch.empty(T, device=dev)
+    for t in (T, T // 2, 700, 129, 1):
+        ctx.token_logprob(Hd, Wd, yd, out, T=t)
+    torch.cuda.synchronize()
+    ctx.set_tuning(0, 0)
+    assert ctx.workspace_bytes() == held
+    assert ctx.check_device_errors() == 0
