@@ -97,6 +97,46 @@ def token_logprob_ref(H_bits, W_bits, y, return_rows=False):
 
 
 # ----------------------------------------------------------------------------------------
+# O2b  the same scoring with the vocabulary sharded over model-parallel ranks: every rank sees
+#      the rows [v_offset, v_offset + V_shard) of W and reports four numbers per token; one
+#      exchange of those numbers and a merge give the full-vocabulary result.  (The paper's
+#      inference and training instances run under tensor parallelism, Section 3.1 and Table 1;
+#      it does not describe the head.  The four statistics are the ones a softmax needs.)
+# ----------------------------------------------------------------------------------------
+def token_logprob_shard_ref(H_bits, W_shard_bits, y, v_offset):
+    """Per token over the shard's logits z_v = H W_shard^T:
+         m = max_v z_v;  s = sum_v exp(z_v - m);  u = sum_v exp(z_v - m) z_v;
+         zy = z at the target if the target id falls into the shard, else -inf.
+    Returns float64 [T, 4] = (m, s, u, zy)."""
+    H = bf16_bits_to_f64(H_bits)
+    W = bf16_bits_to_f64(W_shard_bits)
+    y = np.asarray(y, dtype=np.int64) - int(v_offset)
+    z = H @ W.T
+    m = z.max(axis=1)
+    e = np.exp(z - m[:, None])
+    out = np.empty((z.shape[0], 4), dtype=np.float64)
+    out[:, 0] = m
+    out[:, 1] = e.sum(axis=1)
+    out[:, 2] = (e * z).sum(axis=1)
+    inside = (y >= 0) & (y < z.shape[1])
+    out[:, 3] = np.where(inside, z[np.arange(z.shape[0]), np.clip(y, 0, z.shape[1] - 1)], -np.inf)
+    return out
+
+
+def merge_logprob_shards_ref(partials):
+    """partials [R, T, 4] from token_logprob_shard_ref -> logp, ent, lse over the whole vocabulary:
+         M = max_r m_r;  S = sum_r s_r exp(m_r - M);  U = sum_r u_r exp(m_r - M)
+         lse = M + log S;  logp = max_r zy_r - lse;  ent = lse - U / S."""
+    P = np.asarray(partials, dtype=np.float64)
+    M = P[:, :, 0].max(axis=0)
+    w = np.exp(P[:, :, 0] - M[None, :])
+    S = (P[:, :, 1] * w).sum(axis=0)
+    U = (P[:, :, 2] * w).sum(axis=0)
+    lse = M + np.log(S)
+    return P[:, :, 3].max(axis=0) - lse, lse - U / S, lse
+
+
+# ----------------------------------------------------------------------------------------
 # O3  GRPO group-normalised advantage                       (Section 6.1 "RL algorithms")
 # ----------------------------------------------------------------------------------------
 def grpo_advantage_ref(reward, group_id, n_groups, eps_adv=1e-6, ddof=0):

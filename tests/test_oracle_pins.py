@@ -423,3 +423,34 @@ def test_backward_structure():
     lp = torch.log_softmax(Ht @ Wt.T, 1)[torch.arange(T), torch.from_numpy(y)]
     (lp * torch.from_numpy(g)).sum().backward()
     assert np.allclose(Ht.grad.numpy(), dH, atol=1e-12) and np.allclose(Wt.grad.numpy(), dW, atol=1e-12)
+
+
+# ---------------------------------------------------------------- O2b vocabulary shards
+@pytest.mark.parametrize("cuts", [[0, 50], [0, 17, 50], [0, 1, 2, 49, 50], [0, 25, 25, 50]])
+def test_sharded_scoring_merges_to_the_full_vocabulary_result(cuts):
+    """Any split of the vocabulary into contiguous shards (an empty one included) merges to the
+    full-row definition, which is pinned above on its own."""
+    rng = np.random.default_rng(5)
+    H = to_bits(rng.normal(size=(9, 12)))
+    W = to_bits(rng.normal(size=(50, 12)) * 3.0)          # wide logits: the max shift matters
+    y = rng.integers(0, 50, 9)
+    parts = []
+    for a, b in zip(cuts[:-1], cuts[1:]):
+        if b > a:
+            parts.append(O.token_logprob_shard_ref(H, W[a:b], y, a))
+    logp, ent, lse = O.merge_logprob_shards_ref(np.stack(parts))
+    r_logp, r_ent, r_lse = O.token_logprob_ref(H, W, y)
+    assert np.allclose(logp, r_logp, atol=1e-12) and np.allclose(ent, r_ent, atol=1e-12)
+    assert np.allclose(lse, r_lse, atol=1e-12)
+
+
+def test_shard_statistics_by_hand():
+    # one token, hidden = [1, 0], shard rows give logits (2, 0, 1); target id 11 with offset 10 -> z = 0
+    H = to_bits(np.array([[1.0, 0.0]]))
+    W = to_bits(np.array([[2.0, 5.0], [0.0, -1.0], [1.0, 7.0]]))
+    p = O.token_logprob_shard_ref(H, W, np.array([11]), 10)[0]
+    assert p[0] == 2.0
+    assert abs(p[1] - (1.0 + math.exp(-2.0) + math.exp(-1.0))) < 1e-15
+    assert abs(p[2] - (2.0 + 0.0 + math.exp(-1.0))) < 1e-15
+    assert p[3] == 0.0
+    assert O.token_logprob_shard_ref(H, W, np.array([3]), 10)[0][3] == -np.inf      # target in another shard
