@@ -132,7 +132,7 @@ af_status af_pack_microbatch(af_ctx* ctx, const af_store_view* store, const int3
 /* ---------------------------------------------------------------------------------------------
  * af_token_logprob -- LM-head projection fused with an online log-softmax (the last stage of
  * the `compute_log_prob` task of the paper's backend interface, Appendix "Backend-level
- * interface"; forward-only for reference / actor inference, Section 6.4).
+ * interface"; forward-only for reference / actor inference, Section 7.4).
  *
  * For each token t:  z_tv = sum_k hidden[t,k] * W[v,k]  (bf16 x bf16, fp32 accumulation; the
  * [T,V] logits are never written to memory);  lse_t = log sum_v exp z_tv;
@@ -148,7 +148,7 @@ af_status af_token_logprob(af_ctx* ctx, const void* hidden, const void* W, const
 
 /* ---------------------------------------------------------------------------------------------
  * af_grpo_advantage -- group-normalised advantages: "rewards normalized within a group of
- * responses to the same prompt" (paper Section 6.1 "RL algorithms"; no critic).
+ * responses to the same prompt" (paper Section 7.1 "RL algorithms"; no critic).
  *
  * For each group g with members I_g (n_g = |I_g|):  mu = mean r;  sigma = sqrt(sum (r-mu)^2 /
  * (n_g - ddof));  adv_i = (r_i - mu) / (sigma + eps_adv).  A group of equal rewards gets zeros.
@@ -165,7 +165,7 @@ af_status af_grpo_advantage(af_ctx* ctx, const float* reward, const int32_t* gro
 
 /* ---------------------------------------------------------------------------------------------
  * af_policy_loss -- clipped-ratio GRPO policy loss with a k3 KL penalty against the reference
- * log-probs (the loss of the paper's actor-update task, Section 6.4; GRPO, Section 6.1).
+ * log-probs (the loss of the paper's actor-update task, Section 7.4; GRPO, Section 7.1).
  *
  * Token t of sequence i, A = adv_seq[i]:
  *   rho = exp(logp - old);  pg = -min(rho*A, clip(rho, 1-clip_lo, 1+clip_hi)*A);
@@ -203,7 +203,7 @@ af_status af_policy_loss(af_ctx* ctx, const float* logp, const float* old_logp,
 
 /* ---------------------------------------------------------------------------------------------
  * af_policy_loss_backward -- gradient of the loss through log-softmax and the LM head (the
- * forward-backward actor-update task, paper Section 6.4), without materialising [T,V].
+ * forward-backward actor-update task, paper Section 7.4), without materialising [T,V].
  *
  *   dZ_tv = dlogp[t] * ( 1{v == target[t]} - exp(z_tv - lse[t]) )      (z recomputed per block)
  *   d_hidden[t,:] = sum_v dZ_tv * W[v,:]          -> [T,d] bf16

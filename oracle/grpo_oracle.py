@@ -9,7 +9,7 @@ The paper (AsyncFlow) states the data flow -- a sample-indexed columnar store re
 index (Section 4.3 "Data Plane"), micro-batches handed out as metadata and fetched by the
 worker (Section 4.2 "Interaction Interface"), the ``compute_log_prob`` task (Appendix, Backend
 -level interface listing), GRPO advantages "normalized within a group of responses to the same
-prompt" (Section 6.1 "RL algorithms") -- but prints no formula.  The arithmetic is therefore the
+prompt" (Section 7.1 "RL algorithms") -- but prints no formula.  The arithmetic is therefore the
 textbook definition of each quantity, written out below with no blocking, fusion or reordering:
 
   log-softmax / entropy .... the definition over the full vocabulary row
@@ -99,9 +99,9 @@ def token_logprob_ref(H_bits, W_bits, y, return_rows=False):
 # ----------------------------------------------------------------------------------------
 # O2b  the same scoring with the vocabulary sharded over model-parallel ranks: every rank sees
 #      the rows [v_offset, v_offset + V_shard) of W and reports four numbers per token; one
-#      exchange of those numbers and a merge give the full-vocabulary result.  (The paper's
-#      inference and training instances run under tensor parallelism, Section 3.1 and Table 1;
-#      it does not describe the head.  The four statistics are the ones a softmax needs.)
+#      exchange of those numbers and a merge give the full-vocabulary result.  (The paper names
+#      tensor parallelism among the strategies its instances combine, Section 2.1; it does not
+#      describe the head.  The four statistics are the ones a softmax needs.)
 # ----------------------------------------------------------------------------------------
 def token_logprob_shard_ref(H_bits, W_shard_bits, y, v_offset):
     """Per token over the shard's logits z_v = H W_shard^T:
@@ -137,7 +137,7 @@ def merge_logprob_shards_ref(partials):
 
 
 # ----------------------------------------------------------------------------------------
-# O3  GRPO group-normalised advantage                       (Section 6.1 "RL algorithms")
+# O3  GRPO group-normalised advantage                       (Section 7.1 "RL algorithms")
 # ----------------------------------------------------------------------------------------
 def grpo_advantage_ref(reward, group_id, n_groups, eps_adv=1e-6, ddof=0):
     """A_i = (r_i - mean_g) / (std_g + eps_adv); std with divisor n_g - ddof; any id order."""
