@@ -143,13 +143,32 @@ def allreduce_sum_(t: torch.Tensor, world: int) -> torch.Tensor:
     return t
 
 
+def vocab_shard(V: int, world: int, rank: int):
+    """Rows [lo, hi) of the LM head held by `rank` under vocabulary parallelism (multiples of 8)."""
+    per = -(-V // world)
+    per = -(-per // 8) * 8
+    return min(rank * per, V), min((rank + 1) * per, V)
+
+
+def allgather_partials(mine: torch.Tensor, world: int) -> torch.Tensor:
+    """The one exchange of vocabulary-parallel scoring: every rank contributes its [T, 4] shard
+    statistics (16 bytes per token) and receives all of them as [R, T, 4]."""
+    if world == 1:
+        return mine.unsqueeze(0)
+    import torch.distributed as dist
+    out = torch.empty((world,) + tuple(mine.shape), dtype=mine.dtype, device=mine.device)
+    dist.all_gather(list(out.unbind(0)), mine.contiguous())     # the slices are contiguous views of `out`
+    return out
+
+
 # ------------------------------------------------------------------------------------------
 # the CUDA arm
 # ------------------------------------------------------------------------------------------
 class ScoringJob:
     """Device buffers of one rank and the step function that runs the path through the C ABI."""
 
-    def __init__(self, w: wl.Workload, device: torch.device, gemm_variant: int = 0, world: int = 1, v_splits: int = 0):
+    def __init__(self, w: wl.Workload, device: torch.device, gemm_variant: int = 0, world: int = 1, v_splits: int = 0,
+                 vocab_parallel: bool = False, rank: int = 0):
         from paper_2507_01663_b200 import binding as B
         self.B, self.w, self.dev, self.world = B, w, device, world
         self.ctx = B.Context(device.index or 0)
@@ -160,6 +179,8 @@ class ScoringJob:
             "hidden": wl.gen_hidden(w, device), "target": wl.gen_target(w, device),
         }
         self.W = wl.gen_weight(w, device)
+        self.vocab_parallel = vocab_parallel
+        self.v_lo, self.v_hi = vocab_shard(w.V, world, rank) if vocab_parallel else (0, w.V)
         self.reward = wl.gen_reward(w, device)
         centre = wl.centre_logp_estimate(w, self.store["hidden"], self.W, self.store["target"])
         self.store["old_logp"] = centre + wl.gen_noise(w, wl.S_OLD, T, device)
@@ -181,6 +202,9 @@ class ScoringJob:
             "adv_seq": torch.empty(cap_B, device=device),
         }
         self.logp, self.ent, self.lse, self.dlogp = (torch.empty(cap_T, device=device) for _ in range(4))
+        if vocab_parallel:     # this rank keeps only its rows of the head; statistics are exchanged per micro-batch
+            self.W_shard = self.W[self.v_lo:self.v_hi].contiguous()
+            self.partial = torch.empty(cap_T, 4, device=device)
         self.loss_outs = [B.new_loss_out(device) for _ in self.mbs]
         self.loss_out = self.loss_outs[-1]
         if w.backward:
@@ -204,7 +228,13 @@ class ScoringJob:
             if ev:
                 ev[1].record()
                 ev[2].record()
-            c.token_logprob(self.packed["hidden"], self.W, self.packed["target"], self.logp, self.ent, self.lse, T=T)
+            if self.vocab_parallel:
+                c.token_logprob_shard(self.packed["hidden"], self.W_shard, self.packed["target"], self.v_lo,
+                                      self.partial, T=T)
+                gathered = allgather_partials(self.partial[:T], self.world)
+                c.merge_logprob_shards(gathered, self.packed["target"], w.V, self.logp, self.ent, self.lse, T=T)
+            else:
+                c.token_logprob(self.packed["hidden"], self.W, self.packed["target"], self.logp, self.ent, self.lse, T=T)
             if ev:
                 ev[3].record()
             c.policy_loss(self.logp, self.packed["old_logp"], self.packed["ref_logp"], self.packed["adv_seq"],
@@ -443,8 +473,10 @@ def run_ours(args):
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
-    w = rank_workload(args.workload, rank)
-    job = ScoringJob(w, dev, {"default": 0, "single": 1, "pair": 2}[args.gemm], world, args.v_splits)
+    # data parallel: every rank its own batch; vocabulary parallel: one batch, the head split by rows
+    w = rank_workload(args.workload, 0 if args.vocab_parallel else rank)
+    job = ScoringJob(w, dev, {"default": 0, "single": 1, "pair": 2}[args.gemm], world, args.v_splits,
+                     args.vocab_parallel, rank)
     peaks = measured_peaks()
     hbm_alone = job.hbm_kernels_at_scale(peaks["hbm_gbs"]) if rank == 0 and world == 1 else {}
 
@@ -461,6 +493,8 @@ def run_ours(args):
     pack_ms = float(np.sum([a.elapsed_time(b) for a, b in job.pack_events])) / args.steps
     bwd_ms = float(np.sum([a.elapsed_time(b) for a, b in job.bwd_events])) / args.steps if job.bwd_events else None
     ms_step, tokens = reduce_over_ranks(ms_total / args.steps, job.T, world)
+    if args.vocab_parallel:
+        tokens = job.T           # the ranks score the same tokens together
     flags = job.ctx.check_device_errors()
     if flags:
         raise RuntimeError(f"device error word set: {flags}")
@@ -485,13 +519,13 @@ def run_ours(args):
                    "what": "every step a new LM-head weight is loaded from pinned host memory on a second stream "
                            "while scoring continues with the old one; swapped at a micro-batch boundary"}
 
-    flops = 2.0 * job.T * w.d * w.V
+    flops = 2.0 * job.T * w.d * (job.v_hi - job.v_lo)       # this rank's rows of the head
     achieved = flops / (gemm_ms * 1e-3) / 1e12
     peak = peaks["bf16_tflops_sustained"]
     line = {
         "metric": METRIC, "value": tokens / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "scaling": "strong" if args.vocab_parallel else "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": f"{args.workload}: {head_name(w)} head d={w.d} V={w.V}, {w.N} responses "
                                f"({w.n_prompts} prompts x {w.group_size}), {job.T} scored tokens per GPU, "
                                + (f"{len(job.mbs)} arrival-ordered micro-batches of <= {w.token_budget} tokens, packed, "
@@ -587,6 +621,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2")
     ap.add_argument("--cpu-sample", type=int, default=1536, help="tokens in the CPU-oracle sample")
+    ap.add_argument("--vocab-parallel", action="store_true",
+                    help="split the LM head by vocabulary rows over the ranks (one batch for all; shard statistics "
+                         "all-gathered and merged) instead of giving every rank its own batch")
     ap.add_argument("--v-splits", type=int, default=0,
                     help="vocabulary ranges per row tile of the fused GEMM (af_set_tuning v_splits); 0 = the library's choice")
     ap.add_argument("--weight-refresh", action="store_true",

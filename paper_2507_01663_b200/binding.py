@@ -26,7 +26,8 @@ DEVERR_TARGET_RANGE, DEVERR_WATCHDOG, DEVERR_CU_SEQLENS, DEVERR_SAMPLE_INDEX = 1
 EXPORTS = ["af_create", "af_destroy", "af_status_string", "af_reserve", "af_workspace_bytes",
            "af_set_tuning", "af_check_device_errors", "af_pack_microbatch", "af_token_logprob",
            "af_grpo_advantage", "af_policy_loss", "af_policy_loss_backward", "af_token_logprob_static",
-           "af_controller_put", "af_controller_get", "af_controller_clear", "af_balance_partitions"]
+           "af_controller_put", "af_controller_get", "af_controller_clear", "af_balance_partitions",
+           "af_token_logprob_shard", "af_merge_logprob_shards"]
 
 
 class AfError(RuntimeError):
@@ -107,6 +108,8 @@ def load_library() -> C.CDLL:
     lib.af_controller_get.argtypes = [vp, C.POINTER(ControllerView), u32, u32, i32, i64, vp, vp, vp]
     lib.af_controller_clear.argtypes = [vp, C.POINTER(ControllerView), u32, u32, vp]
     lib.af_balance_partitions.argtypes = [vp, i32, i32, i32, vp, vp]
+    lib.af_token_logprob_shard.argtypes = [vp, vp, vp, vp, i64, i32, i32, i32, vp, vp]
+    lib.af_merge_logprob_shards.argtypes = [vp, vp, vp, i32, i64, i32, vp, vp, vp, vp]
     for name in EXPORTS:
         if name not in ("af_status_string", "af_workspace_bytes"):
             getattr(lib, name).restype = C.c_int
@@ -202,6 +205,22 @@ class Context:
         _check(self.lib.af_token_logprob(self.handle, _ptr(hidden), _ptr(W), _ptr(target), T, d, V,
                                          _ptr(logp), _ptr(entropy), _ptr(lse), _stream(stream)),
                "af_token_logprob")
+
+    def token_logprob_shard(self, hidden, W_shard, target, v_offset, partial_out, T=None, stream=None):
+        """``partial_out``: device float32 [T, 4] = (m, s, u, zy) of this vocabulary shard."""
+        T = hidden.shape[0] if T is None else T
+        d, Vs = W_shard.shape[1], W_shard.shape[0]
+        _check(self.lib.af_token_logprob_shard(self.handle, _ptr(hidden), _ptr(W_shard), _ptr(target), T, d, Vs,
+                                               v_offset, _ptr(partial_out), _stream(stream)),
+               "af_token_logprob_shard")
+
+    def merge_logprob_shards(self, partials, target, V_total, logp, entropy=None, lse=None, T=None, stream=None):
+        """``partials``: device float32 [R, T, 4], the shards' statistics after the exchange."""
+        R = partials.shape[0]
+        T = partials.shape[1] if T is None else T
+        _check(self.lib.af_merge_logprob_shards(self.handle, _ptr(partials), _ptr(target), R, T, V_total,
+                                                _ptr(logp), _ptr(entropy), _ptr(lse), _stream(stream)),
+               "af_merge_logprob_shards")
 
     def grpo_advantage(self, reward, group_id, n_groups, adv, eps_adv=1e-6, ddof=0, N=None, stream=None):
         N = reward.shape[0] if N is None else N

@@ -253,6 +253,31 @@ af_status af_token_logprob(af_ctx* c, const void* hidden, const void* W, const i
                               static_cast<cudaStream_t>(stream));
 }
 
+af_status af_token_logprob_shard(af_ctx* c, const void* hidden, const void* W_shard, const int32_t* target,
+                                 int64_t T, int32_t d, int32_t V_shard, int32_t v_offset, float* partial_out,
+                                 void* stream) {
+  if (!c || T < 0 || d < 1 || V_shard < 1 || v_offset < 0) return AF_ERR_INVALID_ARG;
+  if (T == 0) return AF_OK;
+  if (!hidden || !W_shard || !target || !partial_out) return AF_ERR_INVALID_ARG;
+  if (T >= ((int64_t)1 << 31)) return AF_ERR_SHAPE;
+  if (d % 8 != 0 || !aligned16(hidden) || !aligned16(W_shard) || !aligned16(partial_out)) return AF_ERR_ALIGNMENT;
+  DeviceGuard guard(c->device);
+  return launch_token_logprob_shard(c, hidden, W_shard, target, T, d, V_shard, v_offset, partial_out,
+                                    static_cast<cudaStream_t>(stream));
+}
+
+af_status af_merge_logprob_shards(af_ctx* c, const float* partials, const int32_t* target, int32_t R, int64_t T,
+                                  int32_t V_total, float* logp, float* entropy, float* lse, void* stream) {
+  if (!c || T < 0 || R < 1 || V_total < 1) return AF_ERR_INVALID_ARG;
+  if (T == 0) return AF_OK;
+  if (!partials || !target || !logp) return AF_ERR_INVALID_ARG;
+  if (T >= ((int64_t)1 << 31)) return AF_ERR_SHAPE;
+  if (!aligned16(partials)) return AF_ERR_ALIGNMENT;
+  DeviceGuard guard(c->device);
+  return launch_merge_logprob_shards(c, partials, target, R, T, V_total, logp, entropy, lse,
+                                     static_cast<cudaStream_t>(stream));
+}
+
 af_status af_grpo_advantage(af_ctx* c, const float* reward, const int32_t* group_id, int64_t N,
                             int32_t n_groups, float eps_adv, int32_t ddof, float* adv, void* stream) {
   if (!c || N < 0 || n_groups < 0 || (ddof != 0 && ddof != 1) || !(eps_adv >= 0.f)) return AF_ERR_INVALID_ARG;

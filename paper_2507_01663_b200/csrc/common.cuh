@@ -96,6 +96,13 @@ af_status launch_token_logprob(af_ctx* ctx, const void* hidden, const void* W,
                                const int32_t* target, int64_t T, int32_t d, int32_t V,
                                float* logp, float* entropy, float* lse, cudaStream_t s);
 
+af_status launch_token_logprob_shard(af_ctx* ctx, const void* hidden, const void* W_shard,
+                                     const int32_t* target, int64_t T, int32_t d, int32_t V_shard,
+                                     int32_t v_offset, float* partial_out, cudaStream_t s);
+af_status launch_merge_logprob_shards(af_ctx* ctx, const float* partials, const int32_t* target, int32_t R,
+                                      int64_t T, int32_t V_total, float* logp, float* entropy, float* lse,
+                                      cudaStream_t s);
+
 af_status launch_backward(af_ctx* ctx, const void* hidden, const void* W, const int32_t* target,
                           const float* lse, const float* dlogp, int64_t T, int32_t d, int32_t V,
                           void* d_hidden, float* d_W, int32_t accumulate_dW, cudaStream_t s);

@@ -27,6 +27,7 @@ struct LogprobEpi {
     const int32_t* target;  // [T]
     float4* partial;        // [S, T]
     int T, V;
+    int v_offset;           // vocabulary id of W's first row (0 unless W is one shard of the head)
   };
   struct State {
     float m, s, u, zy;
@@ -35,7 +36,8 @@ struct LogprobEpi {
   static constexpr bool kStaged = false;   // nothing is stored per tile: no staging buffer needed
   static __device__ __forceinline__ void unit_begin(State& st, const Params& p, int row, int, int) {
     st.m = -INFINITY; st.s = 0.f; st.u = 0.f; st.zy = -INFINITY;
-    st.y = row < p.T ? __ldg(p.target + row) : -1;
+    const int y = row < p.T ? __ldg(p.target + row) - p.v_offset : -1;
+    st.y = (y >= 0 && y < p.V) ? y : -1;                          // outside this W's rows: no column matches
   }
   static __device__ __forceinline__ void chunk(State& st, const Params& p, int, int col0,
                                                const uint32_t (&v)[32], uint8_t*) {
@@ -72,10 +74,12 @@ struct LogprobEpi {
   }
 };
 
+// Combines the S partial states of every token.  With `combined` set the result stays a partial
+// state (m, s, u, zy) -- the statistics of one vocabulary shard -- and nothing else is written.
 __global__ void __launch_bounds__(256) merge_partials_kernel(
     const float4* __restrict__ partial, const int32_t* __restrict__ target, int T, int V, int S,
     float* __restrict__ logp, float* __restrict__ entropy, float* __restrict__ lse_out,
-    unsigned int* d_err) {
+    float4* __restrict__ combined, unsigned int* d_err) {
   const int t = blockIdx.x * blockDim.x + threadIdx.x;
   if (t >= T) return;
   float M = -INFINITY;
@@ -88,6 +92,7 @@ __global__ void __launch_bounds__(256) merge_partials_kernel(
     u = fmaf(q.z, w, u);
     zy = fmaxf(zy, q.w);  // exactly one range holds the target; the others report -inf
   }
+  if (combined) { combined[t] = make_float4(M, s, u, zy); return; }
   const float lse = M + kLn2 * log2f(s);
   const int y = __ldg(target + t);
   float lp = zy - lse;
@@ -152,6 +157,37 @@ af_status launch_token_logprob(af_ctx* ctx, const void* hidden, const void* W,
   if (st != AF_OK) return st;
   merge_partials_kernel<<<(int)((T + 255) / 256), 256, 0, s>>>((const float4*)ctx->partial.p, target,
                                                               (int)T, V, S, logp, entropy, lse,
+                                                              nullptr, ctx->d_err);
+  return cudaGetLastError() == cudaSuccess ? AF_OK : AF_ERR_CUDA;
+}
+
+// One vocabulary shard: the same GEMM over the shard's rows of W, the ranges of a token combined
+// into one partial state instead of a final result.
+af_status launch_token_logprob_shard(af_ctx* ctx, const void* hidden, const void* W_shard,
+                                     const int32_t* target, int64_t T, int32_t d, int32_t V_shard,
+                                     int32_t v_offset, float* partial_out, cudaStream_t s) {
+  if (T == 0) return AF_OK;
+  const GemmEnv env = gemm_env(ctx);
+  const int S = logprob_pick_splits(T, d, V_shard, ctx->sm_count, env.pair, ctx->v_splits);
+  af_status st = ws_grow(ctx->partial, (size_t)S * (size_t)T * sizeof(float4));
+  if (st != AF_OK) return st;
+  const Operand Hop{hidden, (uint64_t)T, (uint64_t)d, (uint64_t)d * 2};
+  const Operand Wop{W_shard, (uint64_t)V_shard, (uint64_t)d, (uint64_t)d * 2};
+  LogprobEpi::Params ep{target, (float4*)ctx->partial.p, (int)T, V_shard, v_offset};
+  st = run_gemm<LogprobEpi, false, false>(env, Hop, Wop, S, ep, s);
+  if (st != AF_OK) return st;
+  merge_partials_kernel<<<(int)((T + 255) / 256), 256, 0, s>>>((const float4*)ctx->partial.p, target,
+                                                              (int)T, V_shard, S, nullptr, nullptr, nullptr,
+                                                              reinterpret_cast<float4*>(partial_out), ctx->d_err);
+  return cudaGetLastError() == cudaSuccess ? AF_OK : AF_ERR_CUDA;
+}
+
+af_status launch_merge_logprob_shards(af_ctx* ctx, const float* partials, const int32_t* target, int32_t R,
+                                      int64_t T, int32_t V_total, float* logp, float* entropy, float* lse,
+                                      cudaStream_t s) {
+  if (T == 0) return AF_OK;
+  merge_partials_kernel<<<(int)((T + 255) / 256), 256, 0, s>>>(reinterpret_cast<const float4*>(partials), target,
+                                                              (int)T, V_total, R, logp, entropy, lse, nullptr,
                                                               ctx->d_err);
   return cudaGetLastError() == cudaSuccess ? AF_OK : AF_ERR_CUDA;
 }
@@ -253,6 +289,6 @@ extern "C" af_status af_token_logprob_static(const void* hidden, const void* W, 
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if ((rc = run_gemm<LogprobEpi, false, false>(env, Hop, Wop, S, ep, s)) != AF_OK) return rc;
   merge_partials_kernel<<<(int)((T + 255) / 256), 256, 0, s>>>(partial, target, (int)T, V, S, logp, entropy,
-                                                              lse, err_word);
+                                                              lse, nullptr, err_word);
   return cudaGetLastError() == cudaSuccess ? AF_OK : AF_ERR_CUDA;
 }

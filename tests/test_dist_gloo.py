@@ -1,7 +1,8 @@
 """World-size-2 checks of the data-parallel host logic on CPU (gloo): prompts are split into
 whole groups, rank results concatenate to the single-rank result, bench.py's reduction takes the
 max step time and the token sum over ranks, and the weight gradients of the ranks' batches, each
-scored with loss_scale = B_rank / B_global, sum to the gradient of the global batch."""
+scored with loss_scale = B_rank / B_global, sum to the gradient of the global batch; the
+statistics of vocabulary shards, gathered over the ranks, merge to the full-vocabulary result."""
 import os
 import socket
 
@@ -115,3 +116,30 @@ def test_two_rank_gradient_sum(tmp_path):
     port = _free_port()
     mp.start_processes(_grad_worker, args=(2, port, str(tmp_path)), nprocs=2, join=True, start_method="spawn")
     assert open(tmp_path / "ok_grad").read() == "1"
+
+
+def _vocab_worker(rank, world, port, out_dir):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    import bench
+    w = wl.make_workload("cfg1")
+    H, W, y = wl.bf16_bits(wl.gen_hidden(w)), wl.bf16_bits(wl.gen_weight(w)), wl.gen_target(w).numpy()
+    lo, hi = bench.vocab_shard(w.V, world, rank)
+    mine = torch.from_numpy(O.token_logprob_shard_ref(H, W[lo:hi], y, lo))
+    gathered = bench.allgather_partials(mine, world)                     # [R, T, 4]
+    logp, ent, lse = O.merge_logprob_shards_ref(gathered.numpy())
+    ref = O.token_logprob_ref(H, W, y)
+    ok = all(np.allclose(a, b, atol=1e-12) for a, b in zip((logp, ent, lse), ref))
+    ok = ok and gathered.shape == (world, H.shape[0], 4)
+    los = [bench.vocab_shard(w.V, world, r) for r in range(world)]
+    ok = ok and los[0][0] == 0 and los[-1][1] == w.V and all(a[1] == b[0] for a, b in zip(los[:-1], los[1:]))
+    with open(os.path.join(out_dir, f"ok_vocab_{rank}"), "w") as f:
+        f.write("1" if ok else "0")
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_two_rank_vocabulary_parallel_exchange(tmp_path):
+    port = _free_port()
+    mp.start_processes(_vocab_worker, args=(2, port, str(tmp_path)), nprocs=2, join=True, start_method="spawn")
+    assert open(tmp_path / "ok_vocab_0").read() == "1" and open(tmp_path / "ok_vocab_1").read() == "1"

@@ -250,3 +250,66 @@ def test_reserved_workspace_does_not_grow(ctx):
     ctx.set_tuning(0, 0)
     assert ctx.workspace_bytes() == held
     assert ctx.check_device_errors() == 0
+
+
+@pytest.mark.parametrize("cuts", [[0, 8200], [0, 3000, 8200], [0, 1, 257, 4100, 8199, 8200]])
+def test_vocabulary_shards_merge_to_the_full_result(ctx, cuts):
+    """The head split by vocabulary rows: every shard's statistics against the oracle's, and the
+    merged result against the full-vocabulary oracle and the unsharded call."""
+    dev = device()
+    w = wl.make_workload("cfg2_mini")                       # V = 8200, not a multiple of the tile
+    H, W, y = wl.gen_hidden(w), wl.gen_weight(w), wl.gen_target(w)
+    T = H.shape[0]
+    Hd, Wd, yd = H.to(dev), W.to(dev), y.to(dev)
+    ctx.set_tuning(0, 0, VARIANT)
+    R = len(cuts) - 1
+    partials = torch.full((R, T, 4), 9.0, device=dev)
+    for r, (a, b) in enumerate(zip(cuts[:-1], cuts[1:])):
+        ctx.token_logprob_shard(Hd, Wd[a:b].contiguous(), yd, a, partials[r])
+        ref = O.token_logprob_shard_ref(wl.bf16_bits(H), wl.bf16_bits(W[a:b]), y.numpy(), a)
+        got = np_of(partials[r]).astype(np.float64)
+        assert np.abs(got[:, 0] - ref[:, 0]).max() <= LOGP_TOL                                   # max logit
+        assert np.abs(np.log(got[:, 1]) - np.log(ref[:, 1])).max() <= LOGP_TOL                   # shard normaliser
+        assert np.abs(got[:, 2] / got[:, 1] - ref[:, 2] / ref[:, 1]).max() <= LOGP_TOL          # mean logit
+        inside = np.isfinite(ref[:, 3])
+        assert np.array_equal(np.isfinite(got[:, 3]), inside)
+        assert np.abs(got[inside, 3] - ref[inside, 3]).max(initial=0.0) <= LOGP_TOL
+        assert np.all(got[~inside, 3] == -np.inf)
+    logp, ent, lse = (torch.empty(T, device=dev) for _ in range(3))
+    ctx.merge_logprob_shards(partials, yd, w.V, logp, ent, lse)
+    full = [torch.empty(T, device=dev) for _ in range(3)]
+    ctx.token_logprob(Hd, Wd, yd, *full)
+    flags = ctx.check_device_errors()
+    ctx.set_tuning(0, 0)
+    assert flags == 0
+    r_logp, r_ent, r_lse = O.token_logprob_ref(wl.bf16_bits(H), wl.bf16_bits(W), y.numpy())
+    for got, ref, one in ((logp, r_logp, full[0]), (ent, r_ent, full[1]), (lse, r_lse, full[2])):
+        assert np.abs(np_of(got) - ref).max() <= LOGP_TOL
+        assert np.abs(np_of(got) - np_of(one)).max() <= 1e-4
+    # the merge of the oracle's own shard statistics, fed through the device merge
+    o_parts = np.stack([O.token_logprob_shard_ref(wl.bf16_bits(H), wl.bf16_bits(W[a:b]), y.numpy(), a)
+                        for a, b in zip(cuts[:-1], cuts[1:])]).astype(np.float32)
+    ctx.merge_logprob_shards(torch.as_tensor(o_parts, device=dev), yd, w.V, logp, ent, lse)
+    assert np.abs(np_of(logp) - r_logp).max() <= 1e-4 and np.abs(np_of(ent) - r_ent).max() <= 1e-4
+
+
+def test_shard_argument_errors(ctx):
+    from paper_2507_01663_b200 import binding as B
+    dev = device()
+    H = torch.zeros(4, 16, dtype=torch.bfloat16, device=dev)
+    W = torch.zeros(8, 16, dtype=torch.bfloat16, device=dev)
+    y = torch.zeros(4, dtype=torch.int32, device=dev)
+    part = torch.zeros(1, 4, 4, device=dev)
+    with pytest.raises(B.AfError):
+        ctx.token_logprob_shard(H, W, y, -1, part[0])
+    with pytest.raises(B.AfError):
+        ctx.token_logprob_shard(H, W, y, 0, None)
+    with pytest.raises(B.AfError):
+        ctx.merge_logprob_shards(part, y, 0, torch.zeros(4, device=dev))
+    ctx.merge_logprob_shards(part, y, 8, torch.zeros(4, device=dev), T=0)      # empty batch is a no-op
+    y[1] = 99                                                                  # a global id outside [0, V_total)
+    ctx.token_logprob_shard(H, W, y, 0, part[0])
+    out = torch.zeros(4, device=dev)
+    ctx.merge_logprob_shards(part, y, 8, out)
+    assert ctx.check_device_errors() == B.DEVERR_TARGET_RANGE
+    assert torch.isnan(out[1]) and not torch.isnan(out[0])
