@@ -374,9 +374,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ 
 // ==========================================================================================
 constexpr int kPairBM = 256;                                  // rows of A per pair tile
 constexpr int kPairStages = 6;
-constexpr unsigned int kClockWindow = 1;                      // tiles a pair may start ahead of the slowest pair
+constexpr unsigned int kClockWindow = 1;                      // ticks a pair may start ahead of the slowest pair
+constexpr int kClockTickKBlocks = 64;                         // K blocks per tick when a tile has more than 96
 constexpr unsigned long long kClockPatienceNs = 200000ull;    // longest wait on the tile clock before leaving it,
-constexpr unsigned long long kClockPatiencePerKBlockNs = 2000ull;  // plus this per K block of a tile (~5 tile times)
+constexpr unsigned long long kClockPatiencePerKBlockNs = 2000ull;  // plus this per K block of a tick (~5 tick times)
 constexpr int kPairBBytes = (kBN / 2) * kBK * 2;              // this CTA's half of the B tile
 constexpr int kPairStageBytes = kABytes + kPairBBytes;        // 32 KB
 constexpr int kPairSmemBytes = kPairStages * kPairStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
@@ -485,39 +486,47 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     if (lane == 0) {
       int stage = 0; uint32_t phase = 0; bool ok = true;
       const uint32_t leader_full0 = map_to_cta(full_bar(0), 0);
-      unsigned int my_tiles = 0;                                    // tiles this pair has started
+      // Pacing clock.  Every pair does the same work per K block, so "K blocks issued" measures
+      // progress across pairs; a tick is one tile's worth of K blocks, or kClockTickKBlocks of them
+      // when tiles are long (the backward's products run thousands of K blocks per tile, and pairs
+      // that only met at tile starts drifted far enough apart to lose each other's tiles in L2).
+      // The clock counts ticks over all pairs; a pair starts tick j only when all have started tick
+      // j - kClockWindow.  It is a hint, not a dependency: a pair that waits longer than its patience
+      // (pairs not co-resident, say) leaves the clock for the rest of the launch, counting as
+      // finished so that nobody waits for it.
+      unsigned int my_ticks = 0;
       bool clock_on = tile_clock != nullptr && rank == 0;
-      const unsigned long long patience = kClockPatienceNs + kClockPatiencePerKBlockNs * (unsigned long long)g.k_blocks;
-      // most tiles any pair starts in this launch
-      const unsigned int clock_most = (unsigned int)((total_units + n_pairs - 1) / n_pairs) *
-                                      (unsigned int)((g.n_tiles + g.splits - 1) / g.splits);
+      const int tick_len = g.k_blocks <= 96 ? g.k_blocks : kClockTickKBlocks;
+      int to_next_tick = 0;                                         // K blocks until the next tick
+      const unsigned long long patience = kClockPatienceNs + kClockPatiencePerKBlockNs * (unsigned long long)tick_len;
+      // most ticks any pair starts in this launch
+      const unsigned long long most_kb = (unsigned long long)((total_units + n_pairs - 1) / n_pairs) *
+                                         (unsigned long long)((g.n_tiles + g.splits - 1) / g.splits) *
+                                         (unsigned long long)g.k_blocks;
+      const unsigned int clock_most = (unsigned int)((most_kb + tick_len - 1) / tick_len);
       for (int u = pair; u < total_units && ok; u += n_pairs) {
         const int m_tile = u / g.splits, s = u % g.splits;
         const int nb = split_begin(g, s), ne = split_begin(g, s + 1);
         const int m0 = m_tile * kPairBM + (int)rank * kBM;          // this CTA's 128 rows of A
         for (int nt = nb; nt < ne && ok; ++nt) {
           const int n0 = nt * kBN + (int)rank * (kBN / 2);          // this CTA's 128 rows of B
-          if (clock_on) {
-            // Tile clock: stay within kClockWindow tiles of the slowest pair, so that a B tile
-            // fetched by the first pair is still in L2 when the last one asks for it.  The clock
-            // counts tile starts over all pairs.  It is a pacing hint, not a dependency: a pair
-            // that waits longer than kClockPatienceNs (pairs not co-resident, say) leaves the
-            // clock for the rest of the launch, counting as finished so that nobody waits for it.
-            if (my_tiles >= kClockWindow) {
-              const unsigned int need = (unsigned int)n_pairs * (my_tiles - kClockWindow + 1);
-              const unsigned long long t0 = globaltimer_ns();
-              unsigned int seen;
-              for (;;) {
-                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(tile_clock) : "memory");
-                if (seen >= need) break;
-                if (globaltimer_ns() - t0 > patience) { clock_on = false; break; }
-                __nanosleep(100);
-              }
-            }
-            if (clock_on) { atomicAdd(tile_clock, 1u); ++my_tiles; }
-            else if (clock_most > my_tiles) atomicAdd(tile_clock, clock_most - my_tiles);
-          }
           for (int kb = 0; kb < g.k_blocks; ++kb) {
+            if (clock_on && to_next_tick-- == 0) {
+              to_next_tick = tick_len - 1;
+              if (my_ticks >= kClockWindow) {
+                const unsigned int need = (unsigned int)n_pairs * (my_ticks - kClockWindow + 1);
+                const unsigned long long t0 = globaltimer_ns();
+                unsigned int seen;
+                for (;;) {
+                  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(tile_clock) : "memory");
+                  if (seen >= need) break;
+                  if (globaltimer_ns() - t0 > patience) { clock_on = false; break; }
+                  __nanosleep(100);
+                }
+              }
+              if (clock_on) { atomicAdd(tile_clock, 1u); ++my_ticks; }
+              else if (clock_most > my_ticks) atomicAdd(tile_clock, clock_most - my_ticks);
+            }
             if (!mbar_wait(empty_bar(stage), phase ^ 1u, &abort_flag)) { ok = false; break; }
             const uint32_t a_dst = tiles + stage * kPairStageBytes;
             const uint32_t lbar = leader_full0 + 8u * stage;
@@ -540,8 +549,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
           }
         }
       }
-      // a pair that runs out of work counts as having started every remaining tile
-      if (clock_on && clock_most > my_tiles) atomicAdd(tile_clock, clock_most - my_tiles);
+      // a pair that runs out of work counts as having started every remaining tick
+      if (clock_on && clock_most > my_ticks) atomicAdd(tile_clock, clock_most - my_ticks);
     }
     __syncwarp();
   } else if (warp == 1) {
