@@ -16,15 +16,15 @@
 // row segments, eight rows per instruction.  The dW product is laid out the other way round: its
 // accumulator rows run along d, the contiguous dimension of dW, so 32 lanes holding the same
 // vocabulary row write 128 consecutive bytes without any staging.  That orientation also gives the
-// product the forward's memory behaviour: the H_blk panels (68 MB at the 7B head) stay in L2 and
-// dZ streams through exactly once.
+// product the forward's memory behaviour: the H_blk panels of the row tiles in flight stay in L2
+// while dZ streams past them (once per round of row tiles).
 #include "gemm_launch.cuh"
 
 namespace af {
 namespace {
 
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr int kDefaultTokenBlock = 74 * 128;  // 74 row tiles x 14 column tiles of d = 3584 fill 7 waves of 148 SMs
+constexpr int kDefaultTokenBlock = 74 * 128;  // 37 pair tiles (74 CTA tiles) x 14 column tiles of d = 3584: 7 full rounds of 148 SMs
 
 __device__ __forceinline__ float ex2f(float x) {
   float y;
@@ -208,7 +208,7 @@ af_status launch_backward(af_ctx* ctx, const void* hidden, const void* W, const 
     if (st != AF_OK) return st;
     // 3. dW^T += H_blk^T dZ:  A = H_blk read MN-major (m = d contiguous, K = t rows), B = dZ read
     //    MN-major (n = v contiguous); tile [d, v] stored transposed into dW [V, d].  Vocabulary ranges
-    //    are chosen as in the forward: the H_blk panels stay in L2, dZ streams past once.
+    //    are chosen as in the forward: the H_blk panels in flight stay in L2, dZ streams past them.
     StoreF32TransposedEpi::Params p3{d_W, d, d, V, (!first || accumulate_dW) ? 1 : 0};
     st = run_gemm<StoreF32TransposedEpi, true, true>(env, Hblk, dZop,
                                                      logprob_pick_splits((int64_t)d, (int32_t)tc, V, ctx->sm_count, env.pair, 0),
