@@ -236,3 +236,32 @@ def test_backward_full_size(ctx):
     rhs = float((dH.double() * H.double()).sum())
     scale = float(dW.double().norm() * W.double().norm())
     assert abs(lhs - rhs) <= 2e-3 * scale
+
+
+def test_vocabulary_parallel_head_full_size(ctx):
+    """The 7B head split over two ranks' worth of vocabulary rows at 65536 tokens (the shards are
+    scored one after the other on this GPU): merged result against the unsharded call on every
+    token, and against the oracle on sampled rows."""
+    w = wl.make_workload("cfg4")
+    dev = device()
+    T = w.total_tokens
+    H, y, W = wl.gen_hidden(w, dev), wl.gen_target(w, dev), wl.gen_weight(w, dev)
+    cuts = [0, 76032, w.V]
+    partials = torch.empty(2, T, 4, device=dev)
+    for r in range(2):
+        ctx.token_logprob_shard(H, W[cuts[r]:cuts[r + 1]], y, cuts[r], partials[r])
+    logp, ent, lse = (torch.empty(T, device=dev) for _ in range(3))
+    ctx.merge_logprob_shards(partials, y, w.V, logp, ent, lse)
+    one = [torch.empty(T, device=dev) for _ in range(3)]
+    ctx.token_logprob(H, W, y, *one)
+    assert ctx.check_device_errors() == 0
+    for got, ref in zip((logp, ent, lse), one):
+        assert float((got - ref).abs().max()) <= 1e-4
+    # exactly one shard holds every token's target
+    assert bool((torch.isfinite(partials[:, :, 3]).sum(0) == 1).all())
+    rows = sample_rows(w.tok_offset, T, 64, seed=5)
+    rt = torch.as_tensor(rows, device=dev)
+    o_logp, o_ent, o_lse = oracle_rows(H[rt].cpu(), wl.bf16_bits(W), np_of(y[rt]))
+    assert np.abs(np_of(logp[rt]) - o_logp).max() <= LOGP_TOL
+    assert np.abs(np_of(ent[rt]) - o_ent).max() <= LOGP_TOL
+    assert np.abs(np_of(lse[rt]) - o_lse).max() <= LOGP_TOL
