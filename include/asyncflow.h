@@ -61,8 +61,8 @@ af_status af_destroy(af_ctx* ctx);
 const char* af_status_string(af_status s);
 
 /* Pre-size the workspace for micro-batches of up to max_T tokens and max_B sequences at head
- * shape (d, V).  with_backward != 0 also reserves the scratch of af_policy_loss_backward.
- * Synchronous (allocates). */
+ * shape (d, V).  with_backward != 0 also reserves the scratch of af_policy_loss_backward, and
+ * with_backward == 2 that of af_policy_update too.  Synchronous (allocates). */
 af_status af_reserve(af_ctx* ctx, int64_t max_T, int32_t max_B, int32_t d, int32_t V,
                      int32_t with_backward);
 
@@ -243,6 +243,27 @@ af_status af_policy_loss_backward(af_ctx* ctx, const void* hidden, const void* W
                                   const int32_t* target, const float* lse, const float* dlogp,
                                   int64_t T, int32_t d, int32_t V, void* d_hidden, float* d_W,
                                   int32_t accumulate_dW, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * af_policy_update -- forward, loss and backward of one packed micro-batch in one call (the
+ * forward-backward actor-update task of Section 7.4).
+ *
+ * Computes what af_token_logprob, af_policy_loss and af_policy_loss_backward compute when called
+ * one after the other on the same micro-batch -- logp, entropy, lse [T]; the loss record; dlogp
+ * [T]; d_hidden [T,d] bf16; d_W [V,d] fp32 -- but evaluates the logits once per token instead of
+ * twice: tokens are processed in blocks, a block's fp32 logits stay in scratch between the
+ * log-softmax statistics and dZ, and the per-token loss gradient is taken in between with the
+ * arithmetic of af_policy_loss.  Scratch: one block of logits (fp32) and of dZ (bf16), independent
+ * of T; [T,V] is never materialised.  af_reserve with with_backward = 2 pre-sizes it.
+ * entropy and dlogp may be NULL; every other pointer is required when T > 0.  Requirements and
+ * errors as for the three calls (d % 8 == 0, V % 8 == 0, 16-byte aligned matrices, 0 <= T < 2^31).
+ * ------------------------------------------------------------------------------------------- */
+af_status af_policy_update(af_ctx* ctx, const void* hidden, const void* W, const int32_t* target,
+                           const float* old_logp, const float* ref_logp, const float* adv_seq,
+                           const int32_t* cu_seqlens, int32_t B, int64_t T, int32_t d, int32_t V,
+                           const af_loss_params* params, af_loss_out* out, float* logp, float* entropy,
+                           float* lse, float* dlogp, void* d_hidden, float* d_W, int32_t accumulate_dW,
+                           void* stream);
 
 /* ---------------------------------------------------------------------------------------------
  * af_controller_put / af_controller_get / af_controller_clear -- the status table of the

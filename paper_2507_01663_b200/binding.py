@@ -27,7 +27,7 @@ EXPORTS = ["af_create", "af_destroy", "af_status_string", "af_reserve", "af_work
            "af_set_tuning", "af_check_device_errors", "af_pack_microbatch", "af_token_logprob",
            "af_grpo_advantage", "af_policy_loss", "af_policy_loss_backward", "af_token_logprob_static",
            "af_controller_put", "af_controller_get", "af_controller_clear", "af_balance_partitions",
-           "af_token_logprob_shard", "af_merge_logprob_shards"]
+           "af_token_logprob_shard", "af_merge_logprob_shards", "af_policy_update"]
 
 
 class AfError(RuntimeError):
@@ -110,6 +110,8 @@ def load_library() -> C.CDLL:
     lib.af_balance_partitions.argtypes = [vp, i32, i32, i32, vp, vp]
     lib.af_token_logprob_shard.argtypes = [vp, vp, vp, vp, i64, i32, i32, i32, vp, vp]
     lib.af_merge_logprob_shards.argtypes = [vp, vp, vp, i32, i64, i32, vp, vp, vp, vp]
+    lib.af_policy_update.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i64, i32, i32, C.POINTER(LossParams), vp,
+                                     vp, vp, vp, vp, vp, vp, i32, vp]
     for name in EXPORTS:
         if name not in ("af_status_string", "af_workspace_bytes"):
             getattr(lib, name).restype = C.c_int
@@ -157,7 +159,8 @@ class Context:
             pass
 
     # -- housekeeping ------------------------------------------------------------------------
-    def reserve(self, max_T: int, max_B: int, d: int, V: int, with_backward: bool = False):
+    def reserve(self, max_T: int, max_B: int, d: int, V: int, with_backward=False):
+        """with_backward: False / True (backward scratch) / 2 (also the fused update's)."""
         _check(self.lib.af_reserve(self.handle, max_T, max_B, d, V, int(with_backward)), "af_reserve")
 
     def workspace_bytes(self) -> int:
@@ -248,6 +251,19 @@ class Context:
                                                 _ptr(d_W), int(accumulate_dW), _stream(stream)),
                "af_policy_loss_backward")
 
+
+    def policy_update(self, hidden, W, target, old_logp, ref_logp, adv_seq, cu_seqlens, out, logp, lse, d_hidden,
+                      d_W, entropy=None, dlogp=None, accumulate_dW=False, clip_lo=0.2, clip_hi=0.2, kl_coef=0.04,
+                      agg_mode=0, loss_scale=1.0, B=None, T=None, stream=None):
+        """``af_policy_update``: forward + loss + backward of one packed micro-batch in one call."""
+        B = cu_seqlens.shape[0] - 1 if B is None else B
+        T = hidden.shape[0] if T is None else T
+        d, V = W.shape[1], W.shape[0]
+        prm = LossParams(clip_lo, clip_hi, kl_coef, agg_mode, loss_scale)
+        _check(self.lib.af_policy_update(self.handle, _ptr(hidden), _ptr(W), _ptr(target), _ptr(old_logp),
+                                         _ptr(ref_logp), _ptr(adv_seq), _ptr(cu_seqlens), B, T, d, V, C.byref(prm),
+                                         _ptr(out), _ptr(logp), _ptr(entropy), _ptr(lse), _ptr(dlogp), _ptr(d_hidden),
+                                         _ptr(d_W), int(accumulate_dW), _stream(stream)), "af_policy_update")
 
     # -- controller: status table of the streaming store ----------------------------------------
     @staticmethod

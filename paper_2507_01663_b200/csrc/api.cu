@@ -94,7 +94,7 @@ af_status af_destroy(af_ctx* c) {
   if (!c) return AF_ERR_INVALID_ARG;
   DeviceGuard guard(c->device);
   cudaDeviceSynchronize();
-  Buf* bufs[] = {&c->partial, &c->loss_ws, &c->pack_meta, &c->dz, &c->ctrl_ws};
+  Buf* bufs[] = {&c->partial, &c->loss_ws, &c->pack_meta, &c->dz, &c->ctrl_ws, &c->zlog};
   for (Buf* b : bufs) if (b->p) cudaFree(b->p);
   for (int i = 0; i < kPackRing; ++i) {
     if (c->pack_host[i]) cudaFreeHost(c->pack_host[i]);
@@ -107,7 +107,7 @@ af_status af_destroy(af_ctx* c) {
 
 int64_t af_workspace_bytes(const af_ctx* c) {
   if (!c) return 0;
-  return (int64_t)(c->partial.cap + c->loss_ws.cap + c->pack_meta.cap + c->dz.cap + c->ctrl_ws.cap);
+  return (int64_t)(c->partial.cap + c->loss_ws.cap + c->pack_meta.cap + c->dz.cap + c->ctrl_ws.cap + c->zlog.cap);
 }
 
 af_status af_set_tuning(af_ctx* c, int32_t v_splits, int32_t bwd_token_block, int32_t gemm_variant) {
@@ -162,6 +162,12 @@ af_status af_reserve(af_ctx* c, int64_t max_T, int32_t max_B, int32_t d, int32_t
     // sizes are recomputed (and grown if needed) by the backward call itself
     st = launch_backward(c, nullptr, nullptr, nullptr, nullptr, nullptr, max_T, d, V, nullptr, nullptr,
                          -1 /* reserve only */, nullptr);
+  }
+  if (st == AF_OK && with_backward == 2) {
+    af_loss_params none{};
+    st = launch_policy_update(c, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, 0, max_T, d, V, none,
+                              nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, -1 /* reserve only */,
+                              nullptr);
   }
   return st;
 }
@@ -321,6 +327,24 @@ af_status af_policy_loss_backward(af_ctx* c, const void* hidden, const void* W, 
 
 static bool table_ok(const af_controller_view* t) {
   return t && t->n_samples >= 0 && (t->n_samples == 0 || (t->ready && t->consumed));
+}
+
+af_status af_policy_update(af_ctx* c, const void* hidden, const void* W, const int32_t* target,
+                           const float* old_logp, const float* ref_logp, const float* adv_seq,
+                           const int32_t* cu_seqlens, int32_t B, int64_t T, int32_t d, int32_t V,
+                           const af_loss_params* params, af_loss_out* out, float* logp, float* entropy, float* lse,
+                           float* dlogp, void* d_hidden, float* d_W, int32_t accumulate_dW, void* stream) {
+  if (!c || !params || !out || !cu_seqlens || B < 0 || T < 0 || d < 1 || V < 1 || !d_W) return AF_ERR_INVALID_ARG;
+  if (T > 0 && (!hidden || !W || !target || !old_logp || !ref_logp || !adv_seq || !logp || !lse || !d_hidden || B < 1))
+    return AF_ERR_INVALID_ARG;
+  if (params->agg_mode != 0 && params->agg_mode != 1) return AF_ERR_INVALID_ARG;
+  if (T > ((int64_t)1 << 31) - 65536) return AF_ERR_SHAPE;
+  if (d % 8 != 0 || V % 8 != 0) return AF_ERR_ALIGNMENT;
+  if (!aligned16(hidden) || !aligned16(W) || !aligned16(d_hidden) || !aligned16(d_W)) return AF_ERR_ALIGNMENT;
+  DeviceGuard guard(c->device);
+  return launch_policy_update(c, hidden, W, target, old_logp, ref_logp, adv_seq, cu_seqlens, B, T, d, V, *params, out,
+                              logp, entropy, lse, dlogp, d_hidden, d_W, accumulate_dW ? 1 : 0,
+                              static_cast<cudaStream_t>(stream));
 }
 
 af_status af_controller_put(af_ctx* c, const af_controller_view* table, const int32_t* idx, int64_t n,

@@ -171,13 +171,41 @@ struct StoreF32TransposedEpi {
 
 }  // namespace
 
-af_status launch_backward(af_ctx* ctx, const void* hidden, const void* W, const int32_t* target,
-                          const float* lse, const float* dlogp, int64_t T, int32_t d, int32_t V,
-                          void* d_hidden, float* d_W, int32_t accumulate_dW, cudaStream_t s) {
+// The two products that consume a block of dZ [tc, V] (bf16):
+//   dH_blk = dZ W:        A = dZ (K = v contiguous), B = W read MN-major (n = d contiguous, K = v rows)
+//   dW^T  += H_blk^T dZ:  A = H_blk read MN-major (m = d contiguous, K = t rows), B = dZ read MN-major
+//                         (n = v contiguous); tile [d, v] stored transposed into dW [V, d].  Vocabulary
+//                         ranges are chosen as in the forward: the H_blk panels in flight stay in L2, dZ
+//                         streams past them.
+af_status launch_backward_products(af_ctx* ctx, const void* hidden_blk, const void* W, const void* dz_blk,
+                                   int64_t tc, int32_t d, int32_t V, void* d_hidden_blk, float* d_W,
+                                   int32_t accumulate_dW, cudaStream_t s) {
+  const GemmEnv env = gemm_env(ctx);
+  const uint64_t dB = (uint64_t)d * 2, vB = (uint64_t)V * 2;
+  const Operand Hblk{hidden_blk, (uint64_t)tc, (uint64_t)d, dB};
+  const Operand Wop{W, (uint64_t)V, (uint64_t)d, dB};
+  const Operand dZop{dz_blk, (uint64_t)tc, (uint64_t)V, vB};
+  StoreBf16Epi::Params p2{static_cast<__nv_bfloat16*>(d_hidden_blk), d, (int)tc, d};
+  af_status st = run_gemm<StoreBf16Epi, false, true>(env, dZop, Wop, 0, p2, s);
+  if (st != AF_OK) return st;
+  StoreF32TransposedEpi::Params p3{d_W, d, d, V, accumulate_dW ? 1 : 0};
+  return run_gemm<StoreF32TransposedEpi, true, true>(env, Hblk, dZop,
+                                                     logprob_pick_splits((int64_t)d, (int32_t)tc, V, ctx->sm_count, env.pair, 0),
+                                                     p3, s);
+}
+
+// Token block of the backward (and of the fused update): a multiple of 128 rows.
+int64_t backward_token_block(const af_ctx* ctx, int64_t T) {
   int64_t Tc = ctx->bwd_token_block > 0 ? ctx->bwd_token_block : kDefaultTokenBlock;
   const int64_t T_round = ((T + 127) / 128) * 128;
   if (Tc > T_round) Tc = T_round > 0 ? T_round : 128;
+  return Tc;
+}
 
+af_status launch_backward(af_ctx* ctx, const void* hidden, const void* W, const int32_t* target,
+                          const float* lse, const float* dlogp, int64_t T, int32_t d, int32_t V,
+                          void* d_hidden, float* d_W, int32_t accumulate_dW, cudaStream_t s) {
+  const int64_t Tc = backward_token_block(ctx, T);
   const GemmEnv env = gemm_env(ctx);
   af_status st;
   if ((st = ws_grow(ctx->dz, (size_t)Tc * V * 2)) != AF_OK) return st;
@@ -189,30 +217,21 @@ af_status launch_backward(af_ctx* ctx, const void* hidden, const void* W, const 
   }
   const __nv_bfloat16* H = static_cast<const __nv_bfloat16*>(hidden);
   __nv_bfloat16* dz = static_cast<__nv_bfloat16*>(ctx->dz.p);
-  const uint64_t dB = (uint64_t)d * 2, vB = (uint64_t)V * 2;
+  const uint64_t dB = (uint64_t)d * 2;
 
   bool first = true;
   for (int64_t t0 = 0; t0 < T; t0 += Tc, first = false) {
     const uint64_t tc = (uint64_t)((T - t0) < Tc ? (T - t0) : Tc);
     const Operand Hblk{H + t0 * d, tc, (uint64_t)d, dB};
     const Operand Wop{W, (uint64_t)V, (uint64_t)d, dB};
-    const Operand dZop{dz, tc, (uint64_t)V, vB};
     // 1. dZ block:  Z = H_blk W^T, both K-major
     DzEpi::Params p1{target + t0, lse + t0, dlogp + t0, dz, (int)tc, V};
     st = run_gemm<DzEpi, false, false>(env, Hblk, Wop,
                                        logprob_pick_splits((int64_t)tc, d, V, ctx->sm_count, env.pair, ctx->v_splits), p1, s);
     if (st != AF_OK) return st;
-    // 2. dH block = dZ W:  A = dZ (K = v contiguous), B = W read MN-major (n = d contiguous, K = v rows)
-    StoreBf16Epi::Params p2{static_cast<__nv_bfloat16*>(d_hidden) + t0 * d, d, (int)tc, d};
-    st = run_gemm<StoreBf16Epi, false, true>(env, dZop, Wop, 0, p2, s);
-    if (st != AF_OK) return st;
-    // 3. dW^T += H_blk^T dZ:  A = H_blk read MN-major (m = d contiguous, K = t rows), B = dZ read
-    //    MN-major (n = v contiguous); tile [d, v] stored transposed into dW [V, d].  Vocabulary ranges
-    //    are chosen as in the forward: the H_blk panels in flight stay in L2, dZ streams past them.
-    StoreF32TransposedEpi::Params p3{d_W, d, d, V, (!first || accumulate_dW) ? 1 : 0};
-    st = run_gemm<StoreF32TransposedEpi, true, true>(env, Hblk, dZop,
-                                                     logprob_pick_splits((int64_t)d, (int32_t)tc, V, ctx->sm_count, env.pair, 0),
-                                                     p3, s);
+    st = launch_backward_products(ctx, H + t0 * d, W, dz, (int64_t)tc, d, V,
+                                  static_cast<__nv_bfloat16*>(d_hidden) + t0 * d, d_W,
+                                  (!first || accumulate_dW) ? 1 : 0, s);
     if (st != AF_OK) return st;
   }
   return AF_OK;

@@ -43,6 +43,7 @@ struct af_ctx {
   af::Buf pack_meta;  // per-call sequence table of af_pack_microbatch
   af::Buf dz;         // dZ [Tc, V] bf16 (backward, one token block)
   af::Buf ctrl_ws;    // per-block aggregates of af_controller_get
+  af::Buf zlog;       // fp32 logits [Tc, V] of one token block (fused actor update)
 
   // pinned staging ring for pack metadata
   void* pack_host[af::kPackRing] = {};
@@ -102,6 +103,20 @@ af_status launch_token_logprob_shard(af_ctx* ctx, const void* hidden, const void
 af_status launch_merge_logprob_shards(af_ctx* ctx, const float* partials, const int32_t* target, int32_t R,
                                       int64_t T, int32_t V_total, float* logp, float* entropy, float* lse,
                                       cudaStream_t s);
+
+af_status launch_token_logprob_z(af_ctx* ctx, const void* hidden, const void* W,
+                                 const int32_t* target, int64_t T, int32_t d, int32_t V,
+                                 float* logp, float* entropy, float* lse, float* z, cudaStream_t s);
+int64_t backward_token_block(const af_ctx* ctx, int64_t T);
+af_status launch_backward_products(af_ctx* ctx, const void* hidden_blk, const void* W, const void* dz_blk,
+                                   int64_t tc, int32_t d, int32_t V, void* d_hidden_blk, float* d_W,
+                                   int32_t accumulate_dW, cudaStream_t s);
+af_status launch_policy_update(af_ctx* ctx, const void* hidden, const void* W, const int32_t* target,
+                               const float* old_logp, const float* ref_logp, const float* adv_seq,
+                               const int32_t* cu_seqlens, int32_t B, int64_t T, int32_t d, int32_t V,
+                               const af_loss_params& params, af_loss_out* out, float* logp, float* entropy,
+                               float* lse, float* dlogp, void* d_hidden, float* d_W, int32_t accumulate_dW,
+                               cudaStream_t s);
 
 af_status launch_backward(af_ctx* ctx, const void* hidden, const void* W, const int32_t* target,
                           const float* lse, const float* dlogp, int64_t T, int32_t d, int32_t V,

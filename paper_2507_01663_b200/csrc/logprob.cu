@@ -22,12 +22,17 @@ __device__ __forceinline__ float ex2f(float x) {
   return y;
 }
 
-struct LogprobEpi {
+// kStoreZ: also write the fp32 logits of the tile to z [T, ldz] (one token block of the fused actor
+// update, which turns them into dZ without a second GEMM).
+template <bool kStoreZ>
+struct LogprobEpiT {
   struct Params {
     const int32_t* target;  // [T]
     float4* partial;        // [S, T]
     int T, V;
     int v_offset;           // vocabulary id of W's first row (0 unless W is one shard of the head)
+    float* z;               // [T, ldz] fp32 logits (kStoreZ only)
+    int64_t ldz;
   };
   struct State {
     float m, s, u, zy;
@@ -39,12 +44,26 @@ struct LogprobEpi {
     const int y = row < p.T ? __ldg(p.target + row) - p.v_offset : -1;
     st.y = (y >= 0 && y < p.V) ? y : -1;                          // outside this W's rows: no column matches
   }
-  static __device__ __forceinline__ void chunk(State& st, const Params& p, int, int col0,
+  static __device__ __forceinline__ void chunk(State& st, const Params& p, int row, int col0,
                                                const uint32_t (&v)[32], uint8_t*) {
     if (col0 >= p.V) return;
     float z[32];
 #pragma unroll
     for (int j = 0; j < 32; ++j) z[j] = __uint_as_float(v[j]);
+    if constexpr (kStoreZ) {
+      // a lane owns one row: eight 16-byte stores fill one 128-byte line of that row
+      if (row < p.T) {
+        float* dst = p.z + (size_t)row * p.ldz + col0;
+        if (col0 + 32 <= p.V) {
+#pragma unroll
+          for (int q = 0; q < 8; ++q)
+            reinterpret_cast<float4*>(dst)[q] = make_float4(z[4 * q], z[4 * q + 1], z[4 * q + 2], z[4 * q + 3]);
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) if (col0 + j < p.V) dst[j] = z[j];
+        }
+      }
+    }
     if (col0 + 32 > p.V) {  // ragged vocabulary tail: columns >= V hold zero-fill, not logits
 #pragma unroll
       for (int j = 0; j < 32; ++j) if (col0 + j >= p.V) z[j] = -1.0e30f;
@@ -73,6 +92,7 @@ struct LogprobEpi {
     if (row < p.T) p.partial[(size_t)split * p.T + row] = make_float4(st.m, st.s, st.u, st.zy);
   }
 };
+using LogprobEpi = LogprobEpiT<false>;
 
 // Combines the S partial states of every token.  With `combined` set the result stays a partial
 // state (m, s, u, zy) -- the statistics of one vocabulary shard -- and nothing else is written.
@@ -142,9 +162,9 @@ int logprob_pick_splits(int64_t T, int32_t d, int32_t V, int sm_count, bool pair
   return best;
 }
 
-af_status launch_token_logprob(af_ctx* ctx, const void* hidden, const void* W,
-                               const int32_t* target, int64_t T, int32_t d, int32_t V,
-                               float* logp, float* entropy, float* lse, cudaStream_t s) {
+af_status launch_token_logprob_z(af_ctx* ctx, const void* hidden, const void* W,
+                                 const int32_t* target, int64_t T, int32_t d, int32_t V,
+                                 float* logp, float* entropy, float* lse, float* z, cudaStream_t s) {
   if (T == 0) return AF_OK;
   const GemmEnv env = gemm_env(ctx);
   const int S = logprob_pick_splits(T, d, V, ctx->sm_count, env.pair, ctx->v_splits);
@@ -152,13 +172,24 @@ af_status launch_token_logprob(af_ctx* ctx, const void* hidden, const void* W,
   if (st != AF_OK) return st;
   const Operand Hop{hidden, (uint64_t)T, (uint64_t)d, (uint64_t)d * 2};
   const Operand Wop{W, (uint64_t)V, (uint64_t)d, (uint64_t)d * 2};
-  LogprobEpi::Params ep{target, (float4*)ctx->partial.p, (int)T, V};
-  st = run_gemm<LogprobEpi, false, false>(env, Hop, Wop, S, ep, s);
+  if (z) {
+    LogprobEpiT<true>::Params ep{target, (float4*)ctx->partial.p, (int)T, V, 0, z, (int64_t)V};
+    st = run_gemm<LogprobEpiT<true>, false, false>(env, Hop, Wop, S, ep, s);
+  } else {
+    LogprobEpi::Params ep{target, (float4*)ctx->partial.p, (int)T, V, 0, nullptr, 0};
+    st = run_gemm<LogprobEpi, false, false>(env, Hop, Wop, S, ep, s);
+  }
   if (st != AF_OK) return st;
   merge_partials_kernel<<<(int)((T + 255) / 256), 256, 0, s>>>((const float4*)ctx->partial.p, target,
                                                               (int)T, V, S, logp, entropy, lse,
                                                               nullptr, ctx->d_err);
   return cudaGetLastError() == cudaSuccess ? AF_OK : AF_ERR_CUDA;
+}
+
+af_status launch_token_logprob(af_ctx* ctx, const void* hidden, const void* W,
+                               const int32_t* target, int64_t T, int32_t d, int32_t V,
+                               float* logp, float* entropy, float* lse, cudaStream_t s) {
+  return launch_token_logprob_z(ctx, hidden, W, target, T, d, V, logp, entropy, lse, nullptr, s);
 }
 
 // One vocabulary shard: the same GEMM over the shard's rows of W, the ranges of a token combined
@@ -173,7 +204,7 @@ af_status launch_token_logprob_shard(af_ctx* ctx, const void* hidden, const void
   if (st != AF_OK) return st;
   const Operand Hop{hidden, (uint64_t)T, (uint64_t)d, (uint64_t)d * 2};
   const Operand Wop{W_shard, (uint64_t)V_shard, (uint64_t)d, (uint64_t)d * 2};
-  LogprobEpi::Params ep{target, (float4*)ctx->partial.p, (int)T, V_shard, v_offset};
+  LogprobEpi::Params ep{target, (float4*)ctx->partial.p, (int)T, V_shard, v_offset, nullptr, 0};
   st = run_gemm<LogprobEpi, false, false>(env, Hop, Wop, S, ep, s);
   if (st != AF_OK) return st;
   merge_partials_kernel<<<(int)((T + 255) / 256), 256, 0, s>>>((const float4*)ctx->partial.p, target,
@@ -285,7 +316,7 @@ extern "C" af_status af_token_logprob_static(const void* hidden, const void* W, 
   const GemmEnv env{g_static_encode, st->sm_count, err_word, false, nullptr};
   const Operand Hop{hidden, (uint64_t)T, (uint64_t)d, (uint64_t)d * 2};
   const Operand Wop{W, (uint64_t)V, (uint64_t)d, (uint64_t)d * 2};
-  LogprobEpi::Params ep{target, partial, (int)T, V};
+  LogprobEpi::Params ep{target, partial, (int)T, V, 0, nullptr, 0};
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if ((rc = run_gemm<LogprobEpi, false, false>(env, Hop, Wop, S, ep, s)) != AF_OK) return rc;
   merge_partials_kernel<<<(int)((T + 255) / 256), 256, 0, s>>>(partial, target, (int)T, V, S, logp, entropy,

@@ -19,7 +19,7 @@
 // and the last block to finish adds them in a fixed order -- no float atomics, so results are
 // bit-reproducible.  Buffers that are not 16-byte aligned, and the last 1-3 tokens of a batch
 // whose length is not a multiple of 4, are read with plain loads instead.
-#include "common.cuh"
+#include "loss_math.cuh"
 #include "umma.cuh"
 
 namespace af {
@@ -44,13 +44,7 @@ __device__ __forceinline__ double* ws_partial(LossWs* ws, int block) {
   return reinterpret_cast<double*>(ws + 1) + (size_t)block * kNumSums;
 }
 
-constexpr float kLog2e = 1.4426950408889634f;
 
-__device__ __forceinline__ float ex2f(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
 __device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void* src, uint32_t bytes, uint32_t bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                :: "r"(dst_smem), "l"(src), "r"(bytes), "r"(bar) : "memory");
@@ -104,8 +98,7 @@ __global__ void __launch_bounds__(kThreads, 2) policy_loss_kernel(
   auto full_bar = [&](int st) { return bars + 8u * st; };
   auto empty_bar = [&](int st) { return bars + 8u * (kStages + st); };
   const float lo_b = 1.f - prm.clip_lo, hi_b = 1.f + prm.clip_hi;
-  const float w_all = prm.agg_mode == 0 ? (B > 0 ? prm.loss_scale / (float)B : 0.f)
-                                        : (T > 0 ? prm.loss_scale / (float)T : 0.f);
+  const float w_all = lossmath::batch_weight(prm, B, T);
   const float nbeta = -prm.kl_coef;
   float acc_pg = 0.f, acc_kl = 0.f, acc_ent = 0.f;
   int acc_clip = 0;
@@ -229,7 +222,7 @@ __global__ void __launch_bounds__(kThreads, 2) policy_loss_kernel(
       }
       const int j_max = staged ? j0 + nw - 2 : B - 1;   // last sequence this thread may step to
       float A = staged ? s_adv[j - j0] : __ldg(adv_seq + j);
-      float inv_len = prm.agg_mode == 0 ? __frcp_rn((float)(seq_end - seq_beg)) : 1.f;
+      float inv_len = lossmath::inv_length(prm, seq_end - seq_beg);
       float run_pg = 0.f, run_kl = 0.f;
 #pragma unroll
       for (int k = 0; k < kTokPerThread; ++k) {
@@ -244,19 +237,14 @@ __global__ void __launch_bounds__(kThreads, 2) policy_loss_kernel(
               seq_end = staged ? s_win[j - j0 + 1] : __ldg(cu + j + 1);
             }
             A = staged ? s_adv[j - j0] : __ldg(adv_seq + j);
-            inv_len = prm.agg_mode == 0 ? __frcp_rn((float)(seq_end - seq_beg)) : 1.f;
+            inv_len = lossmath::inv_length(prm, seq_end - seq_beg);
           }
-          const float rho = ex2f((lp[k] - ol[k]) * kLog2e);
-          const float s1 = rho * A;
-          const float s2 = fminf(fmaxf(rho, lo_b), hi_b) * A;
-          const bool clipped = s2 < s1;
-          const float delta = rf[k] - lp[k];
-          const float em1 = ex2f(delta * kLog2e) - 1.f;   // exactly 0 when ref == logp
-          run_pg -= fminf(s1, s2);
-          run_kl += em1 - delta;
+          const lossmath::TokenTerms tt = lossmath::token_terms(lp[k], ol[k], rf[k], A, lo_b, hi_b, nbeta);
+          run_pg += tt.pg;
+          run_kl += tt.k3;
           acc_ent += en[k];
-          acc_clip += clipped ? 1 : 0;
-          g[k] = (w_all * inv_len) * fmaf(nbeta, em1, clipped ? 0.f : -s1);
+          acc_clip += tt.clipped ? 1 : 0;
+          g[k] = (w_all * inv_len) * tt.grad;
         }
       }
       acc_pg += run_pg * inv_len; acc_kl += run_kl * inv_len;
