@@ -210,7 +210,7 @@ class ScoringJob:
         if w.backward:
             self.d_hidden = torch.empty(cap_T, w.d, dtype=torch.bfloat16, device=device)
             self.d_W = torch.empty(w.V, w.d, device=device)
-        self.ctx.reserve(cap_T, cap_B, w.d, w.V, with_backward=w.backward)
+        self.ctx.reserve(cap_T, cap_B, w.d, w.V, with_backward=2 if w.backward else False)
         self.gemm_events, self.pack_events, self.bwd_events = [], [], []
         per_mb = KERNELS_PER_STEP - 1 + (3 * -(-cap_T // BWD_TOKEN_BLOCK) if w.backward else 0)
         self.launches_per_step = 1 + per_mb * len(self.mbs)
@@ -342,6 +342,24 @@ class ScoringJob:
                 "token_spread_equal_counts": int(sums.max() - sums.min()),
                 "token_spread_free_counts": int(sums_pp.max() - sums_pp.min()),
                 "mean_tokens_per_group": float(sums.mean())}
+
+    # -- actor update in one call ------------------------------------------------------------
+    def step_fused_update(self):
+        """advantage -> pack -> af_policy_update (forward + loss + backward, logits evaluated once)."""
+        w, c = self.w, self.ctx
+        c.grpo_advantage(self.reward, None, w.n_prompts, self.adv)
+        store = {"tok_offset_host": self.off, "d": w.d, "adv": self.adv, **self.store}
+        total = 0
+        for mb, loss_out in zip(self.mbs, self.loss_outs):
+            T = c.pack_microbatch(store, mb, self.packed)
+            c.policy_update(self.packed["hidden"], self.W, self.packed["target"], self.packed["old_logp"],
+                            self.packed["ref_logp"], self.packed["adv_seq"], self.packed["cu_seqlens"], loss_out,
+                            self.logp, self.lse, self.d_hidden, self.d_W, entropy=self.ent, dlogp=self.dlogp,
+                            clip_lo=w.clip_eps, clip_hi=w.clip_eps, kl_coef=w.kl_coef, loss_scale=1.0 / self.world,
+                            B=len(mb), T=T)
+            allreduce_sum_(self.d_W, self.world)
+            total += T
+        return total
 
     # -- delayed parameter update: new weights arrive while scoring goes on -----------------
     def make_weight_refresh(self):
@@ -507,6 +525,18 @@ def run_ours(args):
     ms_e2e_total = timed_loop(job.step_e2e, args.steps, world)
     ms_e2e, _ = reduce_over_ranks(ms_e2e_total / args.steps, job.T, world)
 
+    fused = None
+    if w.backward:
+        for _ in range(2):
+            job.step_fused_update()
+        ms_f_total = timed_loop(job.step_fused_update, args.steps, world)
+        ms_f, _ = reduce_over_ranks(ms_f_total / args.steps, job.T, world)
+        loss_f = job.B.read_loss_out(job.loss_out)["loss"]
+        fused = {"value": tokens / (ms_f * 1e-3), "unit": UNIT, "ms_per_step": ms_f, "loss": loss_f,
+                 "tflops_6TdV_model": 6.0 * job.T * w.d * w.V / (ms_f * 1e-3) / 1e12,
+                 "what": "the same step through af_policy_update: forward, loss and backward in one call, the "
+                         "logits evaluated once per token (6 T d V products instead of 8)"}
+
     refresh = None
     if args.weight_refresh and not w.backward:
         job.make_weight_refresh()
@@ -556,6 +586,8 @@ def run_ours(args):
                                                        "where": "inside the timed steps (all micro-batches of a step), "
                                                                 "each right after a GEMM (part at its power cap)"}}
     line["hbm_kernels"].update(hbm_alone)
+    if fused is not None:
+        line["fused_update"] = fused
     if refresh is not None:
         line["weight_refresh"] = refresh
     if rank == 0:

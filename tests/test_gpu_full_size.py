@@ -265,3 +265,48 @@ def test_vocabulary_parallel_head_full_size(ctx):
     assert np.abs(np_of(logp[rt]) - o_logp).max() <= LOGP_TOL
     assert np.abs(np_of(ent[rt]) - o_ent).max() <= LOGP_TOL
     assert np.abs(np_of(lse[rt]) - o_lse).max() <= LOGP_TOL
+
+
+def test_fused_update_full_size(ctx):
+    """cfg4 through af_policy_update against the same micro-batch through the three separate
+    calls (which the tests above tie to the oracle): log-probs, loss record and dlogp agree to
+    fp32 rounding, the gradients within the bf16 rounding of dZ."""
+    from paper_2507_01663_b200 import binding as B
+    w = wl.make_workload("cfg4")
+    dev = device()
+    T = w.total_tokens
+    store, W, reward = build_store(w, dev)
+    H, y, old, ref = store["hidden"], store["target"], store["old_logp"], store["ref_logp"]
+    adv = torch.empty(w.N, device=dev)
+    ctx.grpo_advantage(reward, None, w.n_prompts, adv)
+    cu = torch.as_tensor(w.tok_offset.astype(np.int32), device=dev)
+    # three calls
+    logp, ent, lse, g = (torch.empty(T, device=dev) for _ in range(4))
+    lo = B.new_loss_out(dev)
+    ctx.token_logprob(H, W, y, logp, ent, lse)
+    ctx.policy_loss(logp, old, ref, adv, cu, lo, g, ent, w.clip_eps, w.clip_eps, w.kl_coef)
+    dH = torch.empty(T, w.d, dtype=torch.bfloat16, device=dev)
+    dW = torch.empty(w.V, w.d, device=dev)
+    ctx.policy_loss_backward(H, W, y, lse, g, dH, dW)
+    res = B.read_loss_out(lo)
+    # one call
+    logp2, ent2, lse2, g2 = (torch.empty(T, device=dev) for _ in range(4))
+    lo2 = B.new_loss_out(dev)
+    dH2 = torch.empty_like(dH)
+    dW2 = torch.empty_like(dW)
+    ctx.policy_update(H, W, y, old, ref, adv, cu, lo2, logp2, lse2, dH2, dW2, entropy=ent2, dlogp=g2,
+                      clip_lo=w.clip_eps, clip_hi=w.clip_eps, kl_coef=w.kl_coef)
+    res2 = B.read_loss_out(lo2)
+    assert ctx.check_device_errors() == 0
+    assert float((logp2 - logp).abs().max()) <= 1e-4 and float((lse2 - lse).abs().max()) <= 1e-4
+    assert float((ent2 - ent).abs().max()) <= 1e-4
+    for k in ("loss", "pg_loss", "kl_mean", "entropy_mean"):
+        assert rel(res2[k], res[k]) <= 1e-4, k
+    assert res2["n_tokens"] == T
+    assert float((g2 - g).abs().max()) <= 1e-3 * float(g.abs().max())
+    assert float((dW2 - dW).norm() / dW.norm()) <= 2e-3
+    assert float((dH2.float() - dH.float()).norm() / dH.float().norm()) <= 2e-3
+    # trace identity over the whole fused result: <dW, W> = <dH, H> up to bf16 rounding
+    lhs = float((dW2.double() * W.double()).sum())
+    rhs = float((dH2.double() * H.double()).sum())
+    assert abs(lhs - rhs) <= 2e-3 * float(dW2.double().norm() * W.double().norm())
