@@ -168,11 +168,11 @@ class ScoringJob:
     """Device buffers of one rank and the step function that runs the path through the C ABI."""
 
     def __init__(self, w: wl.Workload, device: torch.device, gemm_variant: int = 0, world: int = 1, v_splits: int = 0,
-                 vocab_parallel: bool = False, rank: int = 0):
+                 vocab_parallel: bool = False, rank: int = 0, bwd_token_block: int = 0):
         from paper_2507_01663_b200 import binding as B
         self.B, self.w, self.dev, self.world = B, w, device, world
         self.ctx = B.Context(device.index or 0)
-        self.ctx.set_tuning(v_splits, 0, gemm_variant)
+        self.ctx.set_tuning(v_splits, bwd_token_block, gemm_variant)
         T = w.total_tokens
         self.T = T
         self.store = {
@@ -446,16 +446,17 @@ def timed_loop(fn, steps: int, world: int):
         import torch.distributed as dist
         dist.barrier()
     torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(steps):
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    marks[0].record()
+    for i in range(steps):
         fn()
-    e1.record()
+        marks[i + 1].record()
     torch.cuda.synchronize()
     if world > 1:
         import torch.distributed as dist
         dist.barrier()
-    return e0.elapsed_time(e1)
+    timed_loop.last_steps_ms = [marks[i].elapsed_time(marks[i + 1]) for i in range(steps)]
+    return marks[0].elapsed_time(marks[-1])
 
 
 def cpu_oracle_sample(w: wl.Workload, hidden_rows: torch.Tensor, W_bits: np.ndarray, target_rows: np.ndarray,
@@ -494,7 +495,7 @@ def run_ours(args):
     # data parallel: every rank its own batch; vocabulary parallel: one batch, the head split by rows
     w = rank_workload(args.workload, 0 if args.vocab_parallel else rank)
     job = ScoringJob(w, dev, {"default": 0, "single": 1, "pair": 2}[args.gemm], world, args.v_splits,
-                     args.vocab_parallel, rank)
+                     args.vocab_parallel, rank, args.bwd_token_block)
     peaks = measured_peaks()
     hbm_alone = job.hbm_kernels_at_scale(peaks["hbm_gbs"]) if rank == 0 and world == 1 else {}
 
@@ -506,6 +507,7 @@ def run_ours(args):
         sampler.start()
     ms_total = timed_loop(lambda: job.step(time_gemm=True), args.steps, world)
     clocks = sampler.stop() if rank == 0 else None
+    steps_ms = list(timed_loop.last_steps_ms)
     # per step: summed over the step's micro-batches
     gemm_ms = float(np.sum([a.elapsed_time(b) for a, b in job.gemm_events])) / args.steps
     pack_ms = float(np.sum([a.elapsed_time(b) for a, b in job.pack_events])) / args.steps
@@ -554,7 +556,10 @@ def run_ours(args):
     peak = peaks["bf16_tflops_sustained"]
     line = {
         "metric": METRIC, "value": tokens / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step,
+        "step_ms_rank0": {"median": float(np.median(steps_ms)), "min": float(np.min(steps_ms)),
+                          "max": float(np.max(steps_ms))},
+        "higher_is_better": True,
         "scaling": "strong" if args.vocab_parallel else "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": f"{args.workload}: {head_name(w)} head d={w.d} V={w.V}, {w.N} responses "
                                f"({w.n_prompts} prompts x {w.group_size}), {job.T} scored tokens per GPU, "
@@ -658,6 +663,9 @@ def main():
                          "all-gathered and merged) instead of giving every rank its own batch")
     ap.add_argument("--v-splits", type=int, default=0,
                     help="vocabulary ranges per row tile of the fused GEMM (af_set_tuning v_splits); 0 = the library's choice")
+    ap.add_argument("--bwd-token-block", type=int, default=0,
+                    help="token rows per block of the backward and fused-update calls (af_set_tuning "
+                         "bwd_token_block, a multiple of 128); 0 = the library's choice")
     ap.add_argument("--weight-refresh", action="store_true",
                     help="also time the steps while a new LM-head weight is loaded and swapped in every step")
     ap.add_argument("--gemm", default="default", choices=["default", "single", "pair"],

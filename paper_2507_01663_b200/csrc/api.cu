@@ -74,14 +74,12 @@ af_status af_create(af_ctx** out, int device) {
   cudaDriverEntryPointQueryResult qres;
   if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
       qres != cudaDriverEntryPointSuccess || !fn) {
-    delete c;
+    af_destroy(c);
     return AF_ERR_CUDA;
   }
   c->encode = reinterpret_cast<EncodeTiledFn>(fn);
-  if (cudaMalloc(&c->d_err, 256) != cudaSuccess || cudaMemset(c->d_err, 0, 256) != cudaSuccess) {
-    delete c;
-    return AF_ERR_WORKSPACE;
-  }
+  if (cudaMalloc(&c->d_err, 256) != cudaSuccess) { c->d_err = nullptr; cudaGetLastError(); af_destroy(c); return AF_ERR_WORKSPACE; }
+  if (cudaMemset(c->d_err, 0, 256) != cudaSuccess) { af_destroy(c); return AF_ERR_CUDA; }
   af_status st = ws_grow(c->loss_ws, loss_workspace_bytes(c->sm_count));
   if (st == AF_OK && cudaMemset(c->loss_ws.p, 0, c->loss_ws.cap) != cudaSuccess) st = AF_ERR_CUDA;
   if (st == AF_OK) st = ws_grow(c->ctrl_ws, controller_workspace_bytes(c->sm_count));
