@@ -21,6 +21,12 @@
  *     (they share its workspace).  Use one context per concurrent stream.
  *   - Workspace grows on demand with cudaMalloc (which may synchronise).  Call af_reserve once
  *     with the largest sizes to keep allocation out of the hot calls.
+ *   - Stream capture: once af_reserve has covered the sizes (and the tuning is unchanged), every
+ *     call except af_pack_microbatch, af_check_device_errors, af_reserve and af_destroy issues
+ *     only kernel launches and asynchronous memsets on `stream`, so a sequence of them may be
+ *     recorded into a CUDA graph and replayed on new contents of the same buffers.
+ *     af_pack_microbatch stages its index list through pinned host memory and waits on an
+ *     event of its own; it cannot be recorded.  Nothing is claimed for af_token_logprob_static.
  *   - Only compute capability 10.0 devices are accepted.  There is no CPU path.
  */
 #ifndef ASYNCFLOW_H_
