@@ -526,6 +526,7 @@ def run_ours(args):
         job.step_e2e()
     ms_e2e_total = timed_loop(job.step_e2e, args.steps, world)
     ms_e2e, _ = reduce_over_ranks(ms_e2e_total / args.steps, job.T, world)
+    e2e_steps_ms = list(timed_loop.last_steps_ms)
 
     fused = None
     if w.backward:
@@ -579,7 +580,10 @@ def run_ours(args):
                                  if GEMM_DRAM_BYTES_PER_TOKEN_7B and (w.d, w.V) == (3584, 152064)
                                  and args.gemm != "single" and args.v_splits == 0 and not w.token_budget else None)},
         "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": job.h2d_bytes,
-                "d2h_bytes_per_step": int(sum(lo.numel() for lo in job.loss_outs)), "ms_per_step": ms_e2e},
+                "d2h_bytes_per_step": int(sum(lo.numel() for lo in job.loss_outs)), "ms_per_step": ms_e2e,
+                # the first timed step cannot hide its own copy behind a previous step's kernels
+                "step_ms_rank0": {"first": e2e_steps_ms[0], "median": float(np.median(e2e_steps_ms)),
+                                  "min": float(np.min(e2e_steps_ms))}},
         "gpu_launches": job.launches_per_step * args.steps,
         "clocks": clocks, "loss": loss,
     }
