@@ -255,11 +255,13 @@ class ScoringJob:
             total += T
         return total
 
-    def hbm_kernels_at_scale(self, peak_gbs: float) -> dict:
+    def hbm_kernels_at_scale(self, peak_gbs: float, log2_n: int = 28) -> dict:
         """The memory-bound kernels timed alone, before the long GEMM loop heats the part (the
         condition the measured copy bandwidth was taken under): pack at the workload's own size,
-        loss and advantage at sizes where bandwidth, not launch latency, decides (2^26 tokens /
-        responses)."""
+        loss, advantage and the controller's scan at 2^log2_n tokens / responses / samples, where
+        bandwidth rather than launch latency decides (the default, 2^28, moves 2-5 GB per call like the
+        4 GB copy that defines the measured peak; at 2^26 the same kernels read 3-7 % lower, and so
+        does a plain copy of that size)."""
         dev, c, B = self.dev, self.ctx, self.B
         out = {}
 
@@ -282,7 +284,7 @@ class ScoringJob:
         gbs = nbytes / ms / 1e6
         out["pack_microbatch"] = {"tokens": t_mb, "bytes_per_token": 2 * (2 * w.d + 12), "ms": ms, "gbs": gbs,
                                   "frac": gbs / peak_gbs, "where": "timed alone, 10 calls (2 kernels + metadata copy each)"}
-        n = 1 << 26
+        n = 1 << log2_n
         seq = 1024
         logp = wl.gen_surrogate_logp(self.w, 1 << 20, dev).repeat(n >> 20)
         old, ref, ent = logp + 0.1, logp - 0.1, -logp
@@ -301,7 +303,7 @@ class ScoringJob:
         out["grpo_advantage"] = {"responses": n, "group_size": G, "bytes_per_response": 8, "ms": ms, "gbs": gbs,
                                  "frac": gbs / peak_gbs}
         del r, a
-        # controller: one read request against a 2^26-sample status table (12 B read per sample:
+        # controller: one read request against a 2^log2_n-sample status table (12 B read per sample:
         # ready, consumed, length) that hands out the first 4096 eligible samples
         tab = {"ready": torch.ones(n, dtype=torch.int32, device=dev),
                "consumed": torch.zeros(n, dtype=torch.int32, device=dev),
@@ -497,7 +499,7 @@ def run_ours(args):
     job = ScoringJob(w, dev, {"default": 0, "single": 1, "pair": 2}[args.gemm], world, args.v_splits,
                      args.vocab_parallel, rank, args.bwd_token_block)
     peaks = measured_peaks()
-    hbm_alone = job.hbm_kernels_at_scale(peaks["hbm_gbs"]) if rank == 0 and world == 1 else {}
+    hbm_alone = job.hbm_kernels_at_scale(peaks["hbm_gbs"], args.hbm_log2) if rank == 0 and world == 1 else {}
 
     for _ in range(args.warmup):
         job.step()
@@ -667,6 +669,8 @@ def main():
                          "all-gathered and merged) instead of giving every rank its own batch")
     ap.add_argument("--v-splits", type=int, default=0,
                     help="vocabulary ranges per row tile of the fused GEMM (af_set_tuning v_splits); 0 = the library's choice")
+    ap.add_argument("--hbm-log2", type=int, default=28, choices=range(20, 30),
+                    help="the memory-bound kernels are also timed alone on 2^N tokens / responses / samples")
     ap.add_argument("--bwd-token-block", type=int, default=0,
                     help="token rows per block of the backward and fused-update calls (af_set_tuning "
                          "bwd_token_block, a multiple of 128); 0 = the library's choice")

@@ -11,15 +11,18 @@
 //          consumed.  An ordered, bounded stream compaction: 8-12 bytes read per sample.
 //
 // A launch of `get` is two passes.  Pass 1: every block reduces its contiguous segment of the
-// table to (eligible count, eligible tokens).  Pass 2: a block sums the aggregates of the blocks
-// before it, and only if the prefix can still reach into its segment re-reads the segment, ranks
-// its eligible samples with a block-wide scan and emits those inside the limits.  Small tables
+// table to (eligible count, eligible tokens, first tile holding an eligible sample).  Pass 2: a
+// block sums the aggregates of the blocks before it, and only if the prefix can still reach into
+// its segment re-reads the segment from that first tile on (a table whose head has been consumed
+// already is the normal case), ranks its eligible samples with a block-wide scan and emits those
+// inside the limits.  Small tables
 // (one segment) run pass 2 alone.  All integer arithmetic; the result is unique.
 //
 // Balancing (host): the k-way largest differencing method of Karmarkar and Karp on token counts,
 // with or without equal sample counts per group.  A sequential heap algorithm over a few thousand
 // integers: it runs on the host, where the index lists live.
 #include <algorithm>
+#include <climits>
 #include <queue>
 #include <vector>
 
@@ -36,7 +39,7 @@ constexpr int64_t kSingleBlockMax = 16384;     // tables up to this size are ser
 
 struct Agg {                                   // per-block aggregate of pass 1
   int count;
-  int pad;
+  int first_tile;                              // first tile of the segment that holds an eligible sample
   long long tokens;
 };
 
@@ -117,25 +120,36 @@ __global__ void __launch_bounds__(kThreads) controller_count_kernel(
     int64_t N, uint32_t mask, uint32_t task_bit, int vec_ok, Agg* __restrict__ agg, af_get_result* __restrict__ out) {
   __shared__ int s_c[kWarps];
   __shared__ long long s_t[kWarps];
+  __shared__ int s_first;
+  if (threadIdx.x == 0) s_first = INT_MAX;
+  __syncthreads();
   int64_t q0, q1;
   segment_of(N, blockIdx.x, gridDim.x, q0, q1);
   int c = 0; long long t = 0;
+  int tile = 0, first = INT_MAX;                          // tile index within the segment (fits: N < 2^31)
   int64_t q = q0 + threadIdx.x;
-  for (; q + kThreads < q1; q += 2 * kThreads) {          // two independent quads in flight per thread
+  for (; q + kThreads < q1; q += 2 * kThreads, tile += 2) {   // two independent quads in flight per thread
     const Quad v0 = load_quad(ready, consumed, length, q * kQuad, N, mask, task_bit, vec_ok != 0);
     const Quad v1 = load_quad(ready, consumed, length, (q + kThreads) * kQuad, N, mask, task_bit, vec_ok != 0);
+    int c0 = 0, c1 = 0;
 #pragma unroll
-    for (int k = 0; k < kQuad; ++k) { c += v0.elig[k] + v1.elig[k]; t += v0.len[k] + v1.len[k]; }
+    for (int k = 0; k < kQuad; ++k) { c0 += v0.elig[k]; c1 += v1.elig[k]; t += v0.len[k] + v1.len[k]; }
+    if (first == INT_MAX && (c0 | c1)) first = c0 ? tile : tile + 1;
+    c += c0 + c1;
   }
-  for (; q < q1; q += kThreads) {
+  for (; q < q1; q += kThreads, ++tile) {
     const Quad v = load_quad(ready, consumed, length, q * kQuad, N, mask, task_bit, vec_ok != 0);
+    int c0 = 0;
 #pragma unroll
-    for (int k = 0; k < kQuad; ++k) { c += v.elig[k]; t += v.len[k]; }
+    for (int k = 0; k < kQuad; ++k) { c0 += v.elig[k]; t += v.len[k]; }
+    if (first == INT_MAX && c0) first = tile;
+    c += c0;
   }
+  if (first != INT_MAX) atomicMin(&s_first, first);
   int c_ex, c_tot; long long t_ex, t_tot;
-  block_scan(c, t, c_ex, t_ex, c_tot, t_tot, s_c, s_t);
+  block_scan(c, t, c_ex, t_ex, c_tot, t_tot, s_c, s_t);   // its barriers also order s_first
   if (threadIdx.x == 0) {
-    agg[blockIdx.x] = Agg{c_tot, 0, t_tot};
+    agg[blockIdx.x] = Agg{c_tot, s_first == INT_MAX ? 0 : s_first, t_tot};
     if (blockIdx.x == 0) { out->count = 0; out->eligible = 0; out->tokens = 0; }
   }
 }
@@ -176,7 +190,9 @@ __global__ void __launch_bounds__(kThreads) controller_select_kernel(
   int run_c = base_c; long long run_t = base_t;          // eligible seen so far, in index order
   int sel_c = 0; long long sel_t = 0;                    // selected by this thread
   int elig_c = 0;
-  for (int64_t qb = q0; qb < q1; qb += kThreads) {       // block-uniform trip count
+  // tiles before the segment's first eligible sample need no visit (pass 1 recorded where it is)
+  const int64_t q_start = single ? q0 : q0 + (int64_t)agg[blockIdx.x].first_tile * kThreads;
+  for (int64_t qb = q_start; qb < q1; qb += kThreads) {   // block-uniform trip count
     const int64_t q = qb + threadIdx.x;
     Quad v;
     if (q < q1) {

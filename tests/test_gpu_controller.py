@@ -81,9 +81,11 @@ def test_get_with_unaligned_tables(ctx, offset):
     one_get(ctx, tab, host, 0b0101, 2, 5000, 300000)
 
 
-def test_selection_ends_deep_inside_a_large_table(ctx):
-    """The prefix ends in a late block of the two-pass path: count limit, then token limit."""
-    n = 300000
+@pytest.mark.parametrize("n", [300000, 5000003])
+def test_selection_ends_deep_inside_a_large_table(ctx, n):
+    """The prefix ends in a late block of the two-pass path: count limit, then token limit.  At the
+    larger size a block's segment spans several tiles and the first eligible sample sits in the
+    middle of one, after tiles the second pass does not visit."""
     ready = np.full(n, 1, np.uint32)
     ready[: n - 5000] = 0                                            # only the last 5000 samples are ready
     consumed = np.zeros(n, np.uint32)
