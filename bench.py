@@ -321,6 +321,7 @@ class ScoringJob:
         gbs = 12.0 * n / ms / 1e6
         out["controller_get"] = {"samples": n, "bytes_per_sample": 12, "ms": ms, "gbs": gbs, "frac": gbs / peak_gbs,
                                  "returned": B.read_get_result(res)["count"],
+                                 "clear": {"ms": ms_clear, "bytes_per_sample": 8, "gbs": 8.0 * n / ms_clear / 1e6},
                                  "where": "2 launches (count, select); time of a get + clear pair minus a clear"}
         return out
 

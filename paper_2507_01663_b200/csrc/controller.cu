@@ -251,13 +251,29 @@ __global__ void __launch_bounds__(kThreads) controller_put_kernel(uint32_t* __re
   }
 }
 
+// Four samples per thread with 128-bit accesses (tail and unaligned tables: one sample per thread),
+// one block per 4 KB run of the table in address order.
 __global__ void __launch_bounds__(kThreads) controller_clear_kernel(uint32_t* __restrict__ ready,
                                                                    uint32_t* __restrict__ consumed, int64_t N,
-                                                                   uint32_t column_bits, uint32_t task_bits) {
+                                                                   uint32_t column_bits, uint32_t task_bits, int vec_ok) {
   const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < N; i += stride) {
-    if (column_bits) ready[i] &= ~column_bits;
-    if (task_bits) consumed[i] &= ~task_bits;
+  const int64_t n_vec = vec_ok ? N / 4 : 0;
+  const uint32_t keep_r = ~column_bits, keep_c = ~task_bits;
+  for (int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; v < n_vec; v += stride) {
+    if (column_bits) {
+      uint4 r = __ldcs(reinterpret_cast<const uint4*>(ready) + v);
+      r.x &= keep_r; r.y &= keep_r; r.z &= keep_r; r.w &= keep_r;
+      __stcs(reinterpret_cast<uint4*>(ready) + v, r);
+    }
+    if (task_bits) {
+      uint4 c = __ldcs(reinterpret_cast<const uint4*>(consumed) + v);
+      c.x &= keep_c; c.y &= keep_c; c.z &= keep_c; c.w &= keep_c;
+      __stcs(reinterpret_cast<uint4*>(consumed) + v, c);
+    }
+  }
+  for (int64_t i = n_vec * 4 + (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < N; i += stride) {
+    if (column_bits) ready[i] &= keep_r;
+    if (task_bits) consumed[i] &= keep_c;
   }
 }
 
@@ -281,9 +297,14 @@ cudaError_t launch_controller_put(const af_controller_view& v, const int32_t* id
 
 cudaError_t launch_controller_clear(const af_controller_view& v, uint32_t column_bits, uint32_t task_bits,
                                     int sm_count, cudaStream_t s) {
-  if (v.n_samples == 0) return cudaSuccess;
-  controller_clear_kernel<<<grid_for(v.n_samples, sm_count), kThreads, 0, s>>>(v.ready, v.consumed, v.n_samples,
-                                                                              column_bits, task_bits);
+  if (v.n_samples == 0 || (column_bits == 0 && task_bits == 0)) return cudaSuccess;
+  const int vec_ok = ((reinterpret_cast<uintptr_t>(v.ready) | reinterpret_cast<uintptr_t>(v.consumed)) & 15) == 0;
+  int64_t blocks = ((vec_ok ? v.n_samples / 4 : v.n_samples) + kThreads - 1) / kThreads;
+  if (blocks < 1) blocks = 1;
+  if (blocks > (int64_t)1 << 30) blocks = (int64_t)1 << 30;
+  (void)sm_count;
+  controller_clear_kernel<<<(int)blocks, kThreads, 0, s>>>(v.ready, v.consumed, v.n_samples, column_bits, task_bits,
+                                                          vec_ok);
   return cudaGetLastError();
 }
 

@@ -170,10 +170,18 @@ def test_put_flags_bad_indices_and_skips_them(ctx):
     assert ctx.check_device_errors() == 0
 
 
-def test_clear_is_selective(ctx):
-    tab = dev_table(np.full(5000, 0b111, np.uint32), np.full(5000, 0b11, np.uint32), np.ones(5000, np.int32))
+@pytest.mark.parametrize("n,offset", [(1, 0), (3, 0), (5000, 0), (5003, 0), (4099, 1), (1 << 20, 0), ((1 << 20) + 2, 3)])
+def test_clear_is_selective(ctx, n, offset):
+    ready, consumed, length = u32_table(n, n)
+    tab = dev_table(ready | 0b010, consumed | 0b01, length, offset=offset)
     ctx.controller_clear(tab, 0b010, 0b01)
-    assert np.all(np_of(tab["ready"]) == 0b101) and np.all(np_of(tab["consumed"]) == 0b10)
+    assert np.array_equal(np_of(tab["ready"]).view(np.uint32), ready & ~np.uint32(0b010))
+    assert np.array_equal(np_of(tab["consumed"]).view(np.uint32), consumed & ~np.uint32(0b01))
+    ctx.controller_clear(tab, 0, 0b10)                              # one column only
+    assert np.array_equal(np_of(tab["ready"]).view(np.uint32), ready & ~np.uint32(0b010))
+    assert np.array_equal(np_of(tab["consumed"]).view(np.uint32), consumed & ~np.uint32(0b11))
+    ctx.controller_clear(tab, 0, 0)                                 # nothing asked: nothing changes
+    assert np.array_equal(np_of(tab["consumed"]).view(np.uint32), consumed & ~np.uint32(0b11))
 
 
 def test_host_argument_errors(ctx):
