@@ -41,7 +41,7 @@ def test_advantage_workload_rewards(ctx, name, ddof):
     assert ctx.check_device_errors() == 0
 
 
-@pytest.mark.parametrize("G", [1, 2, 3, 5, 8, 31, 32, 33, 64, 100, 1000, 5000])
+@pytest.mark.parametrize("G", [1, 2, 3, 4, 5, 8, 16, 31, 32, 33, 64, 100, 128, 256, 1000, 5000])
 def test_advantage_group_sizes(ctx, G):
     n_groups = 37 if G < 1000 else 3
     N = G * n_groups
@@ -49,6 +49,22 @@ def test_advantage_group_sizes(ctx, G):
     ref = O.grpo_advantage_ref(np_of(r), np.arange(N) // G, n_groups, 1e-6, 0)
     adv = torch.full((N,), 9.0, device=device())
     ctx.grpo_advantage(r, None, n_groups, adv)
+    assert np.abs(np_of(adv) - ref).max() <= ADV_TOL
+
+
+@pytest.mark.parametrize("G", [4, 8, 64, 128, 6, 200])
+def test_advantage_of_nearly_equal_rewards(ctx, G):
+    """Rewards of a group a few units in the last place apart: the deviations (~1e-8..1e-6) are of the
+    size of eps, so the mean must be right to far below an fp32 ulp for the advantages to be."""
+    n_groups = 9
+    base = np.float32(0.3)
+    steps = np.random.default_rng(G).integers(0, 40, size=G * n_groups)
+    r = base + steps.astype(np.float32) * np.spacing(base)            # exact in fp32
+    assert np.all(r.astype(np.float32) == r)
+    ref = O.grpo_advantage_ref(r.astype(np.float32), np.arange(G * n_groups) // G, n_groups, 1e-6, 0)
+    adv = torch.full((G * n_groups,), 9.0, device=device())
+    ctx.grpo_advantage(f32(r), None, n_groups, adv)
+    assert np.abs(ref).max() > 0.05                                   # the case is not trivially zero
     assert np.abs(np_of(adv) - ref).max() <= ADV_TOL
 
 
