@@ -178,8 +178,9 @@ af_status af_merge_logprob_shards(af_ctx* ctx, const float* partials, const int3
                                   void* stream);
 
 /* ---------------------------------------------------------------------------------------------
- * af_grpo_advantage -- group-normalised advantages: "rewards normalized within a group of
- * responses to the same prompt" (paper Section 7.1 "RL algorithms"; no critic).
+ * af_grpo_advantage -- group-normalised advantages: GRPO has no critic and takes each response's
+ * advantage from its reward relative to the other responses to the same prompt (paper Section
+ * 7.1 "RL algorithms").
  *
  * For each group g with members I_g (n_g = |I_g|):  mu = mean r;  sigma = sqrt(sum (r-mu)^2 /
  * (n_g - ddof));  adv_i = (r_i - mu) / (sigma + eps_adv).  A group of equal rewards gets zeros.

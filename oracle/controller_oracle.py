@@ -14,8 +14,8 @@ file; it shares no code with the CUDA library.
   balance ..... split samples over k groups so that token totals are as even as possible;
                 "DP" keeps the number of samples per group equal, "PP" drops that constraint
 
-Readings where the paper is silent (it says "select the required number of data samples" and
-nothing more): eligible samples are taken in increasing global index; a request carries a
+Readings where the paper is silent (of the selection it says only that the required number of
+samples is chosen): eligible samples are taken in increasing global index; a request carries a
 sample count and, optionally, a token budget; the selection is the longest prefix of the
 eligible sequence within both limits, except that a first sample longer than the whole budget
 is handed out alone.  Ties in the differencing method are broken as stated in kk_partition_ref.

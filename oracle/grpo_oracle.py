@@ -8,8 +8,8 @@ patterns and are widened exactly to float64).
 The paper (AsyncFlow) states the data flow -- a sample-indexed columnar store read by global
 index (Section 4.3 "Data Plane"), micro-batches handed out as metadata and fetched by the
 worker (Section 4.2 "Interaction Interface"), the ``compute_log_prob`` task (Appendix, Backend
--level interface listing), GRPO advantages "normalized within a group of responses to the same
-prompt" (Section 7.1 "RL algorithms") -- but prints no formula.  The arithmetic is therefore the
+-level interface listing), GRPO advantages taken from rewards relative to the other responses to
+the same prompt (Section 7.1 "RL algorithms") -- but prints no formula.  The arithmetic is therefore the
 textbook definition of each quantity, written out below with no blocking, fusion or reordering:
 
   log-softmax / entropy .... the definition over the full vocabulary row
@@ -69,6 +69,32 @@ def pack_microbatch_ref(tok_offset, idx, columns, adv=None):
     if adv is not None:
         out["adv_seq"] = np.asarray(adv)[idx].copy()
     return out
+
+
+def unpack_microbatch_ref(tok_offset, idx, packed_columns, store_columns):
+    """Write a task's per-token results back to the store by metadata (Section 4.2: once the task
+    has computed, it writes its results to the storage units according to the metadata): the
+    inverse of the gather above, one column at a time, in place.
+
+    tok_offset      : [N+1] int64
+    idx             : [B] sample indices, each at most once (two writers of one row have no defined order)
+    packed_columns  : dict name -> array [T, ...] in packed order (T = sum of the listed lengths)
+    store_columns   : dict name -> array [sum L, ...]; rows of the listed samples are overwritten,
+                      every other row is left as it is
+    returns T
+    """
+    tok_offset = np.asarray(tok_offset, dtype=np.int64)
+    idx = np.asarray(idx, dtype=np.int64)
+    if len(set(idx.tolist())) != idx.shape[0]:
+        raise ValueError("duplicate sample index in a write-back list")
+    t = 0
+    for j in range(idx.shape[0]):
+        lo, hi = int(tok_offset[idx[j]]), int(tok_offset[idx[j] + 1])
+        for name, packed in packed_columns.items():
+            for r in range(lo, hi):
+                store_columns[name][r] = packed[t + (r - lo)]
+        t += hi - lo
+    return t
 
 
 # ----------------------------------------------------------------------------------------

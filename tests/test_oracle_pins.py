@@ -101,6 +101,47 @@ def test_pack_empty():
     assert p["cu_seqlens"].tolist() == [0] and p["hidden"].shape[0] == 0
 
 
+def test_unpack_is_the_inverse_of_pack():
+    rng = np.random.default_rng(21)
+    off, cols, adv = _store(rng, N=11)
+    N = off.shape[0] - 1
+    idx = rng.permutation(N)[:7]
+    p = O.pack_microbatch_ref(off, idx, cols, adv)
+    # results in packed order, written back: the listed samples' rows take them, the rest stay
+    res = {"old_logp": rng.standard_normal(p["old_logp"].shape[0]).astype(np.float32),
+           "target": rng.integers(0, 1000, size=p["target"].shape[0]).astype(np.int32)}
+    store = {"old_logp": cols["old_logp"].copy(), "target": cols["target"].copy()}
+    T = O.unpack_microbatch_ref(off, idx, res, store)
+    assert T == p["cu_seqlens"][-1]
+    # (a) gathering the written columns again returns the results bit for bit
+    again = O.pack_microbatch_ref(off, idx, store)
+    assert again["old_logp"].tobytes() == res["old_logp"].tobytes()
+    assert again["target"].tobytes() == res["target"].tobytes()
+    # (b) rows of samples outside the list are untouched
+    others = np.setdiff1d(np.arange(N), idx)
+    for i in others:
+        assert np.array_equal(store["old_logp"][off[i]:off[i + 1]], cols["old_logp"][off[i]:off[i + 1]])
+        assert np.array_equal(store["target"][off[i]:off[i + 1]], cols["target"][off[i]:off[i + 1]])
+    # (c) the scatter written as one fancy-index assignment through the gather's own row map
+    rows = O.pack_microbatch_ref(off, idx, {"row": np.arange(off[-1])})["row"]
+    direct = cols["old_logp"].copy()
+    direct[rows] = res["old_logp"]
+    assert direct.tobytes() == store["old_logp"].tobytes()
+    # (d) writing back what was gathered changes nothing
+    same = {"old_logp": cols["old_logp"].copy()}
+    O.unpack_microbatch_ref(off, idx, {"old_logp": p["old_logp"]}, same)
+    assert same["old_logp"].tobytes() == cols["old_logp"].tobytes()
+
+
+def test_unpack_empty_list_and_duplicates():
+    off, cols, _ = _store(np.random.default_rng(22))
+    store = {"old_logp": cols["old_logp"].copy()}
+    assert O.unpack_microbatch_ref(off, np.zeros(0, np.int64), {"old_logp": np.zeros(0, np.float32)}, store) == 0
+    assert store["old_logp"].tobytes() == cols["old_logp"].tobytes()
+    with pytest.raises(ValueError):
+        O.unpack_microbatch_ref(off, np.array([2, 5, 2]), {"old_logp": np.zeros(64, np.float32)}, store)
+
+
 # ---------------------------------------------------------------- O2 log-prob / entropy
 def _rand_hw(rng, T, d, V, hs=1.0, ws=0.3):
     return to_bits(rng.standard_normal((T, d)) * hs), to_bits(rng.standard_normal((V, d)) * ws)
