@@ -284,6 +284,13 @@ class ScoringJob:
         gbs = nbytes / ms / 1e6
         out["pack_microbatch"] = {"tokens": t_mb, "bytes_per_token": 2 * (2 * w.d + 12), "ms": ms, "gbs": gbs,
                                   "frac": gbs / peak_gbs, "where": "timed alone, 10 calls (2 kernels + metadata copy each)"}
+        # results written back by the same index list: 4 B read + 4 B written per token of one column
+        col = torch.empty(int(self.off[-1]), device=dev)
+        ms = avg_ms(lambda: c.unpack_microbatch(self.off, self.idx, [self.logp], [col]))
+        out["unpack_microbatch"] = {"tokens": t_mb, "bytes_per_token": 8, "ms": ms, "gbs": 8.0 * t_mb / ms / 1e6,
+                                    "where": "one log-prob column of the same micro-batch back to the store; "
+                                             "launch-bound at this size (2 kernels + metadata copy)"}
+        del col
         n = 1 << log2_n
         seq = 1024
         logp = wl.gen_surrogate_logp(self.w, 1 << 20, dev).repeat(n >> 20)

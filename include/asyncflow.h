@@ -22,11 +22,12 @@
  *   - Workspace grows on demand with cudaMalloc (which may synchronise).  Call af_reserve once
  *     with the largest sizes to keep allocation out of the hot calls.
  *   - Stream capture: once af_reserve has covered the sizes (and the tuning is unchanged), every
- *     call except af_pack_microbatch, af_check_device_errors, af_reserve and af_destroy issues
- *     only kernel launches and asynchronous memsets on `stream`, so a sequence of them may be
- *     recorded into a CUDA graph and replayed on new contents of the same buffers.
- *     af_pack_microbatch stages its index list through pinned host memory and waits on an
- *     event of its own; it cannot be recorded.  Nothing is claimed for af_token_logprob_static.
+ *     call except af_pack_microbatch, af_unpack_microbatch, af_check_device_errors, af_reserve and
+ *     af_destroy issues only kernel launches and asynchronous memsets on `stream`, so a sequence
+ *     of them may be recorded into a CUDA graph and replayed on new contents of the same buffers.
+ *     af_pack_microbatch and af_unpack_microbatch stage their index list through pinned host
+ *     memory and wait on an event of their own; they cannot be recorded.  Nothing is claimed for
+ *     af_token_logprob_static.
  *   - Only compute capability 10.0 devices are accepted.  There is no CPU path.
  */
 #ifndef ASYNCFLOW_H_
@@ -325,6 +326,40 @@ af_status af_controller_get(af_ctx* ctx, const af_controller_view* table, uint32
                             int32_t* out_idx, af_get_result* out, void* stream);
 af_status af_controller_clear(af_ctx* ctx, const af_controller_view* table, uint32_t column_bits,
                               uint32_t task_bits, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * af_unpack_microbatch -- per-token results of a task, in packed order -> the store, by metadata.
+ *
+ * The inverse of af_pack_microbatch for results (Section 4.2 "Interaction Interface": when a task
+ * has computed, it writes its results to the storage units according to the metadata, and the
+ * controllers learn that the data at these locations can now be consumed).  For j in [0, B) and
+ * every listed column k, the packed values at cu[j] .. cu[j+1]-1 (cu as af_pack_microbatch builds
+ * it from the same list) are copied, bit for bit, to rows tok_offset[idx[j]] ..
+ * tok_offset[idx[j]+1]-1 of the store column; rows of samples not listed keep their contents.
+ * Columns hold 4-byte elements (fp32 log-probs, int32 ids).  If `table` is given, the bits
+ * `column_bits` of ready[idx[j]] are set afterwards on the same stream (what af_controller_put
+ * does), so that a later af_controller_get on that stream sees data and status together.
+ *
+ * Errors: AF_ERR_INDEX for an index outside [0, N); AF_ERR_INVALID_ARG for an index listed twice
+ * (two writers of one row have no defined order), for n_cols outside [0, AF_MAX_WRITE_COLS], a
+ * NULL column pointer while there are tokens to move, or a table whose n_samples differs from
+ * N; AF_ERR_CAPACITY if the listed samples hold 2^31 tokens or more.  *T_out (host, nullable) receives the token count.  B == 0 is
+ * valid and writes nothing.  Like af_pack_microbatch the call stages the list through pinned
+ * host memory and cannot be recorded into a CUDA graph.
+ * ------------------------------------------------------------------------------------------- */
+#define AF_MAX_WRITE_COLS 4
+typedef struct {
+  int32_t n_cols;                          /* columns to write: 0 .. AF_MAX_WRITE_COLS              */
+  int32_t reserved;
+  const void* packed[AF_MAX_WRITE_COLS];   /* [T] dev, 4-byte elements in packed order               */
+  void* store[AF_MAX_WRITE_COLS];          /* [sum L] dev, the store's column of the same element   */
+} af_write_cols;
+
+af_status af_unpack_microbatch(af_ctx* ctx, const int64_t* tok_offset_host, int64_t n_samples,
+                               const int32_t* idx_host, int32_t B, const af_write_cols* cols,
+                               const af_controller_view* table, uint32_t column_bits,
+                               int64_t* T_out, void* stream);
+
 
 /* ---------------------------------------------------------------------------------------------
  * af_balance_partitions -- token-balanced split of a batch over k groups (host call, no GPU).

@@ -27,7 +27,8 @@ EXPORTS = ["af_create", "af_destroy", "af_status_string", "af_reserve", "af_work
            "af_set_tuning", "af_check_device_errors", "af_pack_microbatch", "af_token_logprob",
            "af_grpo_advantage", "af_policy_loss", "af_policy_loss_backward", "af_token_logprob_static",
            "af_controller_put", "af_controller_get", "af_controller_clear", "af_balance_partitions",
-           "af_token_logprob_shard", "af_merge_logprob_shards", "af_policy_update"]
+           "af_token_logprob_shard", "af_merge_logprob_shards", "af_policy_update", "af_unpack_microbatch"]
+MAX_WRITE_COLS = 4
 
 
 class AfError(RuntimeError):
@@ -62,6 +63,10 @@ class LossOut(C.Structure):
 
 class ControllerView(C.Structure):
     _fields_ = [("n_samples", C.c_int64), ("ready", C.c_void_p), ("consumed", C.c_void_p), ("length", C.c_void_p)]
+
+
+class WriteCols(C.Structure):
+    _fields_ = [("n_cols", C.c_int32), ("reserved", C.c_int32), ("packed", C.c_void_p * 4), ("store", C.c_void_p * 4)]
 
 
 class GetResult(C.Structure):
@@ -112,6 +117,8 @@ def load_library() -> C.CDLL:
     lib.af_merge_logprob_shards.argtypes = [vp, vp, vp, i32, i64, i32, vp, vp, vp, vp]
     lib.af_policy_update.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i64, i32, i32, C.POINTER(LossParams), vp,
                                      vp, vp, vp, vp, vp, vp, i32, vp]
+    lib.af_unpack_microbatch.argtypes = [vp, vp, i64, vp, i32, C.POINTER(WriteCols), C.POINTER(ControllerView), u32,
+                                         C.POINTER(i64), vp]
     for name in EXPORTS:
         if name not in ("af_status_string", "af_workspace_bytes"):
             getattr(lib, name).restype = C.c_int
@@ -200,6 +207,31 @@ class Context:
         st = self.lib.af_pack_microbatch(self.handle, C.byref(sv), C.c_void_p(idx.ctypes.data),
                                          idx.shape[0], C.byref(pk), C.byref(T), _stream(stream))
         _check(st, "af_pack_microbatch")
+        return int(T.value)
+
+    def unpack_microbatch(self, tok_offset_host: np.ndarray, idx_host: np.ndarray, packed: list, store: list,
+                          table: Optional[dict] = None, column_bits: int = 0, stream=None) -> int:
+        """Write per-token results back by index list: ``packed[k]`` (device, [T], 4-byte elements in
+        packed order) goes to the rows of the listed samples in ``store[k]`` (device, [sum L]).  With
+        ``table`` the ``column_bits`` of the listed samples' ready masks are set afterwards.  Returns T."""
+        off = np.ascontiguousarray(tok_offset_host, dtype=np.int64)
+        idx = np.ascontiguousarray(idx_host, dtype=np.int32)
+        if len(packed) != len(store):
+            raise ValueError("one store column per packed column")
+        for a, b in zip(packed, store):
+            if a.element_size() != 4 or b.element_size() != 4:
+                raise ValueError("write-back columns hold 4-byte elements")
+        wc = WriteCols(n_cols=len(packed), reserved=0)
+        for k in range(min(len(packed), MAX_WRITE_COLS)):
+            wc.packed[k] = _ptr(packed[k]).value
+            wc.store[k] = _ptr(store[k]).value
+        tv = self._table(table) if table is not None else None
+        T = C.c_int64(0)
+        st = self.lib.af_unpack_microbatch(self.handle, C.c_void_p(off.ctypes.data), off.shape[0] - 1,
+                                           C.c_void_p(idx.ctypes.data), idx.shape[0], C.byref(wc),
+                                           C.byref(tv) if tv is not None else None, column_bits, C.byref(T),
+                                           _stream(stream))
+        _check(st, "af_unpack_microbatch")
         return int(T.value)
 
     def token_logprob(self, hidden, W, target, logp, entropy=None, lse=None, T=None, stream=None):

@@ -1,8 +1,11 @@
 // C ABI of the asyncflow library: argument validation, context and workspace management,
 // tensor-map encoding.  All arithmetic lives in the kernels of the other translation units.
+#include <algorithm>
+#include <cstdint>
 #include <cstdio>
 #include <cstring>
 #include <new>
+#include <vector>
 
 #include "common.cuh"
 
@@ -170,23 +173,12 @@ af_status af_reserve(af_ctx* c, int64_t max_T, int32_t max_B, int32_t d, int32_t
   return st;
 }
 
-af_status af_pack_microbatch(af_ctx* c, const af_store_view* store, const int32_t* idx_host,
-                             int32_t B, const af_packed* out, int64_t* T_out, void* stream) {
-  if (!c || !store || !out || B < 0 || (B > 0 && !idx_host) || !store->tok_offset_host ||
-      !out->cu_seqlens || store->n_samples < 0 || store->d < 1)
-    return AF_ERR_INVALID_ARG;
-  if ((store->hidden == nullptr) != (out->hidden == nullptr) ||
-      (store->target == nullptr) != (out->target == nullptr) ||
-      (store->old_logp == nullptr) != (out->old_logp == nullptr) ||
-      (store->ref_logp == nullptr) != (out->ref_logp == nullptr) ||
-      (store->adv == nullptr) != (out->adv_seq == nullptr))
-    return AF_ERR_INVALID_ARG;
-  if (store->hidden && (store->d % 8 != 0 || !aligned16(store->hidden) || !aligned16(out->hidden)))
-    return AF_ERR_ALIGNMENT;
-  if (B > out->seq_capacity) return AF_ERR_CAPACITY;
-  DeviceGuard guard(c->device);
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
-
+// Builds the per-call sequence table ([src_row][cu][idx][chunk_cu]) in a pinned staging slot and
+// queues the kernel that brings it to the device.  *T receives the token count as soon as it is
+// known (also when the capacity check fails).
+static af_status stage_sequence_table(af_ctx* c, const int64_t* tok_offset_host, int64_t n_samples,
+                                      const int32_t* idx_host, int32_t B, int64_t rows_per_chunk,
+                                      int64_t token_capacity, PackSeqTable* tab, int64_t* T_out, cudaStream_t s) {
   // staging slot (pinned): wait until the copy that last used it has been consumed
   const int slot = c->pack_slot;
   c->pack_slot = (slot + 1) % kPackRing;
@@ -210,14 +202,14 @@ af_status af_pack_microbatch(af_ctx* c, const af_store_view* store, const int32_
   int32_t* h_idx = reinterpret_cast<int32_t*>(hb + off_idx);
   const size_t off_chunk = off_idx + (((size_t)B * 4 + 15) & ~(size_t)15);
   int32_t* h_chunk = reinterpret_cast<int32_t*>(hb + off_chunk);
-  const int64_t rpc = store->hidden ? pack_rows_per_chunk(store->d) : 0;
+  const int64_t rpc = rows_per_chunk;
   int64_t T = 0, chunks = 0;
   h_cu[0] = 0;
   h_chunk[0] = 0;
   for (int32_t j = 0; j < B; ++j) {
     const int64_t i = idx_host[j];
-    if (i < 0 || i >= store->n_samples) return AF_ERR_INDEX;
-    const int64_t lo = store->tok_offset_host[i], hi = store->tok_offset_host[i + 1];
+    if (i < 0 || i >= n_samples) return AF_ERR_INDEX;
+    const int64_t lo = tok_offset_host[i], hi = tok_offset_host[i + 1];
     if (hi < lo) return AF_ERR_INVALID_ARG;
     h_src[j] = lo;
     h_idx[j] = (int32_t)i;
@@ -229,7 +221,7 @@ af_status af_pack_microbatch(af_ctx* c, const af_store_view* store, const int32_
     if (chunks >= ((int64_t)1 << 31)) return AF_ERR_CAPACITY;
   }
   if (T_out) *T_out = T;
-  if (T > out->token_capacity) return AF_ERR_CAPACITY;
+  if (T > token_capacity) return AF_ERR_CAPACITY;
 
   char* db = static_cast<char*>(c->pack_meta.p);
   if (launch_pack_meta_fetch(db, hb, bytes, s) != cudaSuccess) return AF_ERR_CUDA;
@@ -238,10 +230,72 @@ af_status af_pack_microbatch(af_ctx* c, const af_store_view* store, const int32_
     c->pack_evt_live[slot] = true;
   }
   if (cudaEventRecord(c->pack_evt[slot], s) != cudaSuccess) return AF_ERR_CUDA;
-  PackSeqTable tab{reinterpret_cast<const int64_t*>(db), reinterpret_cast<const int32_t*>(db + off_cu),
-                   reinterpret_cast<const int32_t*>(db + off_idx),
-                   reinterpret_cast<const int32_t*>(db + off_chunk), (int)chunks};
+  *tab = PackSeqTable{reinterpret_cast<const int64_t*>(db), reinterpret_cast<const int32_t*>(db + off_cu),
+                      reinterpret_cast<const int32_t*>(db + off_idx),
+                      reinterpret_cast<const int32_t*>(db + off_chunk), (int)chunks};
+  return AF_OK;
+}
+
+af_status af_pack_microbatch(af_ctx* c, const af_store_view* store, const int32_t* idx_host,
+                             int32_t B, const af_packed* out, int64_t* T_out, void* stream) {
+  if (!c || !store || !out || B < 0 || (B > 0 && !idx_host) || !store->tok_offset_host ||
+      !out->cu_seqlens || store->n_samples < 0 || store->d < 1)
+    return AF_ERR_INVALID_ARG;
+  if ((store->hidden == nullptr) != (out->hidden == nullptr) ||
+      (store->target == nullptr) != (out->target == nullptr) ||
+      (store->old_logp == nullptr) != (out->old_logp == nullptr) ||
+      (store->ref_logp == nullptr) != (out->ref_logp == nullptr) ||
+      (store->adv == nullptr) != (out->adv_seq == nullptr))
+    return AF_ERR_INVALID_ARG;
+  if (store->hidden && (store->d % 8 != 0 || !aligned16(store->hidden) || !aligned16(out->hidden)))
+    return AF_ERR_ALIGNMENT;
+  if (B > out->seq_capacity) return AF_ERR_CAPACITY;
+  DeviceGuard guard(c->device);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  PackSeqTable tab{};
+  int64_t T = 0;
+  const af_status st = stage_sequence_table(c, store->tok_offset_host, store->n_samples, idx_host, B,
+                                            store->hidden ? pack_rows_per_chunk(store->d) : 0, out->token_capacity,
+                                            &tab, &T, s);
+  if (T_out) *T_out = T;
+  if (st != AF_OK) return st;
   return launch_pack(*store, *out, tab, B, T, c->sm_count, c->d_err, s) == cudaSuccess ? AF_OK : AF_ERR_CUDA;
+}
+
+af_status af_unpack_microbatch(af_ctx* c, const int64_t* tok_offset_host, int64_t n_samples, const int32_t* idx_host,
+                               int32_t B, const af_write_cols* cols, const af_controller_view* table,
+                               uint32_t column_bits, int64_t* T_out, void* stream) {
+  if (!c || !tok_offset_host || n_samples < 0 || B < 0 || (B > 0 && !idx_host) || !cols || cols->n_cols < 0 ||
+      cols->n_cols > AF_MAX_WRITE_COLS)
+    return AF_ERR_INVALID_ARG;
+  if (table && (table->n_samples != n_samples || (n_samples > 0 && !table->ready))) return AF_ERR_INVALID_ARG;
+  // a sample may be listed once: two writers of one row would have no defined order
+  {
+    std::vector<int32_t> sorted(idx_host, idx_host + B);
+    std::sort(sorted.begin(), sorted.end());
+    if (std::adjacent_find(sorted.begin(), sorted.end()) != sorted.end()) return AF_ERR_INVALID_ARG;
+  }
+  DeviceGuard guard(c->device);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  PackSeqTable tab{};
+  int64_t T = 0;
+  // sizes first (no pointer is touched): the columns may be NULL only if there is nothing to move
+  for (int32_t j = 0; j < B; ++j) {
+    const int64_t i = idx_host[j];
+    if (i < 0 || i >= n_samples) return AF_ERR_INDEX;
+    if (tok_offset_host[i + 1] > tok_offset_host[i])
+      for (int k = 0; k < cols->n_cols; ++k)
+        if (!cols->packed[k] || !cols->store[k]) return AF_ERR_INVALID_ARG;
+  }
+  const af_status st = stage_sequence_table(c, tok_offset_host, n_samples, idx_host, B, 0, INT64_MAX, &tab, &T, s);
+  if (T_out) *T_out = T;
+  if (st != AF_OK) return st;
+  if (launch_unpack(*cols, tab, B, T, c->sm_count, s) != cudaSuccess) return AF_ERR_CUDA;
+  // the status update that follows a write (Section 4.2): after the data, on the same stream
+  if (table && column_bits && B > 0 &&
+      launch_controller_put(*table, tab.idx, B, column_bits, c->d_err, c->sm_count, s) != cudaSuccess)
+    return AF_ERR_CUDA;
+  return AF_OK;
 }
 
 af_status af_token_logprob(af_ctx* c, const void* hidden, const void* W, const int32_t* target,

@@ -69,6 +69,9 @@ struct PackSeqTable {     // device views into ctx->pack_meta for one call
 cudaError_t launch_pack_meta_fetch(void* dst_dev, const void* src_pinned, size_t bytes, cudaStream_t s);
 // Rows of the hidden column per bulk-copy chunk for hidden size d (0: rows too wide, no chunks).
 int pack_rows_per_chunk(int32_t d);
+// Per-token 4-byte columns in packed order -> the store rows of their samples.
+cudaError_t launch_unpack(const af_write_cols& cols, const PackSeqTable& tab, int32_t B, int64_t T, int sm_count,
+                          cudaStream_t s);
 cudaError_t launch_pack(const af_store_view& st, const af_packed& out, const PackSeqTable& tab,
                         int32_t B, int64_t T, int sm_count, unsigned int* d_err, cudaStream_t s);
 

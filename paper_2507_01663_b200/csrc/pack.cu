@@ -192,7 +192,41 @@ __global__ void __launch_bounds__(256) pack_cols_kernel(
   }
 }
 
+// The inverse for results: one thread per packed token writes up to four 4-byte columns to the
+// store rows of the token's sample.
+struct UnpackCols {
+  const uint32_t* packed[AF_MAX_WRITE_COLS];
+  uint32_t* store[AF_MAX_WRITE_COLS];
+  int n;
+};
+__global__ void __launch_bounds__(256) unpack_cols_kernel(UnpackCols c, const int64_t* __restrict__ src_row,
+                                                         const int32_t* __restrict__ cu, int B, int T) {
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < T; i += stride) {
+    const int j = find_seq(cu, B, (int)i);
+    const int64_t row = __ldg(src_row + j) + (i - __ldg(cu + j));
+#pragma unroll
+    for (int k = 0; k < AF_MAX_WRITE_COLS; ++k)
+      if (k < c.n) c.store[k][row] = __ldg(c.packed[k] + i);
+  }
+}
+
 }  // namespace
+
+cudaError_t launch_unpack(const af_write_cols& cols, const PackSeqTable& tab, int32_t B, int64_t T, int sm_count,
+                          cudaStream_t s) {
+  if (T == 0 || cols.n_cols == 0) return cudaSuccess;
+  UnpackCols c{};
+  c.n = cols.n_cols;
+  for (int k = 0; k < cols.n_cols; ++k) {
+    c.packed[k] = static_cast<const uint32_t*>(cols.packed[k]);
+    c.store[k] = static_cast<uint32_t*>(cols.store[k]);
+  }
+  int64_t blocks = (T + 255) / 256;
+  if (blocks > (int64_t)sm_count * 8) blocks = (int64_t)sm_count * 8;
+  unpack_cols_kernel<<<(int)blocks, 256, 0, s>>>(c, tab.src_row, tab.cu, B, (int)T);
+  return cudaGetLastError();
+}
 
 // Brings the per-call sequence table from pinned host memory to the device with a kernel (the
 // pinned buffer is mapped into the device's address space) instead of a host-to-device memcpy:

@@ -50,6 +50,7 @@ def test_struct_layouts_match_header():
     assert ctypes.sizeof(B.LossOut) == 32 and B.LossOut.n_tokens.offset == 24
     assert ctypes.sizeof(B.ControllerView) == 8 + 3 * 8
     assert ctypes.sizeof(B.GetResult) == 16 and B.GetResult.tokens.offset == 8
+    assert ctypes.sizeof(B.WriteCols) == 8 + 2 * 4 * 8 and B.WriteCols.store.offset == 8 + 4 * 8
 
 
 def test_create_without_gpu_fails_cleanly(lib):
