@@ -371,6 +371,78 @@ class ScoringJob:
             total += T
         return total
 
+    # -- streaming with the controller in the loop ------------------------------------------
+    def make_live_controller(self, wave: int = 512):
+        """Status table beside the store; responses become ready in arrival order, `wave` at a time."""
+        w, dev, B = self.w, self.dev, self.B
+        self.tab = {"ready": torch.zeros(w.N, dtype=torch.int32, device=dev),
+                    "consumed": torch.zeros(w.N, dtype=torch.int32, device=dev),
+                    "length": torch.as_tensor(w.lengths.astype(np.int32), device=dev)}
+        self.arrival_dev = torch.as_tensor(wl.arrival_order(w).astype(np.int32), device=dev)
+        self.wave = wave
+        self.req_idx = [torch.empty(w.N, dtype=torch.int32, device=dev) for _ in range(2)]
+        self.req_res = [B.new_get_result(dev) for _ in range(2)]
+        self.req_idx_host = [torch.empty(w.N, dtype=torch.int32, pin_memory=True) for _ in range(2)]
+        self.req_res_host = [torch.empty(self.req_res[0].shape, dtype=torch.uint8, pin_memory=True) for _ in range(2)]
+        self.req_done = [torch.cuda.Event() for _ in range(2)]
+        cap_T = max(self.packed["hidden"].shape[0], int(w.token_budget))
+        self.packed_live = {
+            "cu_seqlens": torch.zeros(w.N + 1, dtype=torch.int32, device=dev),
+            "hidden": self.packed["hidden"] if cap_T == self.packed["hidden"].shape[0]
+            else torch.empty(cap_T, w.d, dtype=torch.bfloat16, device=dev),
+            "target": torch.empty(cap_T, dtype=torch.int32, device=dev),
+            "old_logp": torch.empty(cap_T, device=dev), "ref_logp": torch.empty(cap_T, device=dev),
+            "adv_seq": torch.empty(w.N, device=dev),
+        }
+        self.live_logp, self.live_ent, self.live_lse, self.live_g = (torch.empty(cap_T, device=dev) for _ in range(4))
+        self.ctx.reserve(cap_T, w.N, w.d, w.V)
+        self.live_requests = 0
+
+    def _request(self, slot: int):
+        """Queue: the next wave of arrivals marked ready, one read request, its answer to pinned memory."""
+        c, w = self.ctx, self.w
+        if self.next_wave < w.N:
+            c.controller_put(self.tab, self.arrival_dev[self.next_wave:self.next_wave + self.wave], 1)
+            self.next_wave += self.wave
+        c.controller_get(self.tab, 1, 1, w.N, int(w.token_budget), self.req_idx[slot], self.req_res[slot])
+        self.req_idx_host[slot].copy_(self.req_idx[slot], non_blocking=True)
+        self.req_res_host[slot].copy_(self.req_res[slot], non_blocking=True)
+        self.req_done[slot].record()
+
+    def step_live_controller(self):
+        """The streaming step with live production and consumption: every micro-batch is whatever
+        the controller hands out (ready, not yet consumed, within the token budget).  The request
+        for micro-batch k+1 is queued before the kernels of micro-batch k, so its answer is on the
+        host long before the GPU needs the next index list."""
+        w, c, B = self.w, self.ctx, self.B
+        c.controller_clear(self.tab, 0xFFFFFFFF, 0xFFFFFFFF)
+        c.grpo_advantage(self.reward, None, w.n_prompts, self.adv)
+        store = {"tok_offset_host": self.off, "d": w.d, "adv": self.adv, **self.store}
+        self.next_wave, slot, total, k = 0, 0, 0, 0
+        self._request(slot)
+        while True:
+            self.req_done[slot].synchronize()
+            count = B.GetResult.from_buffer_copy(self.req_res_host[slot].numpy().tobytes()).count
+            if count == 0 and self.next_wave >= w.N:
+                break
+            mb = self.req_idx_host[slot][:count].numpy().copy()
+            self._request(slot ^ 1)
+            if count:
+                T = c.pack_microbatch(store, mb, self.packed_live)
+                c.token_logprob(self.packed_live["hidden"], self.W, self.packed_live["target"], self.live_logp,
+                                self.live_ent, self.live_lse, T=T)
+                c.policy_loss(self.live_logp, self.packed_live["old_logp"], self.packed_live["ref_logp"],
+                              self.packed_live["adv_seq"], self.packed_live["cu_seqlens"],
+                              self.loss_outs[k % len(self.loss_outs)], self.live_g, self.live_ent,
+                              w.clip_eps, w.clip_eps, w.kl_coef, 0, 1.0, B=count, T=T)
+                total += T
+                k += 1
+            slot ^= 1
+        self.live_requests = k
+        if total != self.T:
+            raise RuntimeError(f"the controller handed out {total} tokens of {self.T}")
+        return total
+
     # -- delayed parameter update: new weights arrive while scoring goes on -----------------
     def make_weight_refresh(self):
         """A pinned host copy of the LM-head weight (the "received new parameters"), a standby
@@ -550,6 +622,19 @@ def run_ours(args):
                  "what": "the same step through af_policy_update: forward, loss and backward in one call, the "
                          "logits evaluated once per token (6 T d V products instead of 8)"}
 
+    live = None
+    if args.live_controller and w.token_budget and world == 1:
+        job.make_live_controller()
+        for _ in range(2):
+            job.step_live_controller()
+        ms_l_total = timed_loop(job.step_live_controller, args.steps, world)
+        ms_l = ms_l_total / args.steps
+        live = {"value": job.T / (ms_l * 1e-3), "unit": UNIT, "ms_per_step": ms_l, "micro_batches": job.live_requests,
+                "what": "the same store scored with the controller in the loop: responses become ready 512 at a "
+                        "time in arrival order, every micro-batch is the answer to an af_controller_get (ready, "
+                        "not consumed, <= the token budget) read back to the host, then packed, scored and "
+                        "loss-reduced; the next request is queued ahead of the current micro-batch's kernels"}
+
     refresh = None
     if args.weight_refresh and not w.backward:
         job.make_weight_refresh()
@@ -609,6 +694,8 @@ def run_ours(args):
         line["fused_update"] = fused
     if refresh is not None:
         line["weight_refresh"] = refresh
+    if live is not None:
+        line["live_controller"] = live
     if rank == 0:
         line["balance"] = job.balance_report()
     if bwd_ms is not None:
@@ -682,6 +769,9 @@ def main():
     ap.add_argument("--bwd-token-block", type=int, default=0,
                     help="token rows per block of the backward and fused-update calls (af_set_tuning "
                          "bwd_token_block, a multiple of 128); 0 = the library's choice")
+    ap.add_argument("--live-controller", action="store_true",
+                    help="streaming workloads: also time the step with af_controller_put / get handing out the "
+                         "micro-batches")
     ap.add_argument("--weight-refresh", action="store_true",
                     help="also time the steps while a new LM-head weight is loaded and swapped in every step")
     ap.add_argument("--gemm", default="default", choices=["default", "single", "pair"],
