@@ -1,9 +1,10 @@
 // af_grpo_advantage kernels: adv_i = (r_i - mean_g) / (std_g + eps) within each prompt's group.
 //
 // Contiguous groups (group_id == NULL), 4 B read + 4 B written per sample:
-//   G a power of two in 4..128 (every GRPO workload here) and 16-byte aligned buffers: a thread
-//   owns 4 consecutive rewards (one 128-bit load), the G/4 adjacent lanes of a group combine
-//   their sums with shuffles, four independent loads are in flight per thread;
+//   G a power of two in 4..512 (every GRPO workload here) and 16-byte aligned buffers: a thread
+//   owns 4 consecutive rewards of each of four groups (G <= 16) or 16 rewards of one group
+//   (G >= 32), the adjacent lanes of a group combine their sums with shuffles, four independent
+//   128-bit loads are in flight per thread;
 //   other G <= 32: one thread per group, registers;
 //   G <= 4096: a block stages a run of whole groups in shared memory with 128-bit loads, reduces
 //   each group with warp shuffles (two passes: mean, then squared deviations) and writes the
@@ -87,7 +88,7 @@ __global__ void __launch_bounds__(kThreads) advantage_small_group_kernel(
   }
 }
 
-// Power-of-two groups, 4 <= G <= 128.  Thread v of the flat index space owns rewards 4v .. 4v+3;
+// Power-of-two groups, 4 <= G <= 16 (correct up to 128).  Thread v of the flat index space owns rewards 4v .. 4v+3;
 // a group is `team` = G/4 adjacent lanes of one warp (teams never straddle a warp because the
 // warp's first index is a multiple of 32 and team divides 32).  A warp takes kRowUnroll
 // consecutive 512-byte rows, a block kRowUnroll * 8 of them, and there is one block per such run
@@ -128,6 +129,54 @@ __global__ void __launch_bounds__(kThreads) advantage_pow2_kernel(
       const float sigma = var > 0.f ? var * rsqrtf(var) : 0.f;
       const float inv = __frcp_rn(sigma + eps);
       if (u * 32 < left) __stcs(dst + u * 32, make_float4(d0 * inv, d1 * inv, d2 * inv, d3 * inv));
+    }
+  }
+}
+
+// Power-of-two groups, 32 <= G <= 512.  A thread owns 16 rewards of ONE group (four 128-bit loads),
+// a group is `team` = G/16 adjacent lanes, a warp takes 2 KB of consecutive rewards.  Load k of a
+// team covers `team` consecutive 16-byte pieces, so every load instruction of the warp asks for
+// whole 32-byte sectors only.  Against the kernel above at the same G there are log2(G/16) shuffle
+// steps per reduction instead of log2(G/4), once per 16 rewards instead of once per 4, and one root
+// and reciprocal per 16 rewards: at G = 64 the issue slots were 66 % busy there.  Arithmetic as above.
+__global__ void __launch_bounds__(kThreads) advantage_wide_kernel(
+    const float4* __restrict__ reward, float4* __restrict__ adv, int64_t n_vec, int G, float eps, int ddof) {
+  constexpr int kVecPerWarp = 128;                          // 32 lanes x 4 float4
+  const int team = G >> 4;
+  const double inv_g = 1.0 / (double)G;                    // exact: G is a power of two
+  const float inv_denom = G - ddof > 0 ? 1.f / (float)(G - ddof) : 0.f;
+  const int lane = threadIdx.x & 31;
+  const int t = lane & (team - 1), g = lane / team;
+  const int64_t warps = (int64_t)gridDim.x * (kThreads / 32);
+  for (int64_t wv = ((int64_t)blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5)) * kVecPerWarp; wv < n_vec;
+       wv += warps * kVecPerWarp) {                          // warp-uniform trip count
+    const int64_t gv = wv + (int64_t)g * (G >> 2) + t;     // this lane's first piece of its group
+    const bool live = gv < n_vec;                           // N is a multiple of G: a group is whole or absent
+    float4 r[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) r[k] = live ? __ldcs(reward + gv + k * team) : make_float4(0.f, 0.f, 0.f, 0.f);
+    double s = 0.0;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) s += ((double)r[k].x + (double)r[k].y) + ((double)r[k].z + (double)r[k].w);
+    for (int o = team >> 1; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    const double mu = s * inv_g;
+    const float mu_hi = (float)mu;
+    const float mu_lo = (float)(mu - (double)mu_hi);
+    float q = 0.f;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      r[k].x = (r[k].x - mu_hi) - mu_lo; r[k].y = (r[k].y - mu_hi) - mu_lo;
+      r[k].z = (r[k].z - mu_hi) - mu_lo; r[k].w = (r[k].w - mu_hi) - mu_lo;
+      q = fmaf(r[k].x, r[k].x, fmaf(r[k].y, r[k].y, fmaf(r[k].z, r[k].z, fmaf(r[k].w, r[k].w, q))));
+    }
+    for (int o = team >> 1; o > 0; o >>= 1) q += __shfl_xor_sync(0xffffffffu, q, o);
+    const float var = q * inv_denom;
+    const float sigma = var > 0.f ? var * rsqrtf(var) : 0.f;
+    const float inv = __frcp_rn(sigma + eps);
+    if (live) {
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        __stcs(adv + gv + k * team, make_float4(r[k].x * inv, r[k].y * inv, r[k].z * inv, r[k].w * inv));
     }
   }
 }
@@ -234,7 +283,14 @@ cudaError_t launch_advantage(const float* reward, const int32_t* group_id, int64
   if (group_id == nullptr) {
     const int64_t G = N / n_groups;
     const bool aligned = ((reinterpret_cast<uintptr_t>(reward) | reinterpret_cast<uintptr_t>(adv)) & 15) == 0;
-    if (G >= 4 && G <= 128 && (G & (G - 1)) == 0 && aligned) {
+    if (G >= 32 && G <= 512 && (G & (G - 1)) == 0 && aligned) {
+      const int64_t n_vec = N / 4;
+      int64_t blocks = (n_vec + (int64_t)kThreads * 4 - 1) / ((int64_t)kThreads * 4);   // 16 KB of rewards per block
+      if (blocks > (int64_t)1 << 30) blocks = (int64_t)1 << 30;
+      advantage_wide_kernel<<<(int)blocks, kThreads, 0, s>>>(reinterpret_cast<const float4*>(reward),
+                                                             reinterpret_cast<float4*>(adv), n_vec, (int)G,
+                                                             eps_adv, ddof);
+    } else if (G >= 4 && G <= 16 && (G & (G - 1)) == 0 && aligned) {
       const int64_t n_vec = N / 4;
       int64_t blocks = (n_vec + (int64_t)kThreads * kRowUnroll - 1) / ((int64_t)kThreads * kRowUnroll);
       if (blocks > (int64_t)1 << 30) blocks = (int64_t)1 << 30;
