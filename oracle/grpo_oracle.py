@@ -1,6 +1,6 @@
 """CPU oracle for the GRPO scoring path.  TEST INFRASTRUCTURE ONLY.
 
-A plain, slow, fp64 restatement of what the five entry points compute.  It is what the CUDA
+A plain, slow, fp64 restatement of what the entry points of the scoring path compute.  It is what the CUDA
 library is checked against; it is not a fallback and nothing in the product path may import
 it.  It shares no code with the CUDA path (numpy only; bf16 tensors arrive as raw uint16 bit
 patterns and are widened exactly to float64).
@@ -18,7 +18,8 @@ textbook definition of each quantity, written out below with no blocking, fusion
   k3 KL estimator .......... exp(delta) - delta - 1,  delta = ref - logp
   backward ................. dZ = g * (onehot(y) - softmax), dH = dZ W, dW = dZ^T H
 
-Pins (tests/test_oracle_*.py): rows of exp(log-softmax) sum to one; brute-force enumeration
+Pins (tests/test_oracle_*.py): gather and write-back are inverse to each other and leave unlisted
+rows alone; rows of exp(log-softmax) sum to one; brute-force enumeration
 at V <= 16; closed forms (zero weights, V = 2, Bernoulli groups, four-quadrant clip table);
 invariances (logit shift, reward affine maps, group order); central finite differences of the
 whole fp64 chain for every gradient.  No function here is "parity unpinned".
