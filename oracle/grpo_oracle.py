@@ -267,3 +267,23 @@ def policy_loss_backward_ref(H_bits, W_bits, y, lse, g, vocab_rows=None):
     onehot[np.arange(z.shape[0]), y] = 1.0
     dZ = g[:, None] * (onehot - np.exp(z - lse[:, None]))
     return dZ @ W, dZ.T @ H
+
+
+def policy_loss_backward_shard_ref(H_bits, W_shard_bits, y, lse, g, v_offset):
+    """The backward of one vocabulary shard of the head (rows [v_offset, v_offset + V_s) of W):
+    dZ_tv = g_t (1{y_t = v_offset + v} - exp(z_tv - lse_t)) over the shard's columns only, with the
+    logsumexp of the WHOLE vocabulary; returns (dZ W_shard, dZ^T H) = this shard's contribution to
+    dH [T, d] (the shards' contributions add up) and its own rows of dW [V_s, d]."""
+    H = bf16_bits_to_f64(H_bits)
+    Ws = bf16_bits_to_f64(W_shard_bits)
+    y = np.asarray(y, dtype=np.int64)
+    lse = np.asarray(lse, dtype=np.float64)
+    g = np.asarray(g, dtype=np.float64)
+    z = H @ Ws.T
+    onehot = np.zeros_like(z)
+    for t in range(z.shape[0]):
+        if v_offset <= y[t] < v_offset + z.shape[1]:
+            onehot[t, y[t] - v_offset] = 1.0
+    dZ = g[:, None] * (onehot - np.exp(z - lse[:, None]))
+    return dZ @ Ws, dZ.T @ H
+

@@ -485,6 +485,42 @@ def test_sharded_scoring_merges_to_the_full_vocabulary_result(cuts):
     assert np.allclose(lse, r_lse, atol=1e-12)
 
 
+@pytest.mark.parametrize("cuts", [[0, 50], [0, 17, 50], [0, 1, 2, 49, 50]])
+def test_sharded_backward_adds_up_to_the_full_vocabulary_gradient(cuts):
+    """The shards' contributions to dH add up to the dense dH and their dW rows stack to the dense dW
+    (the dense gradient is pinned by finite differences and by autograd above); and by autograd on the
+    sharded head itself: d/dH and d/dW_shard of sum_t g_t logp_t with the softmax over all shards."""
+    rng = np.random.default_rng(6)
+    T, d, V = 9, 12, 50
+    Hb = to_bits(rng.normal(size=(T, d)))
+    Wb = to_bits(rng.normal(size=(V, d)))
+    y = rng.integers(0, V, T)
+    y[0], y[1] = cuts[1] - 1, cuts[1] % V                       # targets on both sides of a cut
+    g = rng.standard_normal(T)
+    _, _, lse = O.token_logprob_ref(Hb, Wb, y)
+    dH, dW = O.policy_loss_backward_ref(Hb, Wb, y, lse, g)
+    dH_sum, rows = np.zeros_like(dH), []
+    for a, b in zip(cuts[:-1], cuts[1:]):
+        dH_s, dW_s = O.policy_loss_backward_shard_ref(Hb, Wb[a:b], y, lse, g, a)
+        assert dW_s.shape == (b - a, d)
+        dH_sum += dH_s
+        rows.append(dW_s)
+    assert np.allclose(dH_sum, dH, atol=1e-12) and np.allclose(np.concatenate(rows), dW, atol=1e-12)
+    Ht = torch.tensor(bits_val(Hb), requires_grad=True)
+    shards = [torch.tensor(bits_val(Wb[a:b]), requires_grad=True) for a, b in zip(cuts[:-1], cuts[1:])]
+    lp = torch.log_softmax(torch.cat([Ht @ w.T for w in shards], 1), 1)[torch.arange(T), torch.from_numpy(y)]
+    (lp * torch.from_numpy(g)).sum().backward()
+    for w, r in zip(shards, rows):
+        assert np.allclose(w.grad.numpy(), r, atol=1e-12)
+    # a target outside the shard contributes only through the softmax term
+    a, b = cuts[0], cuts[1]
+    far = np.full(T, V - 1 if b <= V - 1 else 0)
+    if not (a <= far[0] < b):
+        dH_s, dW_s = O.policy_loss_backward_shard_ref(Hb, Wb[a:b], far, lse, g, a)
+        z = bits_val(Hb) @ bits_val(Wb[a:b]).T
+        assert np.allclose(dW_s, (-(g[:, None]) * np.exp(z - lse[:, None])).T @ bits_val(Hb), atol=1e-12)
+
+
 def test_shard_statistics_by_hand():
     # one token, hidden = [1, 0], shard rows give logits (2, 0, 1); target id 11 with offset 10 -> z = 0
     H = to_bits(np.array([[1.0, 0.0]]))
