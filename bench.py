@@ -180,6 +180,8 @@ class ScoringJob:
         }
         self.W = wl.gen_weight(w, device)
         self.vocab_parallel = vocab_parallel
+        # data parallel: equal batches per rank, each weighs 1 / world; vocabulary parallel: one batch
+        self.loss_scale = 1.0 if vocab_parallel else 1.0 / world
         self.v_lo, self.v_hi = vocab_shard(w.V, world, rank) if vocab_parallel else (0, w.V)
         self.reward = wl.gen_reward(w, device)
         centre = wl.centre_logp_estimate(w, self.store["hidden"], self.W, self.store["target"])
@@ -239,16 +241,25 @@ class ScoringJob:
                 ev[3].record()
             c.policy_loss(self.logp, self.packed["old_logp"], self.packed["ref_logp"], self.packed["adv_seq"],
                           self.packed["cu_seqlens"], loss_out, self.dlogp, self.ent,
-                          w.clip_eps, w.clip_eps, w.kl_coef, 0, 1.0 / self.world, B=len(mb), T=T)
+                          w.clip_eps, w.clip_eps, w.kl_coef, 0, self.loss_scale, B=len(mb), T=T)
             if w.backward:
                 if ev:
                     ev[4].record()
-                c.policy_loss_backward(self.packed["hidden"], self.W, self.packed["target"], self.lse, self.dlogp,
-                                       self.d_hidden, self.d_W, False, T=T)
+                if self.vocab_parallel:
+                    # this rank's rows of dW stay here; the ranks' contributions to dH are summed
+                    c.policy_loss_backward_shard(self.packed["hidden"], self.W_shard, self.packed["target"], self.lse,
+                                                 self.dlogp, self.v_lo, self.d_hidden, self.d_W[self.v_lo:self.v_hi],
+                                                 False, T=T)
+                else:
+                    c.policy_loss_backward(self.packed["hidden"], self.W, self.packed["target"], self.lse, self.dlogp,
+                                           self.d_hidden, self.d_W, False, T=T)
                 if ev:
                     ev[5].record()
                     self.bwd_events.append((ev[4], ev[5]))
-                allreduce_sum_(self.d_W, self.world)    # equal batches per rank: loss_scale = 1 / world
+                if self.vocab_parallel:
+                    allreduce_sum_(self.d_hidden[:T], self.world)
+                else:
+                    allreduce_sum_(self.d_W, self.world)    # equal batches per rank: loss_scale = 1 / world
             if ev:
                 self.pack_events.append((ev[0], ev[1]))
                 self.gemm_events.append((ev[2], ev[3]))
@@ -611,7 +622,7 @@ def run_ours(args):
     e2e_steps_ms = list(timed_loop.last_steps_ms)
 
     fused = None
-    if w.backward:
+    if w.backward and not args.vocab_parallel:
         for _ in range(2):
             job.step_fused_update()
         ms_f_total = timed_loop(job.step_fused_update, args.steps, world)

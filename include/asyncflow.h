@@ -253,6 +253,27 @@ af_status af_policy_loss_backward(af_ctx* ctx, const void* hidden, const void* W
                                   int32_t accumulate_dW, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * af_policy_loss_backward_shard -- the same backward on one vocabulary shard of the head (the
+ * counterpart of af_token_logprob_shard for the actor update; Section 2.1 names tensor parallelism,
+ * the paper says nothing about the head).
+ *
+ * The rank holds rows [v_offset, v_offset + V_shard) of W.  lse is the logsumexp over the WHOLE
+ * vocabulary (from af_merge_logprob_shards), target holds global ids, dlogp comes from
+ * af_policy_loss on the merged log-probs.  Over the shard's columns only:
+ *   dZ_tv = dlogp[t] * ( 1{target[t] == v_offset + v} - exp(z_tv - lse[t]) )
+ *   d_hidden_partial[t,:] = sum_v dZ_tv * W_shard[v,:]   -> [T,d] bf16: this shard's contribution;
+ *                                                           the ranks' contributions add up to
+ *                                                           d_hidden (one all-reduce)
+ *   d_W_shard[v,:]        = sum_t dZ_tv * hidden[t,:]    -> [V_shard,d] fp32: the rank's own rows
+ * Requirements as for af_policy_loss_backward with V_shard in place of V; v_offset >= 0.
+ * ------------------------------------------------------------------------------------------- */
+af_status af_policy_loss_backward_shard(af_ctx* ctx, const void* hidden, const void* W_shard,
+                                        const int32_t* target, const float* lse, const float* dlogp,
+                                        int64_t T, int32_t d, int32_t V_shard, int32_t v_offset,
+                                        void* d_hidden_partial, float* d_W_shard,
+                                        int32_t accumulate_dW, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
  * af_policy_update -- forward, loss and backward of one packed micro-batch in one call (the
  * forward-backward actor-update task of Section 7.4).
  *

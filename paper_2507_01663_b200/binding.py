@@ -27,7 +27,7 @@ EXPORTS = ["af_create", "af_destroy", "af_status_string", "af_reserve", "af_work
            "af_set_tuning", "af_check_device_errors", "af_pack_microbatch", "af_token_logprob",
            "af_grpo_advantage", "af_policy_loss", "af_policy_loss_backward", "af_token_logprob_static",
            "af_controller_put", "af_controller_get", "af_controller_clear", "af_balance_partitions",
-           "af_token_logprob_shard", "af_merge_logprob_shards", "af_policy_update", "af_unpack_microbatch"]
+           "af_token_logprob_shard", "af_merge_logprob_shards", "af_policy_update", "af_unpack_microbatch", "af_policy_loss_backward_shard"]
 MAX_WRITE_COLS = 4
 
 
@@ -117,6 +117,7 @@ def load_library() -> C.CDLL:
     lib.af_merge_logprob_shards.argtypes = [vp, vp, vp, i32, i64, i32, vp, vp, vp, vp]
     lib.af_policy_update.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i64, i32, i32, C.POINTER(LossParams), vp,
                                      vp, vp, vp, vp, vp, vp, i32, vp]
+    lib.af_policy_loss_backward_shard.argtypes = [vp, vp, vp, vp, vp, vp, i64, i32, i32, i32, vp, vp, i32, vp]
     lib.af_unpack_microbatch.argtypes = [vp, vp, i64, vp, i32, C.POINTER(WriteCols), C.POINTER(ControllerView), u32,
                                          C.POINTER(i64), vp]
     for name in EXPORTS:
@@ -283,6 +284,16 @@ class Context:
                                                 _ptr(d_W), int(accumulate_dW), _stream(stream)),
                "af_policy_loss_backward")
 
+
+    def policy_loss_backward_shard(self, hidden, W_shard, target, lse, dlogp, v_offset, d_hidden_partial, d_W_shard,
+                                   accumulate_dW=False, T=None, stream=None):
+        T = hidden.shape[0] if T is None else T
+        d, Vs = W_shard.shape[1], W_shard.shape[0]
+        _check(self.lib.af_policy_loss_backward_shard(self.handle, _ptr(hidden), _ptr(W_shard), _ptr(target),
+                                                      _ptr(lse), _ptr(dlogp), T, d, Vs, v_offset,
+                                                      _ptr(d_hidden_partial), _ptr(d_W_shard), int(accumulate_dW),
+                                                      _stream(stream)),
+               "af_policy_loss_backward_shard")
 
     def policy_update(self, hidden, W, target, old_logp, ref_logp, adv_seq, cu_seqlens, out, logp, lse, d_hidden,
                       d_W, entropy=None, dlogp=None, accumulate_dW=False, clip_lo=0.2, clip_hi=0.2, kl_coef=0.04,

@@ -377,6 +377,23 @@ af_status af_policy_loss_backward(af_ctx* c, const void* hidden, const void* W, 
                          accumulate_dW ? 1 : 0, static_cast<cudaStream_t>(stream));
 }
 
+af_status af_policy_loss_backward_shard(af_ctx* c, const void* hidden, const void* W_shard, const int32_t* target,
+                                        const float* lse, const float* dlogp, int64_t T, int32_t d, int32_t V_shard,
+                                        int32_t v_offset, void* d_hidden_partial, float* d_W_shard,
+                                        int32_t accumulate_dW, void* stream) {
+  if (!c || T < 0 || d < 1 || V_shard < 1 || v_offset < 0) return AF_ERR_INVALID_ARG;
+  if (!hidden || !W_shard || !target || !lse || !dlogp || !d_hidden_partial || !d_W_shard) {
+    if (T > 0 || !d_W_shard) return AF_ERR_INVALID_ARG;
+  }
+  if (T >= ((int64_t)1 << 31)) return AF_ERR_SHAPE;
+  if (d % 8 != 0 || V_shard % 8 != 0) return AF_ERR_ALIGNMENT;
+  if (!aligned16(hidden) || !aligned16(W_shard) || !aligned16(d_hidden_partial) || !aligned16(d_W_shard))
+    return AF_ERR_ALIGNMENT;
+  DeviceGuard guard(c->device);
+  return launch_backward(c, hidden, W_shard, target, lse, dlogp, T, d, V_shard, d_hidden_partial, d_W_shard,
+                         accumulate_dW ? 1 : 0, static_cast<cudaStream_t>(stream), v_offset);
+}
+
 static bool table_ok(const af_controller_view* t) {
   return t && t->n_samples >= 0 && (t->n_samples == 0 || (t->ready && t->consumed));
 }

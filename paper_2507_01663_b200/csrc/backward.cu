@@ -67,6 +67,7 @@ struct DzEpi {
     const float* g;         // [rows] dL/dlogp
     __nv_bfloat16* dz;      // [rows, V]
     int rows, V;
+    int v_offset;           // vocabulary id of W's first row (0 unless W is one shard of the head)
   };
   struct State {
     float g, nl;
@@ -77,7 +78,7 @@ struct DzEpi {
     if (row < p.rows) {
       st.g = __ldg(p.g + row);
       st.nl = -__ldg(p.lse + row) * kLog2e;
-      st.y = __ldg(p.target + row);
+      st.y = __ldg(p.target + row) - p.v_offset;   // outside [0, V): no column of this W matches
     } else {
       st.g = 0.f; st.nl = 0.f; st.y = -1;
     }
@@ -204,7 +205,7 @@ int64_t backward_token_block(const af_ctx* ctx, int64_t T) {
 
 af_status launch_backward(af_ctx* ctx, const void* hidden, const void* W, const int32_t* target,
                           const float* lse, const float* dlogp, int64_t T, int32_t d, int32_t V,
-                          void* d_hidden, float* d_W, int32_t accumulate_dW, cudaStream_t s) {
+                          void* d_hidden, float* d_W, int32_t accumulate_dW, cudaStream_t s, int32_t v_offset) {
   const int64_t Tc = backward_token_block(ctx, T);
   const GemmEnv env = gemm_env(ctx);
   af_status st;
@@ -225,7 +226,7 @@ af_status launch_backward(af_ctx* ctx, const void* hidden, const void* W, const 
     const Operand Hblk{H + t0 * d, tc, (uint64_t)d, dB};
     const Operand Wop{W, (uint64_t)V, (uint64_t)d, dB};
     // 1. dZ block:  Z = H_blk W^T, both K-major
-    DzEpi::Params p1{target + t0, lse + t0, dlogp + t0, dz, (int)tc, V};
+    DzEpi::Params p1{target + t0, lse + t0, dlogp + t0, dz, (int)tc, V, v_offset};
     st = run_gemm<DzEpi, false, false>(env, Hblk, Wop,
                                        logprob_pick_splits((int64_t)tc, d, V, ctx->sm_count, env.pair, ctx->v_splits), p1, s);
     if (st != AF_OK) return st;

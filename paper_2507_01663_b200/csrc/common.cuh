@@ -123,6 +123,7 @@ af_status launch_policy_update(af_ctx* ctx, const void* hidden, const void* W, c
 
 af_status launch_backward(af_ctx* ctx, const void* hidden, const void* W, const int32_t* target,
                           const float* lse, const float* dlogp, int64_t T, int32_t d, int32_t V,
-                          void* d_hidden, float* d_W, int32_t accumulate_dW, cudaStream_t s);
+                          void* d_hidden, float* d_W, int32_t accumulate_dW, cudaStream_t s,
+                          int32_t v_offset = 0);
 
 }  // namespace af

@@ -131,6 +131,12 @@ def _vocab_worker(rank, world, port, out_dir):
     ref = O.token_logprob_ref(H, W, y)
     ok = all(np.allclose(a, b, atol=1e-12) for a, b in zip((logp, ent, lse), ref))
     ok = ok and gathered.shape == (world, H.shape[0], 4)
+    # backward of the sharded head: the ranks' dH contributions are summed, dW rows stay local
+    g = np.random.default_rng(3).standard_normal(H.shape[0]) / H.shape[0]
+    dH_part, dW_rows = O.policy_loss_backward_shard_ref(H, W[lo:hi], y, lse, g, lo)
+    dH = bench.allreduce_sum_(torch.from_numpy(dH_part.copy()), world).numpy()
+    dH_ref, dW_ref = O.policy_loss_backward_ref(H, W, y, ref[2], g)
+    ok = ok and np.allclose(dH, dH_ref, atol=1e-12) and np.allclose(dW_rows, dW_ref[lo:hi], atol=1e-12)
     los = [bench.vocab_shard(w.V, world, r) for r in range(world)]
     ok = ok and los[0][0] == 0 and los[-1][1] == w.V and all(a[1] == b[0] for a, b in zip(los[:-1], los[1:]))
     with open(os.path.join(out_dir, f"ok_vocab_{rank}"), "w") as f:

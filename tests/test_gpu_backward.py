@@ -158,3 +158,57 @@ def test_host_argument_errors(ctx):
     with pytest.raises(AfError) as e:
         ctx.policy_loss_backward(H, W, y, v, v, torch.zeros_like(H), torch.zeros(12, 16, device=dev))
     assert e.value.status == -3
+
+
+@pytest.mark.parametrize("cuts", [[0, 8192], [0, 3000, 8192], [0, 8, 264, 4096, 8184, 8192]])
+def test_vocabulary_shards_of_the_backward(ctx, cuts):
+    """The head split by vocabulary rows: every shard's dH contribution and dW rows against the
+    oracle's shard backward; the contributions add up to the unsharded call's dH, the rows stack to
+    its dW."""
+    dev = device()
+    w = wl.make_workload("cfg4_mini")                       # d = 512, V = 8192
+    H, W, y = wl.gen_hidden(w), wl.gen_weight(w), wl.gen_target(w)
+    T = H.shape[0]
+    g = wl.normal01(w.seed, wl.S_G, 0, T) / T
+    _, _, lse = O.token_logprob_ref(wl.bf16_bits(H), wl.bf16_bits(W), y.numpy())
+    Hd, Wd, yd, gd, lsed = H.to(dev), W.to(dev), y.to(dev), g.to(dev), f32(lse)
+    ctx.set_tuning(0, 256, VARIANT)
+    dH_sum = np.zeros((T, w.d))
+    rows = []
+    for a, b in zip(cuts[:-1], cuts[1:]):
+        dH_p = torch.full((T, w.d), 7.0, dtype=torch.bfloat16, device=dev)
+        dW_s = torch.full((b - a, w.d), 7.0, device=dev)
+        ctx.policy_loss_backward_shard(Hd, Wd[a:b].contiguous(), yd, lsed, gd, a, dH_p, dW_s)
+        dH_ref, dW_ref = O.policy_loss_backward_shard_ref(wl.bf16_bits(H), wl.bf16_bits(W[a:b]), y.numpy(), lse,
+                                                          g.numpy(), a)
+        nH, nW = np.linalg.norm(dH_ref), np.linalg.norm(dW_ref)
+        assert np.linalg.norm(np_of(dH_p.float()) - dH_ref) <= GRAD_RTOL * nH
+        assert np.linalg.norm(np_of(dW_s) - dW_ref) <= GRAD_RTOL * nW
+        dH_sum += np_of(dH_p.float())
+        rows.append(np_of(dW_s))
+    dH_full = torch.empty(T, w.d, dtype=torch.bfloat16, device=dev)
+    dW_full = torch.empty(w.V, w.d, device=dev)
+    ctx.policy_loss_backward(Hd, Wd, yd, lsed, gd, dH_full, dW_full)
+    flags = ctx.check_device_errors()
+    ctx.set_tuning(0, 0)
+    assert flags == 0
+    ref_H, ref_W = O.policy_loss_backward_ref(wl.bf16_bits(H), wl.bf16_bits(W), y.numpy(), lse, g.numpy())
+    compare(dH_sum, np.concatenate(rows), ref_H, ref_W)
+    # each dW row is computed from the same dZ column whichever shard it sits in
+    assert np.abs(np.concatenate(rows) - np_of(dW_full)).max() <= 1e-6 * np.abs(np_of(dW_full)).max() + 1e-12
+    assert np.linalg.norm(dH_sum - np_of(dH_full.float())) <= GRAD_RTOL * np.linalg.norm(ref_H)
+
+
+def test_shard_backward_argument_errors(ctx):
+    from paper_2507_01663_b200 import binding as B
+    dev = device()
+    H = torch.zeros(4, 8, dtype=torch.bfloat16, device=dev)
+    z4 = torch.zeros(4, device=dev)
+    y = torch.zeros(4, dtype=torch.int32, device=dev)
+    with pytest.raises(B.AfError):                       # shard rows must be a multiple of 8
+        ctx.policy_loss_backward_shard(H, torch.zeros(12, 8, dtype=torch.bfloat16, device=dev), y, z4, z4, 0,
+                                       torch.zeros_like(H), torch.zeros(12, 8, device=dev))
+    with pytest.raises(B.AfError):                       # negative offset
+        ctx.policy_loss_backward_shard(H, torch.zeros(16, 8, dtype=torch.bfloat16, device=dev), y, z4, z4, -8,
+                                       torch.zeros_like(H), torch.zeros(16, 8, device=dev))
+    assert ctx.check_device_errors() == 0
