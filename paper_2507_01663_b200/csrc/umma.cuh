@@ -376,8 +376,10 @@ constexpr int kPairBM = 256;                                  // rows of A per p
 constexpr int kPairStages = 6;
 constexpr unsigned int kClockWindow = 1;                      // ticks a pair may start ahead of the slowest pair
 constexpr int kClockTickKBlocks = 64;                         // K blocks per tick when a tile has more than 96
-constexpr unsigned long long kClockPatienceNs = 200000ull;    // longest wait on the tile clock before leaving it,
+constexpr unsigned long long kClockPatienceNs = 200000ull;    // longest single wait on the tile clock,
 constexpr unsigned long long kClockPatiencePerKBlockNs = 2000ull;  // plus this per K block of a tick (~5 tick times)
+constexpr unsigned int kClockRestTicks = 16;                  // ticks a pair goes unpaced after a wait that ran out
+constexpr int kClockQuickRetries = 8;                         // waits in a row that may run out before the rests double
 constexpr int kPairBBytes = (kBN / 2) * kBK * 2;              // this CTA's half of the B tile
 constexpr int kPairStageBytes = kABytes + kPairBBytes;        // 32 KB
 constexpr int kPairSmemBytes = kPairStages * kPairStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
@@ -492,10 +494,16 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
       // that only met at tile starts drifted far enough apart to lose each other's tiles in L2).
       // The clock counts ticks over all pairs; a pair starts tick j only when all have started tick
       // j - kClockWindow.  It is a hint, not a dependency: a pair that waits longer than its patience
-      // (pairs not co-resident, say) leaves the clock for the rest of the launch, counting as
-      // finished so that nobody waits for it.
+      // goes on without the others for kClockRestTicks ticks (still counting its own), then waits
+      // again.  A pair that was held up for a while (one launch in a few hundred sees some SMs
+      // stall for a fraction of a millisecond) is caught up with that way, `patience` at a time;
+      // before, the pairs left the clock for the rest of the launch and a single stall cost a
+      // 200 ms launch 40 ms.  Waits that keep running out (pairs that are not co-resident) are
+      // spaced further and further apart.
       unsigned int my_ticks = 0;
-      bool clock_on = tile_clock != nullptr && rank == 0;
+      unsigned int skip_until = 0;                                  // no waiting before this tick
+      int misses = 0;                                               // waits in a row that ran out
+      const bool clock_on = tile_clock != nullptr && rank == 0;
       const int tick_len = g.k_blocks <= 96 ? g.k_blocks : kClockTickKBlocks;
       int to_next_tick = 0;                                         // K blocks until the next tick
       const unsigned long long patience = kClockPatienceNs + kClockPatiencePerKBlockNs * (unsigned long long)tick_len;
@@ -513,19 +521,27 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
           for (int kb = 0; kb < g.k_blocks; ++kb) {
             if (clock_on && to_next_tick-- == 0) {
               to_next_tick = tick_len - 1;
-              if (my_ticks >= kClockWindow) {
+              if (my_ticks >= kClockWindow && my_ticks >= skip_until) {
                 const unsigned int need = (unsigned int)n_pairs * (my_ticks - kClockWindow + 1);
                 const unsigned long long t0 = globaltimer_ns();
                 unsigned int seen;
+                bool ran_out = false;
                 for (;;) {
                   asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(tile_clock) : "memory");
                   if (seen >= need) break;
-                  if (globaltimer_ns() - t0 > patience) { clock_on = false; break; }
+                  if (globaltimer_ns() - t0 > patience) { ran_out = true; break; }
                   __nanosleep(100);
                 }
+                if (ran_out) {
+                  ++misses;
+                  const int doublings = misses <= kClockQuickRetries ? 0 : (misses - kClockQuickRetries < 16 ? misses - kClockQuickRetries : 16);
+                  skip_until = my_ticks + (kClockRestTicks << doublings);
+                } else {
+                  misses = 0;
+                }
               }
-              if (clock_on) { atomicAdd(tile_clock, 1u); ++my_ticks; }
-              else if (clock_most > my_ticks) atomicAdd(tile_clock, clock_most - my_ticks);
+              atomicAdd(tile_clock, 1u);
+              ++my_ticks;
             }
             if (!mbar_wait(empty_bar(stage), phase ^ 1u, &abort_flag)) { ok = false; break; }
             const uint32_t a_dst = tiles + stage * kPairStageBytes;
