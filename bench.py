@@ -37,10 +37,10 @@ UNIT = "tokens/s"
 KERNELS_PER_STEP = 7  # advantage, pack table fetch, pack columns, pack rows (bulk copy), fused LM-head GEMM, partial merge, loss
 # DRAM bytes per scored token of the fused LM-head kernel (dram__bytes_read + dram__bytes_write of
 # one ncu capture of the CTA-pair kernel at T = 65536, d = 3584, V = 152064 with the three
-# vocabulary ranges the library picks at the bench size: 13.722 GB + 9.3 MB; traffic grows with the
+# vocabulary ranges the library picks at the bench size: 13.752 GB + 8.5 MB; traffic grows with the
 # number of waves of row tiles, i.e. in proportion to T).  Valid for the 7B head shape only; None whenever the kernel
 # or its work decomposition has changed since the counters were taken.
-GEMM_DRAM_BYTES_PER_TOKEN_7B = (13.721580e9 + 9.26e6) / 65536
+GEMM_DRAM_BYTES_PER_TOKEN_7B = (13.752132e9 + 8.53e6) / 65536
 BWD_TOKEN_BLOCK = 9472  # the library's default backward block (3 GEMM launches per block)
 
 
