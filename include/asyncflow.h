@@ -157,14 +157,14 @@ af_status af_token_logprob(af_ctx* ctx, const void* hidden, const void* W, const
  * af_token_logprob_shard / af_merge_logprob_shards -- the same scoring with the LM head split by
  * vocabulary rows over model-parallel ranks.
  *
- * The paper's instances combine tensor parallelism with the other strategies (Section 2.1) and
- * says nothing about the head; these two calls are what a vocabulary-parallel head needs on this
- * path.  Rank r holds the rows [v_offset, v_offset + V_shard) of W and computes, per token, the
+ * The paper's instances combine tensor parallelism with the other strategies (Section 2.1); it
+ * says nothing about the head.  These two calls are what a vocabulary-parallel head needs on the
+ * forward path (af_policy_loss_backward_shard is their counterpart for the actor update).  Rank r holds the rows [v_offset, v_offset + V_shard) of W and computes, per token, the
  * four statistics of its logits z_v = hidden[t,:] . W_shard[v,:]:
  *     m = max_v z_v,  s = sum_v exp(z_v - m),  u = sum_v exp(z_v - m) z_v,
  *     zy = z at the target if target[t] lies in the shard, else -inf
  * written as partial_out[t] = (m, s, u, zy), fp32, [T][4], 16-byte aligned.  The ranks exchange
- * these 16 bytes per token (an all-gather; the only collective of the path) into partials
+ * these 16 bytes per token (one all-gather) into partials
  * [R][T][4], and af_merge_logprob_shards gives, with M = max_r m_r, S = sum_r s_r e^{m_r - M},
  * U = sum_r u_r e^{m_r - M}:  lse = M + log S,  logp = max_r zy_r - lse,  entropy = lse - U / S
  * -- the full-vocabulary result of af_token_logprob up to fp32 rounding.  target holds global ids;
