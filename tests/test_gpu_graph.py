@@ -188,7 +188,9 @@ def test_replay_of_a_launch_bound_scoring_step(ctx):
         torch.cuda.synchronize()
         return e0.elapsed_time(e1) * 1e3 / n
 
-    plain, replay = avg_us(lambda: st.run(scoring_only=True)), avg_us(graph.replay)
+    # best of three: a timing comparison should not depend on one disturbed loop
+    plain = min(avg_us(lambda: st.run(scoring_only=True)) for _ in range(3))
+    replay = min(avg_us(graph.replay) for _ in range(3))
     print(f"cfg1 scoring step: plain calls {plain:.1f} us, graph replay {replay:.1f} us")
     assert replay <= plain * 1.1
     assert ctx.check_device_errors() == 0
