@@ -5,7 +5,9 @@
 //   owns 4 consecutive rewards of each of four groups (G <= 16) or 16 rewards of one group
 //   (G >= 32), the adjacent lanes of a group combine their sums with shuffles, four independent
 //   128-bit loads are in flight per thread;
-//   other G <= 32: one thread per group, registers;
+//   other G <= 16: one thread per group, registers;
+//   other G <= 512: a warp stages a run of whole groups in its slice of shared memory, a team of
+//   lanes takes each group into registers, the slice streams out again (no block-wide barrier);
 //   G <= 4096: a block stages a run of whole groups in shared memory with 128-bit loads, reduces
 //   each group with warp shuffles (two passes: mean, then squared deviations) and writes the
 //   advantages back coalesced;  larger groups: one block per group.
@@ -181,6 +183,92 @@ __global__ void __launch_bounds__(kThreads) advantage_wide_kernel(
   }
 }
 
+// Any group size up to 512 (used for 16 < G <= 512 that are not a power of two).  A warp copies
+// a run of whole groups -- 32 / team of them, at most 512 rewards -- into its own slice of shared
+// memory with coalesced 128-bit streaming loads, `team` adjacent lanes (a power of two, at most 16
+// rewards per lane) take one group each from there into registers, do the arithmetic of the
+// kernels above and put the advantages back, and the warp streams the slice out again.  Only
+// __syncwarp: warps do not wait for one another.
+constexpr int kWarpStage = 512;          // rewards per warp slice
+constexpr int kAnyPerLane = 16;
+template <bool kLanePerGroup>             // team == 1
+__global__ void __launch_bounds__(kThreads, 4) advantage_any_kernel(
+    const float* __restrict__ reward, float* __restrict__ adv, int64_t n_groups, int G, int team, float eps, int ddof) {
+  __shared__ __align__(16) float stage[(kThreads / 32) * kWarpStage];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  float* s = stage + warp * kWarpStage;
+  const int gw = 32 / team;                                   // groups per warp iteration
+  const int g = lane / team, t = lane & (team - 1);
+  const int chunk = gw * G;                                   // <= kWarpStage
+  const bool vec = (chunk & 3) == 0;                          // every full chunk then starts 16-byte aligned
+  const double inv_g = 1.0 / (double)G;
+  const float inv_denom = G - ddof > 0 ? 1.f / (float)(G - ddof) : 0.f;
+  // one lane per group and an even G: lanes would read the same bank; start each lane's walk
+  // through its group at a different element instead
+  const int rot = (kLanePerGroup && (G & 1) == 0) ? g % G : 0;
+  // element i of this lane's share of its group: its position in the group, or -1
+  auto pos = [&](int i, bool live) -> int {
+    int j;
+    bool ok;
+    if (kLanePerGroup) { j = i + rot; if (j >= G) j -= G; ok = i < G; }
+    else { j = t + i * team; ok = j < G; }
+    return ok && live ? j : -1;
+  };
+  const int64_t n_iter = (n_groups + gw - 1) / gw;
+  const int64_t warps = (int64_t)gridDim.x * (kThreads / 32);
+  for (int64_t it = (int64_t)blockIdx.x * (kThreads / 32) + warp; it < n_iter; it += warps) {
+    const int64_t g0 = it * gw;
+    const int ng = (int)((n_groups - g0) < gw ? (n_groups - g0) : gw);
+    const int cnt = ng * G;
+    const float* src = reward + g0 * G;
+    float* dst = adv + g0 * G;
+    if (vec && cnt == chunk) {
+      for (int i = lane; i < (chunk >> 2); i += 32)
+        reinterpret_cast<float4*>(s)[i] = __ldcs(reinterpret_cast<const float4*>(src) + i);
+    } else {
+      for (int i = lane; i < cnt; i += 32) s[i] = __ldcs(src + i);
+    }
+    __syncwarp();
+    const bool live = g < ng;
+    float* mine = s + g * G;
+    float r[kAnyPerLane];
+    double sum = 0.0;
+#pragma unroll
+    for (int i = 0; i < kAnyPerLane; ++i) {
+      const int j = pos(i, live);
+      r[i] = j >= 0 ? mine[j] : 0.f;
+      sum += (double)r[i];
+    }
+    for (int o = team >> 1; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    const double mu = sum * inv_g;
+    const float mu_hi = (float)mu;
+    const float mu_lo = (float)(mu - (double)mu_hi);
+    float q = 0.f;
+#pragma unroll
+    for (int i = 0; i < kAnyPerLane; ++i) {
+      r[i] = pos(i, live) >= 0 ? (r[i] - mu_hi) - mu_lo : 0.f;
+      q = fmaf(r[i], r[i], q);
+    }
+    for (int o = team >> 1; o > 0; o >>= 1) q += __shfl_xor_sync(0xffffffffu, q, o);
+    const float var = q * inv_denom;
+    const float sigma = var > 0.f ? var * rsqrtf(var) : 0.f;
+    const float inv = __frcp_rn(sigma + eps);
+#pragma unroll
+    for (int i = 0; i < kAnyPerLane; ++i) {
+      const int j = pos(i, live);
+      if (j >= 0) mine[j] = r[i] * inv;
+    }
+    __syncwarp();
+    if (vec && cnt == chunk) {
+      for (int i = lane; i < (chunk >> 2); i += 32)
+        __stcs(reinterpret_cast<float4*>(dst) + i, reinterpret_cast<const float4*>(s)[i]);
+    } else {
+      for (int i = lane; i < cnt; i += 32) __stcs(dst + i, s[i]);
+    }
+    __syncwarp();                                             // the slice is refilled next
+  }
+}
+
 // Groups of equal size G, G <= kStage: each block iteration owns `gpb` whole groups.
 __global__ void __launch_bounds__(kThreads) advantage_contiguous_kernel(
     const float* __restrict__ reward, float* __restrict__ adv, int64_t n_groups, int G, int gpb,
@@ -297,6 +385,17 @@ cudaError_t launch_advantage(const float* reward, const int32_t* group_id, int64
       advantage_pow2_kernel<<<(int)blocks, kThreads, 0, s>>>(reinterpret_cast<const float4*>(reward),
                                                              reinterpret_cast<float4*>(adv), n_vec, (int)G,
                                                              eps_adv, ddof);
+    } else if (G > 16 && G <= 512 && aligned) {
+      // (smaller groups fill too little of a warp's slice: one thread per group is faster there)
+      int team = 1;
+      while (team * kAnyPerLane < G) team <<= 1;                     // 1, 2, 4, ... 32
+      const int64_t n_iter = (n_groups + 32 / team - 1) / (32 / team);
+      int64_t blocks = (n_iter + kThreads / 32 - 1) / (kThreads / 32);
+      if (blocks > (int64_t)1 << 30) blocks = (int64_t)1 << 30;
+      if (team == 1)
+        advantage_any_kernel<true><<<(int)blocks, kThreads, 0, s>>>(reward, adv, n_groups, (int)G, team, eps_adv, ddof);
+      else
+        advantage_any_kernel<false><<<(int)blocks, kThreads, 0, s>>>(reward, adv, n_groups, (int)G, team, eps_adv, ddof);
     } else if (G >= 1 && G <= kSmallG) {
       const int vec_ok = (G % 4 == 0) && ((reinterpret_cast<uintptr_t>(reward) & 15) == 0) &&
                          ((reinterpret_cast<uintptr_t>(adv) & 15) == 0);

@@ -41,7 +41,7 @@ def test_advantage_workload_rewards(ctx, name, ddof):
     assert ctx.check_device_errors() == 0
 
 
-@pytest.mark.parametrize("G", [1, 2, 3, 4, 5, 8, 16, 31, 32, 33, 64, 100, 128, 256, 512, 1000, 1024, 5000])
+@pytest.mark.parametrize("G", [1, 2, 3, 4, 5, 8, 16, 17, 24, 31, 32, 33, 48, 64, 100, 128, 256, 300, 511, 512, 513, 1000, 1024, 5000])
 def test_advantage_group_sizes(ctx, G):
     n_groups = 37 if G < 1000 else 3
     N = G * n_groups
@@ -52,7 +52,7 @@ def test_advantage_group_sizes(ctx, G):
     assert np.abs(np_of(adv) - ref).max() <= ADV_TOL
 
 
-@pytest.mark.parametrize("G", [4, 8, 16, 32, 64, 128, 512, 6, 200])
+@pytest.mark.parametrize("G", [4, 8, 16, 32, 64, 128, 512, 6, 24, 200, 500])
 def test_advantage_of_nearly_equal_rewards(ctx, G):
     """Rewards of a group a few units in the last place apart: the deviations (~1e-8..1e-6) are of the
     size of eps, so the mean must be right to far below an fp32 ulp for the advantages to be."""
