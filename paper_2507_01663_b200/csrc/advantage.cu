@@ -5,7 +5,8 @@
 //   owns 4 consecutive rewards of each of four groups (G <= 16) or 16 rewards of one group
 //   (G >= 32), the adjacent lanes of a group combine their sums with shuffles, four independent
 //   128-bit loads are in flight per thread;
-//   other G <= 16: one thread per group, registers;
+//   other G < 16: a kernel per group size (a lane owns 16 / G whole groups, staged through a
+//   warp-private slice of shared memory); G = 1, 2 and unaligned buffers: one thread per group;
 //   other G <= 512: a warp stages a run of whole groups in its slice of shared memory, a team of
 //   lanes takes each group into registers, the slice streams out again (no block-wide barrier);
 //   G <= 4096: a block stages a run of whole groups in shared memory with 128-bit loads, reduces
@@ -181,6 +182,88 @@ __global__ void __launch_bounds__(kThreads) advantage_wide_kernel(
         __stcs(adv + gv + k * team, make_float4(r[k].x * inv, r[k].y * inv, r[k].z * inv, r[k].w * inv));
     }
   }
+}
+
+// Group sizes below 16 that are not a power of two, known at compile time.  A lane owns
+// M = 16 / G whole groups (E = M G rewards); a warp copies 32 E consecutive rewards into its slice
+// of shared memory with coalesced 128-bit streaming loads, placing lane l's share at l * (E | 1)
+// (an odd stride: the lanes then read and write different banks), works on registers with every
+// loop unrolled, and streams the advantages out the same way.  Arithmetic as in the kernels above.
+template <int G>
+__global__ void __launch_bounds__(kThreads) advantage_fixed_kernel(
+    const float* __restrict__ reward, float* __restrict__ adv, int64_t n_groups, float eps, int ddof) {
+  constexpr int M = 16 / G, E = M * G, EP = E | 1, CH = 32 * E;
+  __shared__ float stage[(kThreads / 32) * 32 * EP];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  float* s = stage + warp * 32 * EP;
+  const double inv_g = 1.0 / (double)G;
+  const float inv_denom = G - ddof > 0 ? 1.f / (float)(G - ddof) : 0.f;
+  const int64_t n_iter = (n_groups + 32 * M - 1) / (32 * M);
+  const int64_t warps = (int64_t)gridDim.x * (kThreads / 32);
+  for (int64_t it = (int64_t)blockIdx.x * (kThreads / 32) + warp; it < n_iter; it += warps) {
+    const int64_t g0 = it * 32 * M;
+    const int64_t left = (n_groups - g0) * G;                 // rewards from here to the end
+    const int cnt = left < CH ? (int)left : CH;
+    const float* src = reward + g0 * G;                       // 128 E bytes per iteration: 16-byte aligned
+    float* dst = adv + g0 * G;
+    if (cnt == CH) {
+#pragma unroll
+      for (int i = lane; i < CH / 4; i += 32) {
+        const float4 v = __ldcs(reinterpret_cast<const float4*>(src) + i);
+        const int f = 4 * i;
+        s[(f / E) * EP + f % E] = v.x;
+        s[((f + 1) / E) * EP + (f + 1) % E] = v.y;
+        s[((f + 2) / E) * EP + (f + 2) % E] = v.z;
+        s[((f + 3) / E) * EP + (f + 3) % E] = v.w;
+      }
+    } else {
+      for (int f = lane; f < cnt; f += 32) s[(f / E) * EP + f % E] = __ldcs(src + f);
+    }
+    __syncwarp();
+    float* mine = s + lane * EP;
+#pragma unroll
+    for (int gi = 0; gi < M; ++gi) {
+      if ((int64_t)(lane * M + gi) * G < cnt) {               // this group exists (groups are whole)
+        float r[G];
+        double sum = 0.0;
+#pragma unroll
+        for (int k = 0; k < G; ++k) { r[k] = mine[gi * G + k]; sum += (double)r[k]; }
+        const double mu = sum * inv_g;
+        const float mu_hi = (float)mu;
+        const float mu_lo = (float)(mu - (double)mu_hi);
+        float q = 0.f;
+#pragma unroll
+        for (int k = 0; k < G; ++k) { r[k] = (r[k] - mu_hi) - mu_lo; q = fmaf(r[k], r[k], q); }
+        const float var = q * inv_denom;
+        const float sigma = var > 0.f ? var * rsqrtf(var) : 0.f;
+        const float inv = __frcp_rn(sigma + eps);
+#pragma unroll
+        for (int k = 0; k < G; ++k) mine[gi * G + k] = r[k] * inv;
+      }
+    }
+    __syncwarp();
+    if (cnt == CH) {
+#pragma unroll
+      for (int i = lane; i < CH / 4; i += 32) {
+        const int f = 4 * i;
+        __stcs(reinterpret_cast<float4*>(dst) + i,
+               make_float4(s[(f / E) * EP + f % E], s[((f + 1) / E) * EP + (f + 1) % E],
+                           s[((f + 2) / E) * EP + (f + 2) % E], s[((f + 3) / E) * EP + (f + 3) % E]));
+      }
+    } else {
+      for (int f = lane; f < cnt; f += 32) __stcs(dst + f, s[(f / E) * EP + f % E]);
+    }
+    __syncwarp();                                             // the slice is refilled next
+  }
+}
+
+template <int G>
+void launch_advantage_fixed(const float* reward, float* adv, int64_t n_groups, float eps, int ddof, cudaStream_t s) {
+  constexpr int M = 16 / G;
+  const int64_t n_iter = (n_groups + 32 * M - 1) / (32 * M);
+  int64_t blocks = (n_iter + kThreads / 32 - 1) / (kThreads / 32);
+  if (blocks > (int64_t)1 << 30) blocks = (int64_t)1 << 30;
+  advantage_fixed_kernel<G><<<(int)blocks, kThreads, 0, s>>>(reward, adv, n_groups, eps, ddof);
 }
 
 // Any group size up to 512 (used for 16 < G <= 512 that are not a power of two).  A warp copies
@@ -385,6 +468,20 @@ cudaError_t launch_advantage(const float* reward, const int32_t* group_id, int64
       advantage_pow2_kernel<<<(int)blocks, kThreads, 0, s>>>(reinterpret_cast<const float4*>(reward),
                                                              reinterpret_cast<float4*>(adv), n_vec, (int)G,
                                                              eps_adv, ddof);
+    } else if (aligned && (G == 3 || (G >= 5 && G <= 7) || (G >= 9 && G <= 15))) {
+      switch ((int)G) {
+        case 3: launch_advantage_fixed<3>(reward, adv, n_groups, eps_adv, ddof, s); break;
+        case 5: launch_advantage_fixed<5>(reward, adv, n_groups, eps_adv, ddof, s); break;
+        case 6: launch_advantage_fixed<6>(reward, adv, n_groups, eps_adv, ddof, s); break;
+        case 7: launch_advantage_fixed<7>(reward, adv, n_groups, eps_adv, ddof, s); break;
+        case 9: launch_advantage_fixed<9>(reward, adv, n_groups, eps_adv, ddof, s); break;
+        case 10: launch_advantage_fixed<10>(reward, adv, n_groups, eps_adv, ddof, s); break;
+        case 11: launch_advantage_fixed<11>(reward, adv, n_groups, eps_adv, ddof, s); break;
+        case 12: launch_advantage_fixed<12>(reward, adv, n_groups, eps_adv, ddof, s); break;
+        case 13: launch_advantage_fixed<13>(reward, adv, n_groups, eps_adv, ddof, s); break;
+        case 14: launch_advantage_fixed<14>(reward, adv, n_groups, eps_adv, ddof, s); break;
+        default: launch_advantage_fixed<15>(reward, adv, n_groups, eps_adv, ddof, s); break;
+      }
     } else if (G > 16 && G <= 512 && aligned) {
       // (smaller groups fill too little of a warp's slice: one thread per group is faster there)
       int team = 1;

@@ -41,18 +41,20 @@ def test_advantage_workload_rewards(ctx, name, ddof):
     assert ctx.check_device_errors() == 0
 
 
-@pytest.mark.parametrize("G", [1, 2, 3, 4, 5, 8, 16, 17, 24, 31, 32, 33, 48, 64, 100, 128, 256, 300, 511, 512, 513, 1000, 1024, 5000])
+@pytest.mark.parametrize("G", [1, 2, 3, 4, 5, 6, 7, 8, 9, 10, 11, 12, 13, 14, 15, 16, 17, 24, 31, 32, 33, 48, 64, 100, 128, 256, 300, 511, 512, 513, 1000, 1024, 5000])
 def test_advantage_group_sizes(ctx, G):
-    n_groups = 37 if G < 1000 else 3
-    N = G * n_groups
-    r = wl.uniform01(G, wl.S_REWARD, 0, N, device())
-    ref = O.grpo_advantage_ref(np_of(r), np.arange(N) // G, n_groups, 1e-6, 0)
-    adv = torch.full((N,), 9.0, device=device())
-    ctx.grpo_advantage(r, None, n_groups, adv)
-    assert np.abs(np_of(adv) - ref).max() <= ADV_TOL
+    # a handful of groups (a ragged run only) and a few thousand (full runs of every kernel plus a tail)
+    for n_groups in ((37, 4099) if G < 1000 else (3,)):
+        N = G * n_groups
+        r = wl.uniform01(G, wl.S_REWARD, 0, N, device())
+        ref = O.grpo_advantage_ref(np_of(r), np.arange(N) // G, n_groups, 1e-6, 0)
+        adv = torch.full((N + 8,), 9.0, device=device())
+        ctx.grpo_advantage(r, None, n_groups, adv[:N], N=N)
+        assert np.abs(np_of(adv[:N]) - ref).max() <= ADV_TOL
+        assert np.all(np_of(adv[N:]) == 9.0)                      # nothing written past the end
 
 
-@pytest.mark.parametrize("G", [4, 8, 16, 32, 64, 128, 512, 6, 24, 200, 500])
+@pytest.mark.parametrize("G", [4, 8, 16, 32, 64, 128, 512, 3, 6, 7, 12, 15, 24, 200, 500])
 def test_advantage_of_nearly_equal_rewards(ctx, G):
     """Rewards of a group a few units in the last place apart: the deviations (~1e-8..1e-6) are of the
     size of eps, so the mean must be right to far below an fp32 ulp for the advantages to be."""
