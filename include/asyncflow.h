@@ -190,7 +190,8 @@ af_status af_merge_logprob_shards(af_ctx* ctx, const float* partials, const int3
  * NULL for contiguous equal groups (sample i belongs to group i / (N / n_groups); then
  * N % n_groups must be 0).  With group_id given the kernel scans the id array once per group
  * (deterministic, no float atomics) and N * n_groups must stay below 2^33 (AF_ERR_SHAPE).
- * ddof is 0 or 1.  adv [N] fp32 dev.
+ * ddof is 0 or 1.  eps_adv must be > 0 (AF_ERR_INVALID_ARG otherwise: with eps_adv = 0 a group of
+ * equal rewards would divide 0 by 0).  adv [N] fp32 dev.
  * ------------------------------------------------------------------------------------------- */
 af_status af_grpo_advantage(af_ctx* ctx, const float* reward, const int32_t* group_id, int64_t N,
                             int32_t n_groups, float eps_adv, int32_t ddof, float* adv,
@@ -412,25 +413,33 @@ af_status af_balance_partitions(const int32_t* length_host, int32_t n, int32_t k
  * (The paper has no counterpart for this call; it exists for the sake of embedding.)  Some hosts
  * of this library cannot call cudaMalloc on the path that scores tokens: code running while a
  * memory pool owns the whole device, a serving loop with a frozen memory plan, a plug-in handed
- * only the buffers its caller chose to give it.  For them this entry point computes exactly what
- * af_token_logprob computes -- same kernels, same arguments, same results -- but takes no
- * context and keeps its only scratch (the per-split online-softmax partials) in a fixed array
- * inside the library's device image: 2 MiB + 256 B that every GPU loading the library holds
- * until the process exits.  It never calls cudaMalloc, cudaFree or an allocating library routine.
+ * only the buffers its caller chose to give it.  For them this entry point computes what
+ * af_token_logprob computes, with the same arguments, but takes no context and keeps its only
+ * scratch (the per-range online-softmax partials) in a fixed array inside the library's device
+ * image: 2 MiB + 256 B that every GPU loading the library holds until the process exits.  The call
+ * itself never calls cudaMalloc, cudaFree or an allocating library routine.
+ *
+ * Kernel and results: always the one-CTA-per-tile main loop (gemm_variant 1 of af_set_tuning),
+ * with the number of vocabulary ranges cut down to what the fixed array holds (4 x 32768 partials).
+ * Its results agree with af_token_logprob within the log-prob tolerance (2e-3 absolute); they are
+ * bit-equal only to a context set to gemm_variant 1 that happens to use the same number of ranges.
  *
  * Limit: 0 <= T <= 32768 tokens per call (AF_ERR_CAPACITY above that); d, V, pointers and
  * alignment as for af_token_logprob.  Runs on the current CUDA device, which must be compute
  * capability 10.0.
- * First call on a device: resolves the array's device address, reads the SM count, fetches the
- * tensor-map encoder and sets the kernel's shared-memory limit (and, with lazy module loading,
- * loads the kernels).  Make that first call before any stream capture begins.
+ * First call on a device: resolves the array's device address (cudaGetSymbolAddress), reads the SM
+ * count, fetches the tensor-map encoder and sets the kernel's shared-memory limit.  With lazy
+ * module loading this is also when the driver loads the library's kernels and materialises the
+ * array, which allocates device memory inside the driver; so make that first call during start-up,
+ * before memory is frozen and before any stream capture begins.
  * Sharing: every call on a device uses the same array.  Nothing in it has to start at zero (a
  * call overwrites each partial before reading it, so stale contents of an earlier call are
  * harmless), but two calls that overlap on the GPU -- different streams, no ordering -- race on
  * it and corrupt each other's results.  Serialise them (one stream, or events).
  * device_flags: optional device pointer to a caller-owned uint32 that receives the AF_DEVERR_*
- * bits (OR-ed in; clear it yourself).  With NULL the bits are dropped; a target outside [0, V)
- * still shows as a NaN log-prob.
+ * bits (OR-ed in; clear it yourself).  With NULL the bits are OR-ed into a word of the fixed
+ * array's header that nothing reads: they are lost, and a target outside [0, V) then shows only as
+ * a NaN log-prob.  entropy and lse are optional; a NULL one is not written.
  * ------------------------------------------------------------------------------------------- */
 af_status af_token_logprob_static(const void* hidden, const void* W, const int32_t* target,
                                   int64_t T, int32_t d, int32_t V, float* logp, float* entropy,

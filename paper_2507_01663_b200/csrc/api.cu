@@ -270,10 +270,12 @@ af_status af_unpack_microbatch(af_ctx* c, const int64_t* tok_offset_host, int64_
     return AF_ERR_INVALID_ARG;
   if (table && (table->n_samples != n_samples || (n_samples > 0 && !table->ready))) return AF_ERR_INVALID_ARG;
   // a sample may be listed once: two writers of one row would have no defined order
-  {
+  try {
     std::vector<int32_t> sorted(idx_host, idx_host + B);
     std::sort(sorted.begin(), sorted.end());
     if (std::adjacent_find(sorted.begin(), sorted.end()) != sorted.end()) return AF_ERR_INVALID_ARG;
+  } catch (...) {   // no exception may cross the C boundary (the copy of the list could not be allocated)
+    return AF_ERR_WORKSPACE;
   }
   DeviceGuard guard(c->device);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -338,7 +340,7 @@ af_status af_merge_logprob_shards(af_ctx* c, const float* partials, const int32_
 
 af_status af_grpo_advantage(af_ctx* c, const float* reward, const int32_t* group_id, int64_t N,
                             int32_t n_groups, float eps_adv, int32_t ddof, float* adv, void* stream) {
-  if (!c || N < 0 || n_groups < 0 || (ddof != 0 && ddof != 1) || !(eps_adv >= 0.f)) return AF_ERR_INVALID_ARG;
+  if (!c || N < 0 || n_groups < 0 || (ddof != 0 && ddof != 1) || !(eps_adv > 0.f)) return AF_ERR_INVALID_ARG;
   if (N == 0) return AF_OK;
   if (!reward || !adv || n_groups < 1) return AF_ERR_INVALID_ARG;
   if (!group_id && N % n_groups != 0) return AF_ERR_SHAPE;

@@ -124,6 +124,11 @@ __global__ void __launch_bounds__(kThreads, 2) policy_loss_kernel(
     bulk_load(dst + 2 * kColBytes, ref_logp + c0, nb, bar);
     if (entropy) bulk_load(dst + 3 * kColBytes, entropy + c0, nb, bar);
   };
+  // cu_seqlens must be non-decreasing (its ends are checked by the last block): every entry is
+  // compared with its successor once, spread over the grid; a violation only raises the flag --
+  // nothing below indexes memory with a value taken from cu_seqlens
+  for (int q = blockIdx.x * kThreads + threadIdx.x; q < B; q += gridDim.x * kThreads)
+    if (__ldg(cu + q) > __ldg(cu + q + 1)) atomicOr(d_err, AF_DEVERR_CU_SEQLENS);
   if (threadIdx.x == 0) {
     abort_flag = 0;
     s_first = 0; s_count = 0; s_cover = -1;

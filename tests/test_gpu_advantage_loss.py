@@ -93,6 +93,10 @@ def test_advantage_degenerate_groups(ctx):
     with pytest.raises(AfError) as e:
         ctx.grpo_advantage(r, None, 5, adv)
     assert e.value.status == -2
+    # eps_adv = 0 would turn a group of equal rewards into 0 / 0: refused
+    with pytest.raises(AfError) as e:
+        ctx.grpo_advantage(r, None, 4, adv, eps_adv=0.0)
+    assert e.value.status == -1
 
 
 # ---------------------------------------------------------------- loss
@@ -191,4 +195,34 @@ def test_loss_bad_cu_seqlens_is_flagged(ctx):
     logp, old, ref, ent = loss_inputs(w, 64, [64])
     run_loss(ctx, logp, old, ref, None, [1.0, 1.0], [0, 32, 60])      # cu[B] != T
     assert ctx.check_device_errors() & B.DEVERR_CU_SEQLENS
+    assert ctx.check_device_errors() == 0
+    run_loss(ctx, logp, old, ref, None, [1.0, 1.0], [4, 32, 64])      # cu[0] != 0
+    assert ctx.check_device_errors() & B.DEVERR_CU_SEQLENS
+    run_loss(ctx, logp, old, ref, None, [1.0, 1.0, 1.0], [0, 40, 32, 64])   # decreasing in the middle, ends right
+    assert ctx.check_device_errors() & B.DEVERR_CU_SEQLENS
+    res, _ = run_loss(ctx, logp, old, ref, None, [1.0, 1.0, 1.0], [0, 32, 32, 64])  # an empty sequence is fine
+    assert ctx.check_device_errors() == 0 and res["n_tokens"] == 64
+
+
+def test_kl_term_close_to_the_reference_policy(ctx):
+    """Late in training the policy sits close to the reference: delta = ref - logp ~ N(0, 0.01), k3 ~
+    5e-5 per token.  kl_mean and the KL part of the gradient must still meet the loss tolerance."""
+    w = wl.make_workload("cfg2_mini")
+    lens = w.lengths[:24]
+    cu = np.concatenate([[0], np.cumsum(lens)])
+    T = int(cu[-1])
+    logp, old, _, ent = loss_inputs(w, T, lens)
+    A = np_of(wl.normal01(8, wl.S_MISC, 0, 24))
+    for std in (1e-2, 1e-3, 0.3):
+        ref = logp + std * wl.normal01(w.seed, wl.S_REF, 0, T)
+        for agg_mode in (0, 1):
+            kw = dict(clip_lo=0.2, clip_hi=0.2, kl_coef=0.04, agg_mode=agg_mode, loss_scale=1.0)
+            res, g = run_loss(ctx, logp, old, ref, ent, A, cu, **kw)
+            oref = O.policy_loss_ref(logp.numpy(), old.numpy(), ref.numpy(), A, cu, entropy=ent.numpy(), **kw)
+            assert rel(res["kl_mean"], oref["kl_mean"]) <= LOSS_RTOL, (std, res["kl_mean"], oref["kl_mean"])
+            compare_loss(res, g, oref, T)
+            # the KL part of dL/dlogp alone: advantages of zero leave nothing else
+            res0, g0 = run_loss(ctx, logp, old, ref, ent, np.zeros(24, np.float32), cu, **kw)
+            o0 = O.policy_loss_ref(logp.numpy(), old.numpy(), ref.numpy(), np.zeros(24), cu, entropy=ent.numpy(), **kw)
+            assert np.abs(g0 - o0["dlogp"]).max() <= 1e-4 * np.abs(o0["dlogp"]).max()
     assert ctx.check_device_errors() == 0

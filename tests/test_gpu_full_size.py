@@ -10,7 +10,12 @@ import torch
 
 from oracle import grpo_oracle as O
 from paper_2507_01663_b200 import workloads as wl
-from gpu_util import ADV_TOL, GRAD_RTOL, LOGP_TOL, LOSS_RTOL, device, f32, i32, np_of, rel, sample_rows
+from gpu_util import (ADV_TOL, GRAD_RTOL, LOGP_TOL, LOSS_RTOL, device, f32, i32, np_of, off_the_clip_bounds, rel,
+                      sample_rows)
+
+N_ROWS = 2048        # token rows scored by the oracle per full-size batch (every row over the full vocabulary)
+N_ROWS_MB = 256      # the same per micro-batch of the streaming store
+N_VOCAB_ROWS = 256   # rows of dW formed by the oracle (each a sum over every token of the batch)
 
 pytestmark = pytest.mark.gpu
 
@@ -72,18 +77,60 @@ def check_pack_everywhere(w, store, adv, idx, out, T):
     return cu
 
 
+def vocab_rows_sample(V, targets, n, seed):
+    """Vocabulary ids for sampled rows of dW: ids that occur as targets, both sides of the 128- and
+    256-row tile edges at either end of the vocabulary, the last row, then seeded random ids."""
+    last256 = (V - 1) // 256 * 256
+    vs = {0, 127, 128, 255, 256, 257, last256 - 1, last256, last256 + 127, last256 + 128, V - 2, V - 1}
+    vs = {min(max(int(v), 0), V - 1) for v in vs}
+    vs.update(int(t) for t in targets)
+    rng = np.random.default_rng(seed)
+    while len(vs) < n:
+        vs.add(int(rng.integers(0, V)))
+    return sorted(vs)
+
+
+def token_gradient_ref(o_logp, old, ref, A, wt, clip_eps, kl_coef):
+    """dL/dlogp of the given tokens from oracle quantities only, through the oracle's loss: every
+    token becomes a sequence of its own (length 1) in token-mean mode, where the oracle's weight is
+    1/n; the token's real weight `wt` (from the batch it sits in) replaces it."""
+    n = len(o_logp)
+    r = O.policy_loss_ref(o_logp, old, ref, A, np.arange(n + 1), clip_eps, clip_eps, kl_coef, agg_mode=1, loss_scale=1.0)
+    return r["dlogp"] * n * wt, r
+
+
 def scored_chain_check(ctx, w, store, W, reward, idx, n_rows, seed, agg_mode=0):
-    """advantage -> pack -> log-prob -> loss on one micro-batch; sampled rows against the oracle."""
+    """advantage -> pack -> log-prob -> loss on one micro-batch; sampled rows against the oracle.
+    At the sampled rows the store's old / ref log-probs are, as the workload defines them, the
+    oracle's log-prob plus noise (moved off the clip bounds); elsewhere they are centred on the
+    estimate of the generator module."""
     from paper_2507_01663_b200 import binding as B
     dev = device()
+    idx = np.asarray(idx)
+    cu = np.concatenate([[0], np.cumsum(w.lengths[idx])]).astype(np.int64)
+    T_host = int(cu[-1])
+    rows = sample_rows(cu, T_host, n_rows, seed)
+    rt = torch.as_tensor(rows, device=dev)
+    seq_of = np.searchsorted(cu, rows, side="right") - 1
+    src_rows = w.tok_offset[idx[seq_of]] + (rows - cu[seq_of])          # store rows, by the definition of pack
+    src_t = torch.as_tensor(src_rows, device=dev)
+    W_bits = wl.bf16_bits(W)
+    # the oracle reads the very bits the kernel will see
+    o_logp, o_ent, o_lse = oracle_rows(store["hidden"][src_t].cpu(), W_bits, np_of(store["target"][src_t]))
+    n_old = np_of(wl.gen_noise(w, wl.S_OLD, w.total_tokens, dev)[src_t]).astype(np.float64)
+    n_ref = np_of(wl.gen_noise(w, wl.S_REF, w.total_tokens, dev)[src_t]).astype(np.float64)
+    old = off_the_clip_bounds(o_logp, (o_logp + n_old).astype(np.float32), w.clip_eps, w.clip_eps)
+    ref = (o_logp + n_ref).astype(np.float32).astype(np.float64)
+    store["old_logp"][src_t] = f32(old)
+    store["ref_logp"][src_t] = f32(ref)
+
     adv = torch.empty(w.N, device=dev)
     ctx.grpo_advantage(reward, None, w.n_prompts, adv)
     adv_ref = O.grpo_advantage_ref(np_of(reward), w.group_id, w.n_prompts)
     assert np.abs(np_of(adv) - adv_ref).max() <= ADV_TOL
-    T_cap = int(w.lengths[idx].sum())
-    out = packed_out(T_cap, len(idx), w.d, dev)
+    out = packed_out(T_host, len(idx), w.d, dev)
     T = ctx.pack_microbatch({"tok_offset_host": w.tok_offset, "d": w.d, "adv": adv, **store}, idx, out)
-    cu = check_pack_everywhere(w, store, adv, idx, out, T)
+    assert np.array_equal(check_pack_everywhere(w, store, adv, idx, out, T), cu)
     logp, ent, lse, g = (torch.empty(T, device=dev) for _ in range(4))
     ctx.token_logprob(out["hidden"], W, out["target"], logp, ent, lse)
     lo = B.new_loss_out(dev)
@@ -91,14 +138,6 @@ def scored_chain_check(ctx, w, store, W, reward, idx, n_rows, seed, agg_mode=0):
                     w.clip_eps, w.clip_eps, w.kl_coef, agg_mode, 1.0)
     res = B.read_loss_out(lo)
     assert ctx.check_device_errors() == 0
-    # sampled rows: regenerate nothing, read the very bits the kernel saw
-    rows = sample_rows(cu, T, n_rows, seed)
-    rt = torch.as_tensor(rows, device=dev)
-    W_bits = wl.bf16_bits(W)
-    seq_of = np.searchsorted(cu, rows, side="right") - 1
-    src_rows = w.tok_offset[idx[seq_of]] + (rows - cu[seq_of])          # store rows, by the definition of pack
-    src_t = torch.as_tensor(src_rows, device=dev)
-    o_logp, o_ent, o_lse = oracle_rows(store["hidden"][src_t].cpu(), W_bits, np_of(store["target"][src_t]))
     assert np.abs(np_of(logp[rt]) - o_logp).max() <= LOGP_TOL
     assert np.abs(np_of(ent[rt]) - o_ent).max() <= LOGP_TOL
     assert np.abs(np_of(lse[rt]) - o_lse).max() <= LOGP_TOL
@@ -106,13 +145,8 @@ def scored_chain_check(ctx, w, store, W, reward, idx, n_rows, seed, agg_mode=0):
     A = adv_ref[idx[seq_of]]
     L = np.diff(cu)[seq_of].astype(np.float64)
     wt = 1.0 / (len(idx) * L) if agg_mode == 0 else np.full(len(rows), 1.0 / T)
-    old, ref = np_of(store["old_logp"][src_t]).astype(np.float64), np_of(store["ref_logp"][src_t]).astype(np.float64)
-    rho = np.exp(o_logp - old)
-    s1, s2 = rho * A, np.clip(rho, 1 - w.clip_eps, 1 + w.clip_eps) * A
-    g_ref = wt * (np.where(s2 < s1, 0.0, -A * rho) + w.kl_coef * (1.0 - np.exp(ref - o_logp)))
-    near = (np.abs(rho - (1 - w.clip_eps)) < 2 * LOGP_TOL) | (np.abs(rho - (1 + w.clip_eps)) < 2 * LOGP_TOL)
-    err = np.abs(np_of(g[rt]) - g_ref)[~near]
-    assert err.max() <= 5e-3 * np.abs(g_ref).max() + 1e-12
+    g_ref, _ = token_gradient_ref(o_logp, old, ref, A, wt, w.clip_eps, w.kl_coef)
+    assert np.abs(np_of(g[rt]) - g_ref).max() <= 5e-3 * np.abs(g_ref).max() + 1e-12
     # properties at full size: finite outputs, entropy range, loss aggregates its own tokens
     lp = np_of(logp)
     assert np.isfinite(lp).all() and (lp <= 1e-5).all()
@@ -123,12 +157,12 @@ def scored_chain_check(ctx, w, store, W, reward, idx, n_rows, seed, agg_mode=0):
     return res
 
 
-@pytest.mark.parametrize("name,n_rows", [("cfg2", 192), ("cfg3", 128)])
-def test_forward_workloads_full_size(ctx, name, n_rows):
+@pytest.mark.parametrize("name", ["cfg2", "cfg3"])
+def test_forward_workloads_full_size(ctx, name):
     w = wl.make_workload(name)
     dev = device()
     store, W, reward = build_store(w, dev)
-    scored_chain_check(ctx, w, store, W, reward, wl.arrival_order(w), n_rows, seed=w.seed)
+    scored_chain_check(ctx, w, store, W, reward, wl.arrival_order(w), N_ROWS, seed=w.seed)
 
 
 def test_streaming_store_full_size(ctx):
@@ -141,7 +175,7 @@ def test_streaming_store_full_size(ctx):
     mbs = wl.microbatches(w)
     assert all(int(w.lengths[m].sum()) <= w.token_budget or len(m) == 1 for m in mbs)
     for k in (0, len(mbs) // 2, len(mbs) - 1):
-        scored_chain_check(ctx, w, store, W, reward, mbs[k], 48, seed=k)
+        scored_chain_check(ctx, w, store, W, reward, mbs[k], N_ROWS_MB, seed=k)
     # back-to-back on one stream with shared buffers: every batch ends with finite, sane scalars
     adv = torch.empty(w.N, device=dev)
     ctx.grpo_advantage(reward, None, w.n_prompts, adv)
@@ -191,10 +225,24 @@ def test_loss_stage_full_size(ctx):
     assert ctx.check_device_errors() == 0
 
 
+def dH_rows_ref(H_rows, W_bits, y_rows, lse_rows, g_rows, chunk=64):
+    """Oracle dH of the given token rows (each row needs the whole vocabulary, nothing else)."""
+    return np.concatenate([
+        O.policy_loss_backward_ref(wl.bf16_bits(H_rows[s:s + chunk]), W_bits, y_rows[s:s + chunk],
+                                   lse_rows[s:s + chunk], g_rows[s:s + chunk])[0]
+        for s in range(0, H_rows.shape[0], chunk)])
+
+
+def assert_grad_close(got, ref, what):
+    n = np.linalg.norm(ref)
+    assert abs(np.linalg.norm(got) - n) <= GRAD_RTOL * n, what          # gradient norm (the stated bar)
+    assert np.linalg.norm(got - ref) <= GRAD_RTOL * n, what            # and the direction, element-wise
+
+
 def test_backward_full_size(ctx):
     """cfg4: one 65536-token micro-batch, d = 3584, V = 152064.  dH on sampled rows and dW on
-    sampled vocabulary rows against the oracle; column sums and the <dW,W> = <dH,H> identity
-    over the whole result.  The stage's lse input is synthetic (the oracle uses the same)."""
+    sampled vocabulary rows against the oracle; the <dW,W> = <dH,H> identity over the whole result.
+    The stage's lse input is synthetic (the oracle uses the same)."""
     w = wl.make_workload("cfg4")
     dev = device()
     T = w.total_tokens
@@ -208,30 +256,18 @@ def test_backward_full_size(ctx):
     ctx.policy_loss_backward(H, W, y, lse, g, dH, dW)
     assert ctx.check_device_errors() == 0
     W_bits = wl.bf16_bits(W)
-    cu = w.tok_offset
-    rows = sample_rows(cu, T, 96, seed=1)
+    rows = sample_rows(w.tok_offset, T, N_ROWS, seed=1)
     rt = torch.as_tensor(rows, device=dev)
-    dH_ref = np.concatenate([
-        O.policy_loss_backward_ref(wl.bf16_bits(H[rt[s:s + 32]]), W_bits, np_of(y[rt[s:s + 32]]),
-                                   np_of(lse[rt[s:s + 32]]), np_of(g[rt[s:s + 32]]))[0]
-        for s in range(0, len(rows), 32)])
-    got = np_of(dH[rt].float())
-    nH = np.linalg.norm(dH_ref)
-    assert abs(np.linalg.norm(got) - nH) <= GRAD_RTOL * nH
-    assert np.linalg.norm(got - dH_ref) <= GRAD_RTOL * nH
+    dH_ref = dH_rows_ref(H[rt].cpu(), W_bits, np_of(y[rt]), np_of(lse[rt]), np_of(g[rt]))
+    assert_grad_close(np_of(dH[rt].float()), dH_ref, "dH")
     # dW rows: ids that occur as targets, tile edges, the last row
     ys = np_of(y)
-    vs = sorted({0, 127, 128, 255, 256, w.V - 1, w.V - 129, int(ys[0]), int(ys[T // 2]), int(ys[-1])}
-                | set(np.random.default_rng(2).integers(0, w.V, 54).tolist()))
+    vs = vocab_rows_sample(w.V, ys[[0, T // 2, T - 1, 255, 256]], N_VOCAB_ROWS, seed=2)
     dW_ref = O.policy_loss_backward_ref(wl.bf16_bits(H), W_bits, ys, np_of(lse), np_of(g), vocab_rows=vs)
-    gotW = np_of(dW[torch.as_tensor(vs, device=dev)])
-    nW = np.linalg.norm(dW_ref)
-    assert abs(np.linalg.norm(gotW) - nW) <= GRAD_RTOL * nW
-    assert np.linalg.norm(gotW - dW_ref) <= GRAD_RTOL * nW
-    # whole-result properties.  sum_v dZ_tv = g_t (1 - sum_v p_tv): with the synthetic lse the
-    # "probabilities" do not sum to one, so the column-sum identity reads sum_v dW[v] = c^T H
-    # with c_t = g_t (1 - S_t); S_t comes from the oracle on the sampled rows only, so check the
-    # trace identity instead, which needs no S: <dW, W> - <dH, H> = 0 up to bf16 rounding
+    assert_grad_close(np_of(dW[torch.as_tensor(vs, device=dev)]), dW_ref, "dW")
+    # whole-result property.  With a synthetic lse the "probabilities" do not sum to one, so the
+    # column sums of dZ are not zero; the trace identity needs no such assumption:
+    # <dW, W> - <dH, H> = 0 up to bf16 rounding
     lhs = float((dW.double() * W.double()).sum())
     rhs = float((dH.double() * H.double()).sum())
     scale = float(dW.double().norm() * W.double().norm())
@@ -240,8 +276,8 @@ def test_backward_full_size(ctx):
 
 def test_vocabulary_parallel_head_full_size(ctx):
     """The 7B head split over two ranks' worth of vocabulary rows at 65536 tokens (the shards are
-    scored one after the other on this GPU): merged result against the unsharded call on every
-    token, and against the oracle on sampled rows."""
+    scored one after the other on this GPU): merged result against the oracle on sampled rows, and
+    against the unsharded call on every token."""
     w = wl.make_workload("cfg4")
     dev = device()
     T = w.total_tokens
@@ -255,58 +291,155 @@ def test_vocabulary_parallel_head_full_size(ctx):
     one = [torch.empty(T, device=dev) for _ in range(3)]
     ctx.token_logprob(H, W, y, *one)
     assert ctx.check_device_errors() == 0
-    for got, ref in zip((logp, ent, lse), one):
-        assert float((got - ref).abs().max()) <= 1e-4
-    # exactly one shard holds every token's target
-    assert bool((torch.isfinite(partials[:, :, 3]).sum(0) == 1).all())
-    rows = sample_rows(w.tok_offset, T, 64, seed=5)
+    rows = sample_rows(w.tok_offset, T, N_ROWS_MB, seed=5)
     rt = torch.as_tensor(rows, device=dev)
     o_logp, o_ent, o_lse = oracle_rows(H[rt].cpu(), wl.bf16_bits(W), np_of(y[rt]))
     assert np.abs(np_of(logp[rt]) - o_logp).max() <= LOGP_TOL
     assert np.abs(np_of(ent[rt]) - o_ent).max() <= LOGP_TOL
     assert np.abs(np_of(lse[rt]) - o_lse).max() <= LOGP_TOL
+    for got, ref in zip((logp, ent, lse), one):
+        assert float((got - ref).abs().max()) <= 1e-4
+    # exactly one shard holds every token's target
+    assert bool((torch.isfinite(partials[:, :, 3]).sum(0) == 1).all())
 
 
-def test_fused_update_full_size(ctx):
-    """cfg4 through af_policy_update against the same micro-batch through the three separate
-    calls (which the tests above tie to the oracle): log-probs, loss record and dlogp agree to
-    fp32 rounding, the gradients within the bf16 rounding of dZ."""
+# ------------------------------------------------------------------------------------------
+# the actor update as a chain at full size: log-prob -> loss -> backward, three calls or one
+# ------------------------------------------------------------------------------------------
+_ORACLE_CACHE = {}      # oracle results of a chain workload (generator inputs only), shared by both modes
+
+
+def run_actor_update(ctx, mode, w, H, W, y, old, ref, reward, kl_coef):
+    """The cfg4-shaped micro-batch (samples in index order) through the three calls or the fused one."""
     from paper_2507_01663_b200 import binding as B
-    w = wl.make_workload("cfg4")
     dev = device()
     T = w.total_tokens
-    store, W, reward = build_store(w, dev)
-    H, y, old, ref = store["hidden"], store["target"], store["old_logp"], store["ref_logp"]
     adv = torch.empty(w.N, device=dev)
     ctx.grpo_advantage(reward, None, w.n_prompts, adv)
     cu = torch.as_tensor(w.tok_offset.astype(np.int32), device=dev)
-    # three calls
     logp, ent, lse, g = (torch.empty(T, device=dev) for _ in range(4))
     lo = B.new_loss_out(dev)
-    ctx.token_logprob(H, W, y, logp, ent, lse)
-    ctx.policy_loss(logp, old, ref, adv, cu, lo, g, ent, w.clip_eps, w.clip_eps, w.kl_coef)
     dH = torch.empty(T, w.d, dtype=torch.bfloat16, device=dev)
     dW = torch.empty(w.V, w.d, device=dev)
-    ctx.policy_loss_backward(H, W, y, lse, g, dH, dW)
+    if mode == "three_calls":
+        ctx.token_logprob(H, W, y, logp, ent, lse)
+        ctx.policy_loss(logp, old, ref, adv, cu, lo, g, ent, w.clip_eps, w.clip_eps, kl_coef)
+        ctx.policy_loss_backward(H, W, y, lse, g, dH, dW)       # the forward's own lse
+    else:
+        ctx.policy_update(H, W, y, old, ref, adv, cu, lo, logp, lse, dH, dW, entropy=ent, dlogp=g,
+                          clip_lo=w.clip_eps, clip_hi=w.clip_eps, kl_coef=kl_coef)
     res = B.read_loss_out(lo)
-    # one call
-    logp2, ent2, lse2, g2 = (torch.empty(T, device=dev) for _ in range(4))
-    lo2 = B.new_loss_out(dev)
-    dH2 = torch.empty_like(dH)
-    dW2 = torch.empty_like(dW)
-    ctx.policy_update(H, W, y, old, ref, adv, cu, lo2, logp2, lse2, dH2, dW2, entropy=ent2, dlogp=g2,
-                      clip_lo=w.clip_eps, clip_hi=w.clip_eps, kl_coef=w.kl_coef)
-    res2 = B.read_loss_out(lo2)
     assert ctx.check_device_errors() == 0
-    assert float((logp2 - logp).abs().max()) <= 1e-4 and float((lse2 - lse).abs().max()) <= 1e-4
-    assert float((ent2 - ent).abs().max()) <= 1e-4
-    for k in ("loss", "pg_loss", "kl_mean", "entropy_mean"):
-        assert rel(res2[k], res[k]) <= 1e-4, k
-    assert res2["n_tokens"] == T
-    assert float((g2 - g).abs().max()) <= 1e-3 * float(g.abs().max())
-    assert float((dW2 - dW).norm() / dW.norm()) <= 2e-3
-    assert float((dH2.float() - dH.float()).norm() / dH.float().norm()) <= 2e-3
-    # trace identity over the whole fused result: <dW, W> = <dH, H> up to bf16 rounding
-    lhs = float((dW2.double() * W.double()).sum())
-    rhs = float((dH2.double() * H.double()).sum())
-    assert abs(lhs - rhs) <= 2e-3 * float(dW2.double().norm() * W.double().norm())
+    return res, adv, logp, ent, lse, g, dH, dW
+
+
+@pytest.mark.parametrize("mode", ["three_calls", "fused"])
+def test_actor_update_chain_full_size(ctx, mode):
+    """cfg4 as stated (Bernoulli(0.5) rewards, eps 0.2, KL coefficient 0.04): on 2048 sampled rows
+    the log-prob, entropy, lse, dL/dlogp and dH of the CUDA chain against the oracle chain
+    advantage -> log-prob -> loss -> backward, whose inputs are the generators' alone."""
+    w = wl.make_workload("cfg4")
+    dev = device()
+    T = w.total_tokens
+    H, y, W = wl.gen_hidden(w, dev), wl.gen_target(w, dev), wl.gen_weight(w, dev)
+    reward = wl.gen_reward(w, dev)
+    cu = w.tok_offset
+    rows = sample_rows(cu, T, N_ROWS, seed=7)
+    rt = torch.as_tensor(rows, device=dev)
+    if "cfg4" not in _ORACLE_CACHE:
+        W_bits = wl.bf16_bits(W)
+        o = oracle_rows(H[rt].cpu(), W_bits, np_of(y[rt]))
+        adv_ref = O.grpo_advantage_ref(np_of(reward), w.group_id, w.n_prompts)
+        n_old = np_of(wl.gen_noise(w, wl.S_OLD, T, dev)[rt]).astype(np.float64)
+        n_ref = np_of(wl.gen_noise(w, wl.S_REF, T, dev)[rt]).astype(np.float64)
+        old_r = off_the_clip_bounds(o[0], (o[0] + n_old).astype(np.float32), w.clip_eps, w.clip_eps)
+        ref_r = (o[0] + n_ref).astype(np.float32).astype(np.float64)
+        seq_of = np.searchsorted(cu, rows, side="right") - 1
+        wt = 1.0 / (w.N * np.diff(cu)[seq_of].astype(np.float64))
+        g_ref, _ = token_gradient_ref(o[0], old_r, ref_r, adv_ref[seq_of], wt, w.clip_eps, w.kl_coef)
+        dH_ref = dH_rows_ref(H[rt].cpu(), W_bits, np_of(y[rt]), o[2], g_ref)
+        _ORACLE_CACHE["cfg4"] = (o, adv_ref, old_r, ref_r, g_ref, dH_ref)
+    (o_logp, o_ent, o_lse), adv_ref, old_r, ref_r, g_ref, dH_ref = _ORACLE_CACHE["cfg4"]
+    # store columns: centred on the generator module's estimate, the oracle's log-prob + noise at the sampled rows
+    centre = wl.centre_logp_estimate(w, H, W, y)
+    old = centre + wl.gen_noise(w, wl.S_OLD, T, dev)
+    ref = centre + wl.gen_noise(w, wl.S_REF, T, dev)
+    old[rt], ref[rt] = f32(old_r), f32(ref_r)
+    res, adv, logp, ent, lse, g, dH, dW = run_actor_update(ctx, mode, w, H, W, y, old, ref, reward, w.kl_coef)
+    assert np.abs(np_of(adv) - adv_ref).max() <= ADV_TOL
+    assert np.abs(np_of(logp[rt]) - o_logp).max() <= LOGP_TOL
+    assert np.abs(np_of(ent[rt]) - o_ent).max() <= LOGP_TOL
+    assert np.abs(np_of(lse[rt]) - o_lse).max() <= LOGP_TOL
+    assert np.abs(np_of(g[rt]) - g_ref).max() <= 5e-3 * np.abs(g_ref).max()
+    assert_grad_close(np_of(dH[rt].float()), dH_ref, "dH")
+    # whole-result properties: the record counts its tokens, sum_v dW[v,:] = 0 (softmax rows sum to
+    # one when lse is the forward's own) and <dW, W> = <dH, H>, both up to the bf16 rounding of dZ
+    assert res["n_tokens"] == T and np.isfinite(res["loss"]) and 0.0 <= res["clip_frac"] <= 1.0
+    col = dW.double().sum(0)
+    assert float(col.abs().max()) <= 2e-2 * float(dW.double().abs().sum(0).max())
+    lhs = float((dW.double() * W.double()).sum())
+    rhs = float((dH.double() * H.double()).sum())
+    assert abs(lhs - rhs) <= 2e-3 * float(dW.double().norm() * W.double().norm())
+
+
+@pytest.mark.parametrize("mode", ["three_calls", "fused"])
+def test_actor_update_chain_sparse_advantages_full_size(ctx, mode):
+    """dW -- every row of it a sum over all 65536 tokens -- against the oracle chain at the full
+    cfg4 shape.  The oracle cannot score 65536 tokens over 152064 logits in test time, so the batch
+    is made to need only some of them: all groups but two get equal rewards (the degenerate case of
+    the group normalisation: zero advantages) and the KL coefficient is 0, so that tokens outside
+    the two live groups have dL/dlogp = 0 exactly and drop out of dW, dH and the loss.  The oracle
+    scores the live tokens (about an eighth of the batch); the CUDA path runs the whole batch in
+    the launch configuration of the benchmark."""
+    w = wl.make_workload("cfg4")
+    dev = device()
+    T, G = w.total_tokens, w.group_size
+    H, y, W = wl.gen_hidden(w, dev), wl.gen_target(w, dev), wl.gen_weight(w, dev)
+    r = np_of(wl.gen_reward(w)).copy()
+    mixed = [p for p in range(w.n_prompts) if 0 < r[p * G:(p + 1) * G].sum() < G]
+    live_groups = [mixed[0], mixed[-1]]
+    for p in range(w.n_prompts):
+        if p not in live_groups:
+            r[p * G:(p + 1) * G] = r[p * G]
+    reward = f32(r)
+    cu = w.tok_offset
+    live_samples = np.concatenate([np.arange(p * G, (p + 1) * G) for p in live_groups])
+    live_tok = np.concatenate([np.arange(cu[i], cu[i + 1]) for i in live_samples])
+    lt = torch.as_tensor(live_tok, device=dev)
+    ys = np_of(y)
+    vs = vocab_rows_sample(w.V, ys[live_tok[[0, len(live_tok) // 2, -1]]], N_VOCAB_ROWS, seed=8)
+    if "sparse" not in _ORACLE_CACHE:
+        W_bits = wl.bf16_bits(W)
+        H_live = H[lt].cpu()
+        o = oracle_rows(H_live, W_bits, ys[live_tok])
+        adv_ref = O.grpo_advantage_ref(r, w.group_id, w.n_prompts)
+        assert np.count_nonzero(adv_ref) == len(live_samples)
+        n_old = np_of(wl.gen_noise(w, wl.S_OLD, T, dev)[lt]).astype(np.float64)
+        old_l = off_the_clip_bounds(o[0], (o[0] + n_old).astype(np.float32), w.clip_eps, w.clip_eps)
+        # the live responses as a batch of their own, each weighing 1/N as in the whole batch
+        cu_live = np.concatenate([[0], np.cumsum(w.lengths[live_samples])])
+        lref = O.policy_loss_ref(o[0], old_l, o[0], adv_ref[live_samples], cu_live, w.clip_eps, w.clip_eps, 0.0,
+                                 0, len(live_samples) / w.N)
+        dW_ref = O.policy_loss_backward_ref(wl.bf16_bits(H_live), W_bits, ys[live_tok], o[2], lref["dlogp"], vocab_rows=vs)
+        pick = sample_rows(cu_live, len(live_tok), 512, seed=9)
+        dH_ref = dH_rows_ref(H_live[pick], W_bits, ys[live_tok[pick]], o[2][pick], lref["dlogp"][pick])
+        _ORACLE_CACHE["sparse"] = (o, adv_ref, old_l, lref, dW_ref, pick, dH_ref)
+    (o_logp, o_ent, o_lse), adv_ref, old_l, lref, dW_ref, pick, dH_ref = _ORACLE_CACHE["sparse"]
+    centre = wl.centre_logp_estimate(w, H, W, y)
+    old = centre + wl.gen_noise(w, wl.S_OLD, T, dev)
+    ref = centre + wl.gen_noise(w, wl.S_REF, T, dev)
+    old[lt] = f32(old_l)
+    res, adv, logp, ent, lse, g, dH, dW = run_actor_update(ctx, mode, w, H, W, y, old, ref, reward, 0.0)
+    assert np.abs(np_of(adv) - adv_ref).max() <= ADV_TOL
+    dead = torch.ones(T, dtype=torch.bool, device=dev)
+    dead[lt] = False
+    assert int(torch.count_nonzero(g[dead])) == 0 and int(torch.count_nonzero(dH[dead].float())) == 0
+    assert np.abs(np_of(logp[lt]) - o_logp).max() <= LOGP_TOL
+    assert np.abs(np_of(lse[lt]) - o_lse).max() <= LOGP_TOL
+    assert np.abs(np_of(ent[lt]) - o_ent).max() <= LOGP_TOL
+    assert np.abs(np_of(g[lt]) - lref["dlogp"]).max() <= 5e-3 * np.abs(lref["dlogp"]).max()
+    for k in ("loss", "pg_loss"):
+        assert rel(res[k], lref["pg_loss"]) <= LOSS_RTOL, (k, res[k], lref["pg_loss"])
+    assert abs(res["clip_frac"] - lref["clipped"].sum() / T) <= 0.5 / T
+    assert_grad_close(np_of(dW[torch.as_tensor(vs, device=dev)]), dW_ref, "dW")
+    assert_grad_close(np_of(dH[lt[torch.as_tensor(pick, device=dev)]].float()), dH_ref, "dH")

@@ -6,7 +6,7 @@ import torch
 
 from oracle import grpo_oracle as O
 from paper_2507_01663_b200 import workloads as wl
-from gpu_util import GRAD_RTOL, LOGP_TOL, LOSS_RTOL, device, f32, np_of, rel
+from gpu_util import GRAD_RTOL, LOGP_TOL, LOSS_RTOL, device, f32, np_of, off_the_clip_bounds, rel
 
 pytestmark = pytest.mark.gpu
 
@@ -28,6 +28,7 @@ def chain_inputs(name, seed_shift=0):
     adv = O.grpo_advantage_ref(np_of(wl.gen_reward(w)), w.group_id, w.n_prompts).astype(np.float32)
     lp, ent, lse = O.token_logprob_ref(wl.bf16_bits(H), wl.bf16_bits(W), y.numpy())
     old = torch.tensor(lp, dtype=torch.float32) + wl.gen_noise(w, wl.S_OLD, T)
+    old = torch.tensor(off_the_clip_bounds(lp, old.numpy(), w.clip_eps, w.clip_eps), dtype=torch.float32)
     ref = torch.tensor(lp, dtype=torch.float32) + wl.gen_noise(w, wl.S_REF, T)
     return w, H, W, y, cu, adv, old, ref, (lp, ent, lse)
 
@@ -72,6 +73,19 @@ def test_fused_update_matches_oracle_chain(ctx, name, token_block, agg_mode, var
     assert np.linalg.norm(np_of(dW) - dW_ref) <= GRAD_RTOL * nW
     assert abs(np.linalg.norm(np_of(dH.float())) - nH) <= GRAD_RTOL * nH
     assert abs(np.linalg.norm(np_of(dW)) - nW) <= GRAD_RTOL * nW
+    # and the whole chain from the oracle's own log-probs and lse (no device value enters): no token
+    # sits near a clip bound (chain_inputs), so both sides clip the same tokens
+    cref = O.policy_loss_ref(lp, old.numpy(), ref.numpy(), adv, cu, w.clip_eps, w.clip_eps, w.kl_coef, agg_mode, 1.0,
+                             entropy=ent_r)
+    assert res["clip_frac"] == pytest.approx(cref["clip_frac"], abs=1e-7)
+    assert np.abs(np_of(g) - cref["dlogp"]).max() <= 5e-3 * np.abs(cref["dlogp"]).max()
+    # a log-prob error e moves a token's loss by at most (|A| rho + kl_coef |exp(delta) - 1|) |e|
+    slack = LOGP_TOL * float(np.abs(cref["dlogp"]).sum())
+    for k in ("loss", "pg_loss"):
+        assert abs(res[k] - cref[k]) <= LOSS_RTOL * abs(cref[k]) + slack, k
+    dH_c, dW_c = O.policy_loss_backward_ref(wl.bf16_bits(H), wl.bf16_bits(W), y.numpy(), lse_r, cref["dlogp"])
+    assert np.linalg.norm(np_of(dH.float()) - dH_c) <= GRAD_RTOL * np.linalg.norm(dH_c)
+    assert np.linalg.norm(np_of(dW) - dW_c) <= GRAD_RTOL * np.linalg.norm(dW_c)
 
 
 @pytest.mark.parametrize("variant", [1, 2], ids=["cta", "pair"])
