@@ -10,14 +10,20 @@ fused LM-head log-prob / entropy -> clipped policy loss + k3 KL (with dL/dlogp).
 Prints ONE JSON line (rank 0).  ``value`` is scored tokens/s over all ranks with the inputs
 resident in HBM; ``e2e`` is the same metric with the store columns starting in pinned host
 memory: every step's host->device copies (on a second stream, into the device copy the previous
-step is not reading) and the device->host read of the loss are inside the timed region.
-``--impl reference`` times the fp64 CPU oracle on a bounded sample of the same workload.
+step is not reading) and the device->host read of the step's results (per-token log-probs and the
+loss record) are inside the timed region.  With the default workload on one GPU the line also
+carries ``configs``: short timed legs of the other four workloads (cfg1, cfg3, cfg4, cfg5).
+``--gpus N`` (N > 1) without a launcher's RANK in the environment starts N ranks itself, one per
+GPU, through ``torch.distributed.run``.  ``--impl reference`` times the fp64 CPU oracle on a
+bounded sample of the same workload.
 """
 from __future__ import annotations
 
 import argparse
+import ctypes
 import json
 import os
+import socket
 import subprocess
 import sys
 import threading
@@ -116,8 +122,89 @@ def dist_env():
 
 
 def rank_workload(name: str, rank: int) -> wl.Workload:
-    """Weak scaling: every rank scores its own batch of the same shape (own seed => own lengths)."""
+    """Draw number `rank` of a workload: the same shape, its own seed (own lengths and values)."""
     return wl.make_workload(name, seed_offset=1000 * rank)
+
+
+class DataParallelShare:
+    """One rank's share of a data-parallel step (Section 4.1: the batch is streamed to the DP groups
+    of a task; Section 4.4, last paragraph: the controller gives every DP group the same number of
+    samples and balances their token totals with Karmarkar-Karp).
+
+    The global batch is `world` draws of the workload (weak scaling: the per-GPU work stays fixed).
+    Its responses are dealt to the ranks by af_balance_partitions with equal sample counts, so the
+    responses to one prompt end up on different ranks; each rank therefore contributes the rewards
+    of its own responses to one all-gather, computes the group-normalised advantages of the whole
+    batch from the gathered vector (group ids in arbitrary order) and keeps its own slice.  The
+    metadata (lengths, group ids, the partition) is computed by every rank alike from the seeds;
+    hidden states, targets and rewards are generated only for the rank's own responses.
+    """
+
+    def __init__(self, name: str, world: int, rank: int, balance: bool = True):
+        self.name, self.world, self.rank = name, world, rank
+        self.sources = [rank_workload(name, s) for s in range(world)]
+        w0 = self.sources[0]
+        self.n_per_source = w0.N
+        self.lengths = np.concatenate([w.lengths for w in self.sources]).astype(np.int64)
+        self.source = np.repeat(np.arange(world), w0.N)
+        self.local_index = np.tile(np.arange(w0.N), world)
+        self.group_id = (self.source * w0.n_prompts + self.local_index // w0.group_size).astype(np.int32)
+        self.n_groups = world * w0.n_prompts
+        self.N_global = world * w0.N
+        contiguous = np.repeat(np.arange(world), w0.N).astype(np.int32)      # dealt by prompt index
+        if balance and world > 1:
+            from paper_2507_01663_b200 import binding as B
+            part, _ = B.balance_partitions(self.lengths.astype(np.int32), world, True)
+        else:
+            part = contiguous
+        self.part = np.asarray(part, dtype=np.int32)
+        self.tokens_per_rank = np.bincount(self.part, weights=self.lengths, minlength=world).astype(np.int64)
+        self.tokens_per_rank_by_prompt = np.bincount(contiguous, weights=self.lengths, minlength=world).astype(np.int64)
+        # responses of rank r in increasing global index; all ranks' lists back to back = the order of
+        # the gathered reward vector
+        self.members = [np.nonzero(self.part == r)[0] for r in range(world)]
+        counts = {len(m) for m in self.members}
+        if len(counts) != 1:
+            raise RuntimeError(f"ranks got unequal sample counts {sorted(counts)}")
+        self.mine = self.members[rank]
+        self.gathered_order = np.concatenate(self.members)
+        self.gathered_group_id = self.group_id[self.gathered_order].astype(np.int32)
+        self.n_mine = len(self.mine)
+        self.loss_scale = self.n_mine / self.N_global        # B_rank / B_global: rank losses and gradients add up
+
+    def rank_view(self) -> wl.Workload:
+        """The rank's responses as a workload of their own (lengths only; group structure lives here)."""
+        w0 = self.sources[0]
+        import dataclasses
+        return dataclasses.replace(w0, lengths=self.lengths[self.mine].copy(), seed=w0.seed + 7919 * (self.rank + 1))
+
+    def build_columns(self, device):
+        """hidden / target rows and rewards of the rank's own responses, from their sources' generators."""
+        H, y, r = [], [], []
+        rewards = [wl.gen_reward(w).numpy() for w in self.sources]
+        for g in self.mine:
+            w, i = self.sources[self.source[g]], int(self.local_index[g])
+            off = w.tok_offset
+            H.append(wl.gen_hidden(w, device, int(off[i]), int(off[i + 1] - off[i])))
+            y.append(wl.gen_target(w, device, int(off[i]), int(off[i + 1] - off[i])))
+            r.append(rewards[self.source[g]][i])
+        return torch.cat(H, 0), torch.cat(y, 0), torch.as_tensor(np.asarray(r, dtype=np.float32), device=device)
+
+    def gather_rewards(self, mine: torch.Tensor) -> torch.Tensor:
+        """All ranks' reward slices back to back (rank-major): 4 bytes per response cross the links."""
+        if self.world == 1:
+            return mine
+        import torch.distributed as dist
+        out = torch.empty(self.N_global, dtype=mine.dtype, device=mine.device)
+        dist.all_gather_into_tensor(out, mine.contiguous())
+        return out
+
+    def report(self) -> dict:
+        t, b = self.tokens_per_rank, self.tokens_per_rank_by_prompt
+        return {"ranks": self.world, "responses_per_rank": int(self.n_mine), "tokens_per_rank": [int(x) for x in t],
+                "token_spread_balanced": int(t.max() - t.min()), "token_spread_by_prompt_index": int(b.max() - b.min()),
+                "how": "af_balance_partitions (Karmarkar-Karp, equal sample counts) over the global batch; rewards "
+                       "all-gathered, advantages by group id on every rank"}
 
 
 def reduce_over_ranks(ms_local: float, tokens_local: int, world: int):
@@ -168,27 +255,36 @@ class ScoringJob:
     """Device buffers of one rank and the step function that runs the path through the C ABI."""
 
     def __init__(self, w: wl.Workload, device: torch.device, gemm_variant: int = 0, world: int = 1, v_splits: int = 0,
-                 vocab_parallel: bool = False, rank: int = 0, bwd_token_block: int = 0):
+                 vocab_parallel: bool = False, rank: int = 0, bwd_token_block: int = 0,
+                 dp: "DataParallelShare | None" = None):
         from paper_2507_01663_b200 import binding as B
-        self.B, self.w, self.dev, self.world = B, w, device, world
+        self.B, self.dev, self.world, self.rank, self.dp = B, device, world, rank, dp
         self.ctx = B.Context(device.index or 0)
         self.ctx.set_tuning(v_splits, bwd_token_block, gemm_variant)
+        if dp is not None:
+            # this rank's token-balanced share of the global batch; the head is replicated
+            w = dp.rank_view()
+            hidden, target, self.reward = dp.build_columns(device)
+            self.store = {"hidden": hidden, "target": target}
+            self.W = wl.gen_weight(dp.sources[0], device)
+            self.gid = torch.as_tensor(dp.gathered_group_id, device=device)
+            self.adv_all = torch.empty(dp.N_global, device=device)
+        else:
+            self.store = {"hidden": wl.gen_hidden(w, device), "target": wl.gen_target(w, device)}
+            self.W = wl.gen_weight(w, device)
+            self.reward = wl.gen_reward(w, device)
+        self.w = w
         T = w.total_tokens
         self.T = T
-        self.store = {
-            "hidden": wl.gen_hidden(w, device), "target": wl.gen_target(w, device),
-        }
-        self.W = wl.gen_weight(w, device)
         self.vocab_parallel = vocab_parallel
-        # data parallel: equal batches per rank, each weighs 1 / world; vocabulary parallel: one batch
-        self.loss_scale = 1.0 if vocab_parallel else 1.0 / world
+        # data parallel: the rank's batch weighs B_rank / B_global; vocabulary parallel: one batch
+        self.loss_scale = 1.0 if vocab_parallel else (dp.loss_scale if dp is not None else 1.0 / world)
         self.v_lo, self.v_hi = vocab_shard(w.V, world, rank) if vocab_parallel else (0, w.V)
-        self.reward = wl.gen_reward(w, device)
         centre = wl.centre_logp_estimate(w, self.store["hidden"], self.W, self.store["target"])
         self.store["old_logp"] = centre + wl.gen_noise(w, wl.S_OLD, T, device)
         self.store["ref_logp"] = centre + wl.gen_noise(w, wl.S_REF, T, device)
         del centre
-        self.adv = torch.empty(w.N, device=device)
+        self.adv = self.adv_all[rank * dp.n_mine:(rank + 1) * dp.n_mine] if dp is not None else torch.empty(w.N, device=device)
         # micro-batches: the whole arrival-ordered batch, or (streaming store) greedy arrival-ordered
         # index lists under the workload's token budget, issued back to back on one stream
         self.mbs = wl.microbatches(w)
@@ -209,17 +305,53 @@ class ScoringJob:
             self.partial = torch.empty(cap_T, 4, device=device)
         self.loss_outs = [B.new_loss_out(device) for _ in self.mbs]
         self.loss_out = self.loss_outs[-1]
+        self.overlap_dw = False
         if w.backward:
             self.d_hidden = torch.empty(cap_T, w.d, dtype=torch.bfloat16, device=device)
             self.d_W = torch.empty(w.V, w.d, device=device)
+            if world > 1 and not vocab_parallel:
+                # the gradient all-reduce runs on its own stream, started by the event the backward
+                # records as soon as d_W is complete (its last block runs the dW product first)
+                self.overlap_dw = True
+                self.comm_stream = torch.cuda.Stream()
+                self.dw_ready, self.dw_reduced = torch.cuda.Event(), torch.cuda.Event()
+                self.dw_ready.record()
+                self.dw_reduced.record()
+                self.ctx.set_dw_ready_event(self.dw_ready)
+        self.e2e_logp_host = None
         self.ctx.reserve(cap_T, cap_B, w.d, w.V, with_backward=2 if w.backward else False)
         self.gemm_events, self.pack_events, self.bwd_events = [], [], []
         per_mb = KERNELS_PER_STEP - 1 + (3 * -(-cap_T // BWD_TOKEN_BLOCK) if w.backward else 0)
         self.launches_per_step = 1 + per_mb * len(self.mbs)
 
+    def advantages(self, reward=None):
+        """Group-normalised advantages of this rank's responses (into self.adv)."""
+        w, c = self.w, self.ctx
+        reward = self.reward if reward is None else reward
+        if self.dp is None:
+            c.grpo_advantage(reward, None, w.n_prompts, self.adv)
+        else:
+            # groups are spread over the ranks: gather every rank's rewards, normalise the whole
+            # batch by group id, keep the own slice (self.adv is a view of it)
+            c.grpo_advantage(self.dp.gather_rewards(reward), self.gid, self.dp.n_groups, self.adv_all)
+
+    def sum_dW_over_ranks(self):
+        """The one exchange of a data-parallel actor update.  With the overlap set up, the all-reduce
+        waits for the backward's "d_W complete" event on the communication stream and runs beside
+        the last block's dH product; the compute stream waits for it only before d_W is next written."""
+        if self.world == 1:
+            return
+        if not self.overlap_dw:
+            allreduce_sum_(self.d_W, self.world)
+            return
+        with torch.cuda.stream(self.comm_stream):
+            self.comm_stream.wait_event(self.dw_ready)
+            allreduce_sum_(self.d_W, self.world)
+            self.dw_reduced.record(self.comm_stream)
+
     def step(self, time_gemm: bool = False, store_cols=None, reward=None):
         w, c = self.w, self.ctx
-        c.grpo_advantage(self.reward if reward is None else reward, None, w.n_prompts, self.adv)
+        self.advantages(reward)
         store = {"tok_offset_host": self.off, "d": w.d, "adv": self.adv, **(self.store if store_cols is None else store_cols)}
         total = 0
         for mb, loss_out in zip(self.mbs, self.loss_outs):
@@ -242,9 +374,13 @@ class ScoringJob:
             c.policy_loss(self.logp, self.packed["old_logp"], self.packed["ref_logp"], self.packed["adv_seq"],
                           self.packed["cu_seqlens"], loss_out, self.dlogp, self.ent,
                           w.clip_eps, w.clip_eps, w.kl_coef, 0, self.loss_scale, B=len(mb), T=T)
+            if self.e2e_logp_host is not None:      # end-to-end steps return the task's result to the host
+                self.e2e_logp_host[total:total + T].copy_(self.logp[:T], non_blocking=True)
             if w.backward:
                 if ev:
                     ev[4].record()
+                if self.overlap_dw:
+                    torch.cuda.current_stream().wait_event(self.dw_reduced)   # the previous sum has read d_W
                 if self.vocab_parallel:
                     # this rank's rows of dW stay here; the ranks' contributions to dH are summed
                     c.policy_loss_backward_shard(self.packed["hidden"], self.W_shard, self.packed["target"], self.lse,
@@ -259,7 +395,7 @@ class ScoringJob:
                 if self.vocab_parallel:
                     allreduce_sum_(self.d_hidden[:T], self.world)
                 else:
-                    allreduce_sum_(self.d_W, self.world)    # equal batches per rank: loss_scale = 1 / world
+                    self.sum_dW_over_ranks()
             if ev:
                 self.pack_events.append((ev[0], ev[1]))
                 self.gemm_events.append((ev[2], ev[3]))
@@ -320,7 +456,18 @@ class ScoringJob:
         gbs = 8.0 * n / ms / 1e6
         out["grpo_advantage"] = {"responses": n, "group_size": G, "bytes_per_response": 8, "ms": ms, "gbs": gbs,
                                  "frac": gbs / peak_gbs}
-        del r, a
+        # the same call with membership by group id (any order): exact fixed-point sums with integer
+        # atomics, four streaming passes; ids in index order (a warp's lanes share groups and combine
+        # before the atomics) and ids drawn at random (every atomic lands on its own line of a table
+        # larger than L2)
+        n_id = min(n, 1 << 26)
+        for label, ids in (("ids_in_order", (torch.arange(n_id, device=dev, dtype=torch.int32) // G)),
+                           ("ids_shuffled", wl.randint(self.w.seed, wl.S_MISC, 0, n_id, n_id // G, dev).to(torch.int32))):
+            ms = avg_ms(lambda: c.grpo_advantage(r[:n_id], ids, n_id // G, a[:n_id]), n=5)
+            gbs = 36.0 * n_id / ms / 1e6
+            out["grpo_advantage_" + label] = {"responses": n_id, "groups": n_id // G, "bytes_per_response": 36, "ms": ms,
+                                              "gbs": gbs, "frac": gbs / peak_gbs}
+        del r, a, ids
         # controller: one read request against a 2^log2_n-sample status table (12 B read per sample:
         # ready, consumed, length) that hands out the first 4096 eligible samples
         tab = {"ready": torch.ones(n, dtype=torch.int32, device=dev),
@@ -368,17 +515,19 @@ class ScoringJob:
     def step_fused_update(self):
         """advantage -> pack -> af_policy_update (forward + loss + backward, logits evaluated once)."""
         w, c = self.w, self.ctx
-        c.grpo_advantage(self.reward, None, w.n_prompts, self.adv)
+        self.advantages()
         store = {"tok_offset_host": self.off, "d": w.d, "adv": self.adv, **self.store}
         total = 0
         for mb, loss_out in zip(self.mbs, self.loss_outs):
             T = c.pack_microbatch(store, mb, self.packed)
+            if self.overlap_dw:
+                torch.cuda.current_stream().wait_event(self.dw_reduced)
             c.policy_update(self.packed["hidden"], self.W, self.packed["target"], self.packed["old_logp"],
                             self.packed["ref_logp"], self.packed["adv_seq"], self.packed["cu_seqlens"], loss_out,
                             self.logp, self.lse, self.d_hidden, self.d_W, entropy=self.ent, dlogp=self.dlogp,
-                            clip_lo=w.clip_eps, clip_hi=w.clip_eps, kl_coef=w.kl_coef, loss_scale=1.0 / self.world,
+                            clip_lo=w.clip_eps, clip_hi=w.clip_eps, kl_coef=w.kl_coef, loss_scale=self.loss_scale,
                             B=len(mb), T=T)
-            allreduce_sum_(self.d_W, self.world)
+            self.sum_dW_over_ranks()
             total += T
         return total
 
@@ -454,6 +603,138 @@ class ScoringJob:
             raise RuntimeError(f"the controller handed out {total} tokens of {self.T}")
         return total
 
+    # -- the streaming pieces as one path: two tasks, one store, one status table -----------
+    COL_RESPONSE, COL_OLD_LOGP = 1, 2         # column bits of the status table
+    TASK_INFER, TASK_UPDATE = 1, 2            # consumption bits: actor inference, actor-update forward
+
+    def make_closed_loop(self, wave: int = 512):
+        """Section 4.2's interaction, end to end on one device.  Responses become ready (hidden
+        states and targets written) `wave` at a time in arrival order.  Actor inference asks the
+        controller for ready samples, fetches them, scores them and writes its per-token log-probs
+        back to the store's old_logp column by the same index list, which also marks that column
+        written.  The loss task asks for samples whose response AND old_logp columns are written,
+        fetches them -- old_logp now being what the first task stored -- scores them and reduces
+        the loss.  Every micro-batch of either task is whatever af_controller_get hands out."""
+        w, dev, B = self.w, self.dev, self.B
+        if not hasattr(self, "W_host"):
+            self.make_weight_refresh()
+        self.cl_tab = {"ready": torch.zeros(w.N, dtype=torch.int32, device=dev),
+                       "consumed": torch.zeros(w.N, dtype=torch.int32, device=dev),
+                       "length": torch.as_tensor(w.lengths.astype(np.int32), device=dev)}
+        self.cl_arrival = torch.as_tensor(wl.arrival_order(w).astype(np.int32), device=dev)
+        self.cl_wave = wave
+
+        def channel():
+            return {"idx": [torch.empty(w.N, dtype=torch.int32, device=dev) for _ in range(2)],
+                    "res": [B.new_get_result(dev) for _ in range(2)],
+                    "idx_host": [torch.empty(w.N, dtype=torch.int32, pin_memory=True) for _ in range(2)],
+                    "res_host": [torch.empty(ctypes.sizeof(B.GetResult), dtype=torch.uint8, pin_memory=True) for _ in range(2)]}
+
+        self.cl_req = {self.TASK_INFER: channel(), self.TASK_UPDATE: channel()}
+        self.cl_done = [torch.cuda.Event() for _ in range(2)]
+        budget = int(w.token_budget or w.total_tokens)
+        cap_T = max(budget, int(w.lengths.max()))
+        self.cl_budget = budget
+        self.cl_packed1 = {"cu_seqlens": torch.zeros(w.N + 1, dtype=torch.int32, device=dev),
+                           "hidden": torch.empty(cap_T, w.d, dtype=torch.bfloat16, device=dev),
+                           "target": torch.empty(cap_T, dtype=torch.int32, device=dev)}
+        self.cl_packed2 = {"cu_seqlens": torch.zeros(w.N + 1, dtype=torch.int32, device=dev),
+                           "hidden": torch.empty(cap_T, w.d, dtype=torch.bfloat16, device=dev),
+                           "target": torch.empty(cap_T, dtype=torch.int32, device=dev),
+                           "old_logp": torch.empty(cap_T, device=dev), "ref_logp": torch.empty(cap_T, device=dev),
+                           "adv_seq": torch.empty(w.N, device=dev)}
+        self.cl_logp1 = torch.empty(cap_T, device=dev)
+        self.cl_logp2, self.cl_ent2, self.cl_lse2, self.cl_g2 = (torch.empty(cap_T, device=dev) for _ in range(4))
+        self.cl_old_col = torch.empty(w.total_tokens, device=dev)     # the column actor inference fills
+        self.cl_loss_outs = []
+        self.ctx.reserve(cap_T, w.N, w.d, w.V)
+        self.cl_iterations = 0
+
+    def _cl_request(self, slot: int):
+        """Queue: the next wave of arrivals marked written, one read request per task, answers to pinned memory."""
+        c, w = self.ctx, self.w
+        if self.cl_next_wave < w.N:
+            c.controller_put(self.cl_tab, self.cl_arrival[self.cl_next_wave:self.cl_next_wave + self.cl_wave],
+                             self.COL_RESPONSE)
+            self.cl_next_wave += self.cl_wave
+        for task, mask in ((self.TASK_INFER, self.COL_RESPONSE), (self.TASK_UPDATE, self.COL_RESPONSE | self.COL_OLD_LOGP)):
+            ch = self.cl_req[task]
+            c.controller_get(self.cl_tab, mask, task, w.N, self.cl_budget, ch["idx"][slot], ch["res"][slot])
+            ch["idx_host"][slot].copy_(ch["idx"][slot], non_blocking=True)
+            ch["res_host"][slot].copy_(ch["res"][slot], non_blocking=True)
+        self.cl_done[slot].record()
+
+    def step_closed_loop(self, refresh_weights: bool = True):
+        """One pass of the whole store through both tasks.  Requests are queued one iteration ahead
+        of the kernels that use their answers, so the host never waits for the GPU to drain; a loss
+        request therefore sees the log-probs written up to the previous iteration.  With
+        `refresh_weights` a new LM-head weight is loaded on a second stream meanwhile and swapped in
+        at an iteration boundary (Section 5.2)."""
+        w, c, B = self.w, self.ctx, self.B
+        main = torch.cuda.current_stream()
+        pending = False
+        if refresh_weights:
+            with torch.cuda.stream(self.w_stream):
+                self.w_stream.wait_event(self.w_released)
+                self.W_standby.copy_(self.W_host, non_blocking=True)
+                self.w_loaded.record(self.w_stream)
+            pending = True
+        c.controller_clear(self.cl_tab, 0xFFFFFFFF, 0xFFFFFFFF)
+        self.cl_old_col.fill_(float("nan"))       # a row read before it was written would poison its loss
+        self.advantages()
+        store1 = {"tok_offset_host": self.off, "d": w.d, "hidden": self.store["hidden"], "target": self.store["target"]}
+        store2 = {"tok_offset_host": self.off, "d": w.d, "adv": self.adv, "hidden": self.store["hidden"],
+                  "target": self.store["target"], "old_logp": self.cl_old_col, "ref_logp": self.store["ref_logp"]}
+        self.cl_next_wave, slot, tot1, tot2, it, k2 = 0, 0, 0, 0, 0, 0
+        self.cl_history = []                      # (task, index list) of every micro-batch handed out
+        self._cl_request(slot)
+        while tot1 < self.T or tot2 < self.T:
+            it += 1
+            if it > 8 * w.N + 64:
+                raise RuntimeError("the closed loop made no progress")
+            self.cl_done[slot].synchronize()
+            mbs = {}
+            for task, ch in self.cl_req.items():
+                n = B.GetResult.from_buffer_copy(ch["res_host"][slot].numpy().tobytes()).count
+                mbs[task] = ch["idx_host"][slot][:n].numpy().copy()
+            self._cl_request(slot ^ 1)
+            if pending and (self.w_loaded.query() or (tot1 >= self.T)):
+                main.wait_event(self.w_loaded)
+                self.W, self.W_standby = self.W_standby, self.W
+                self.w_released.record(main)
+                self.w_swaps += 1
+                pending = False
+            mb = mbs[self.TASK_INFER]
+            if len(mb):      # actor inference: fetch, score, write the log-probs back, mark them written
+                self.cl_history.append((self.TASK_INFER, mb))
+                T1 = c.pack_microbatch(store1, mb, self.cl_packed1)
+                c.token_logprob(self.cl_packed1["hidden"], self.W, self.cl_packed1["target"], self.cl_logp1, T=T1)
+                c.unpack_microbatch(self.off, mb, [self.cl_logp1], [self.cl_old_col], self.cl_tab, self.COL_OLD_LOGP)
+                tot1 += T1
+            mb = mbs[self.TASK_UPDATE]
+            if len(mb):      # loss task: its old_logp column is what actor inference stored
+                self.cl_history.append((self.TASK_UPDATE, mb))
+                while len(self.cl_loss_outs) <= k2:
+                    self.cl_loss_outs.append(B.new_loss_out(self.dev))
+                T2 = c.pack_microbatch(store2, mb, self.cl_packed2)
+                c.token_logprob(self.cl_packed2["hidden"], self.W, self.cl_packed2["target"], self.cl_logp2,
+                                self.cl_ent2, self.cl_lse2, T=T2)
+                c.policy_loss(self.cl_logp2, self.cl_packed2["old_logp"], self.cl_packed2["ref_logp"],
+                              self.cl_packed2["adv_seq"], self.cl_packed2["cu_seqlens"], self.cl_loss_outs[k2],
+                              self.cl_g2, self.cl_ent2, w.clip_eps, w.clip_eps, w.kl_coef, 0, 1.0, B=len(mb), T=T2)
+                tot2 += T2
+                k2 += 1
+            slot ^= 1
+        if pending:          # nothing was left to score when the load finished: swap for the next step
+            main.wait_event(self.w_loaded)
+            self.W, self.W_standby = self.W_standby, self.W
+            self.w_released.record(main)
+            self.w_swaps += 1
+        self.cl_iterations, self.cl_loss_count = it, k2
+        if tot1 != self.T or tot2 != self.T:
+            raise RuntimeError(f"the two tasks saw {tot1} and {tot2} tokens of {self.T}")
+        return tot1 + tot2
+
     # -- delayed parameter update: new weights arrive while scoring goes on -----------------
     def make_weight_refresh(self):
         """A pinned host copy of the LM-head weight (the "received new parameters"), a standby
@@ -515,6 +796,9 @@ class ScoringJob:
         self.e2e_steps = 0
         self.h2d_bytes = sum(t.numel() * t.element_size() for t in self.host.values())
         self.host_loss = [torch.empty(lo.shape, dtype=torch.uint8, pin_memory=True) for lo in self.loss_outs]
+        # the result of the scoring task: per-token log-probs in packed order, read back every step
+        self.e2e_logp_host = torch.empty(self.T, dtype=torch.float32, pin_memory=True)
+        self.d2h_bytes = self.e2e_logp_host.numel() * 4 + sum(lo.numel() for lo in self.loss_outs)
 
     def step_e2e(self):
         b = self.e2e_steps & 1
@@ -576,6 +860,158 @@ def blas_threads() -> int:
         return os.cpu_count() or 1
 
 
+def describe(w, job, name: str) -> str:
+    return (f"{name}: {head_name(w)} head d={w.d} V={w.V}, {w.N} responses "
+            f"({w.n_prompts} prompts x {w.group_size}), {job.T} scored tokens per GPU, "
+            + (f"{len(job.mbs)} arrival-ordered micro-batches of <= {w.token_budget} tokens, packed, "
+               "scored and loss-reduced back to back on one stream" if w.token_budget
+               else "one arrival-ordered packed micro-batch")
+            + (", forward + backward (dH, dW)" if w.backward else ""))
+
+
+def host_enqueue_us(job, n: int = 20) -> float:
+    """Host time of one step's calls (no synchronisation inside the loop): what the CPU pays to
+    enqueue a step, which bounds the step rate of a launch-bound workload."""
+    job.step()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(n):
+        job.step()
+    dt = time.perf_counter() - t0
+    torch.cuda.synchronize()
+    return 1e6 * dt / n
+
+
+def graph_replay_us(job, n: int = 50) -> float:
+    """Device time per scoring step (advantage, log-prob, loss on the packed batch) when the calls
+    are recorded once into a CUDA graph and replayed: what a launch-bound workload costs once the
+    host's calls are out of the way.  (The pack stages its index list through the host and is not
+    recorded.)"""
+    w, c = job.w, job.ctx
+    T = job.T
+
+    def scoring():
+        c.grpo_advantage(job.reward, None, w.n_prompts, job.adv)
+        c.token_logprob(job.packed["hidden"], job.W, job.packed["target"], job.logp, job.ent, job.lse, T=T)
+        c.policy_loss(job.logp, job.packed["old_logp"], job.packed["ref_logp"], job.packed["adv_seq"],
+                      job.packed["cu_seqlens"], job.loss_out, job.dlogp, job.ent, w.clip_eps, w.clip_eps, w.kl_coef,
+                      0, job.loss_scale, B=len(job.mbs[-1]), T=T)
+
+    job.step()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        scoring()
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        scoring()
+    for _ in range(3):
+        graph.replay()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(n):
+        graph.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    return 1e3 * e0.elapsed_time(e1) / n
+
+
+def timed_leg(fn, steps: int, warmup: int, world: int, tokens: int):
+    for _ in range(warmup):
+        fn()
+    ms_total = timed_loop(fn, steps, world)
+    ms, _ = reduce_over_ranks(ms_total / steps, tokens, world)
+    return ms
+
+
+def streaming_legs(job, args, world: int, tokens: int, steps: int, warmup: int) -> dict:
+    """The streaming store's extra legs: the controller in the loop, the delayed weight update, and
+    the two-task closed loop with write-back."""
+    out = {}
+    w = job.w
+    job.make_live_controller()
+    ms = timed_leg(job.step_live_controller, steps, warmup, world, tokens)
+    out["live_controller"] = {
+        "value": job.T / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms, "micro_batches": job.live_requests,
+        "what": "the same store scored with the controller in the loop: responses become ready 512 at a "
+                "time in arrival order, every micro-batch is the answer to an af_controller_get (ready, "
+                "not consumed, <= the token budget) read back to the host, then packed, scored and "
+                "loss-reduced; the next request is queued ahead of the current micro-batch's kernels"}
+    job.make_weight_refresh()
+    ms = timed_leg(job.step_with_weight_refresh, steps, warmup, world, tokens)
+    out["weight_refresh"] = {
+        "value": tokens / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms,
+        "h2d_bytes_per_step": int(job.W.numel() * job.W.element_size()), "swaps": job.w_swaps,
+        "what": "every step a new LM-head weight is loaded from pinned host memory on a second stream "
+                "while scoring continues with the old one; swapped at a micro-batch boundary"}
+    job.make_closed_loop()
+    ms = timed_leg(job.step_closed_loop, steps, max(1, warmup - 1), world, tokens)
+    losses = [job.B.read_loss_out(lo) for lo in job.cl_loss_outs[:job.cl_loss_count]]
+    if not all(np.isfinite(r["loss"]) for r in losses):
+        raise RuntimeError("closed loop: a loss record is not finite (a row was read before it was written)")
+    out["closed_loop"] = {
+        "value": job.T / (ms * 1e-3), "unit": "store tokens/s through both tasks", "ms_per_step": ms,
+        "scored_tokens_per_s": 2.0 * job.T / (ms * 1e-3), "iterations": job.cl_iterations,
+        "loss_micro_batches": job.cl_loss_count, "max_clip_frac": float(max(r["clip_frac"] for r in losses)),
+        "weight_swaps": job.w_swaps,
+        "what": "controller get -> pack -> log-prob -> write-back of the log-probs to the store's old_logp column "
+                "with its ready bit (actor inference), and controller get on that bit -> pack -> log-prob -> loss "
+                "(actor-update forward), interleaved on one stream over one status table, while a new weight "
+                "loads and is swapped in at an iteration boundary; every token is scored twice"}
+    return out
+
+
+def side_leg(name: str, args, dev, peaks, steps: int = 5, warmup: int = 3) -> dict:
+    """A short timed leg of another workload on one GPU (its own buffers, its own clock record)."""
+    w = wl.make_workload(name)
+    job = ScoringJob(w, dev, {"default": 0, "single": 1, "pair": 2}[args.gemm])
+    out = {"workload": describe(w, job, name), "steps": steps, "warmup": warmup}
+    for _ in range(warmup):
+        job.step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(dev.index or 0)
+    sampler.start()
+    ms_total = timed_loop(lambda: job.step(time_gemm=True), steps, 1)
+    out["clocks"] = sampler.stop()
+    ms = ms_total / steps
+    gemm_ms = float(np.sum([a.elapsed_time(b) for a, b in job.gemm_events])) / steps
+    pack_ms = float(np.sum([a.elapsed_time(b) for a, b in job.pack_events])) / steps
+    tf = 2.0 * job.T * w.d * w.V / (gemm_ms * 1e-3) / 1e12
+    pack_gbs = (2.0 * job.T * (2 * w.d + 12) + 8.0 * w.N) / (pack_ms * 1e-3) / 1e9
+    out.update({"value": job.T / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms,
+                "logprob_ms": gemm_ms, "logprob_tflops": tf, "frac_of_sustained": tf / peaks["bf16_tflops_sustained"],
+                "frac_of_burst": tf / peaks["bf16_tflops"], "frac_of_nominal_2250": tf / 2250.0,
+                "pack_ms": pack_ms, "pack_gbs": pack_gbs, "pack_frac_of_hbm": pack_gbs / peaks["hbm_gbs"],
+                "gpu_launches": job.launches_per_step * steps})
+    if job.T < 10000:
+        out["host_enqueue_us_per_step"] = host_enqueue_us(job)
+        if not w.token_budget and not w.backward:
+            out["graph_replay_us_per_scoring_step"] = graph_replay_us(job)
+        out["note"] = ("launch- and epilogue-bound: the device work of a step is tens of microseconds, the host's "
+                       "calls take longer; tokens/s here measures call overhead, not the kernels")
+    if w.backward:
+        bwd_ms = float(np.sum([a.elapsed_time(b) for a, b in job.bwd_events])) / steps
+        out["three_calls"] = {"ms_per_step": ms, "backward_ms": bwd_ms,
+                              "backward_tflops_6TdV": 6.0 * job.T * w.d * w.V / (bwd_ms * 1e-3) / 1e12,
+                              "step_tflops_8TdV": 8.0 * job.T * w.d * w.V / (ms * 1e-3) / 1e12}
+        ms_f = timed_leg(job.step_fused_update, steps, 2, 1, job.T)
+        out["fused_update"] = {"ms_per_step": ms_f, "value": job.T / (ms_f * 1e-3), "unit": UNIT,
+                               "tflops_6TdV_model": 6.0 * job.T * w.d * w.V / (ms_f * 1e-3) / 1e12,
+                               "frac_of_sustained": 6.0 * job.T * w.d * w.V / (ms_f * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"]}
+    if w.token_budget:
+        out.update(streaming_legs(job, args, 1, job.T, 3, 2))
+    flags = job.ctx.check_device_errors()
+    if flags:
+        raise RuntimeError(f"{name}: device error word set: {flags}")
+    out["loss"] = job.B.read_loss_out(job.loss_out)["loss"]
+    job.ctx.close()
+    del job
+    torch.cuda.empty_cache()
+    return out
+
+
 def run_ours(args):
     rank, local_rank, world = dist_env()
     if not torch.cuda.is_available():
@@ -585,10 +1021,17 @@ def run_ours(args):
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
-    # data parallel: every rank its own batch; vocabulary parallel: one batch, the head split by rows
+    variant = {"default": 0, "single": 1, "pair": 2}[args.gemm]
+    base = wl.make_workload(args.workload)
+    # data parallel: the global batch (one draw of the workload per rank) is dealt to the ranks by
+    # token count; a streaming store stays whole on its rank; vocabulary parallel: one batch, the
+    # head split by rows
+    dp = None
+    if world > 1 and not args.vocab_parallel and not base.token_budget:
+        dp = DataParallelShare(args.workload, world, rank, balance=not args.no_balance)
     w = rank_workload(args.workload, 0 if args.vocab_parallel else rank)
-    job = ScoringJob(w, dev, {"default": 0, "single": 1, "pair": 2}[args.gemm], world, args.v_splits,
-                     args.vocab_parallel, rank, args.bwd_token_block)
+    job = ScoringJob(w, dev, variant, world, args.v_splits, args.vocab_parallel, rank, args.bwd_token_block, dp)
+    w = job.w
     peaks = measured_peaks()
     hbm_alone = job.hbm_kernels_at_scale(peaks["hbm_gbs"], args.hbm_log2) if rank == 0 and world == 1 else {}
 
@@ -620,43 +1063,23 @@ def run_ours(args):
     ms_e2e_total = timed_loop(job.step_e2e, args.steps, world)
     ms_e2e, _ = reduce_over_ranks(ms_e2e_total / args.steps, job.T, world)
     e2e_steps_ms = list(timed_loop.last_steps_ms)
+    logp_back = job.e2e_logp_host[:job.T]
+    if not bool(torch.isfinite(logp_back).all()):
+        raise RuntimeError("end-to-end step: log-probs read back to the host are not finite")
+    job.e2e_logp_host = None
 
     fused = None
     if w.backward and not args.vocab_parallel:
-        for _ in range(2):
-            job.step_fused_update()
-        ms_f_total = timed_loop(job.step_fused_update, args.steps, world)
-        ms_f, _ = reduce_over_ranks(ms_f_total / args.steps, job.T, world)
+        ms_f = timed_leg(job.step_fused_update, args.steps, 2, world, job.T)
         loss_f = job.B.read_loss_out(job.loss_out)["loss"]
         fused = {"value": tokens / (ms_f * 1e-3), "unit": UNIT, "ms_per_step": ms_f, "loss": loss_f,
                  "tflops_6TdV_model": 6.0 * job.T * w.d * w.V / (ms_f * 1e-3) / 1e12,
                  "what": "the same step through af_policy_update: forward, loss and backward in one call, the "
                          "logits evaluated once per token (6 T d V products instead of 8)"}
 
-    live = None
-    if args.live_controller and w.token_budget and world == 1:
-        job.make_live_controller()
-        for _ in range(2):
-            job.step_live_controller()
-        ms_l_total = timed_loop(job.step_live_controller, args.steps, world)
-        ms_l = ms_l_total / args.steps
-        live = {"value": job.T / (ms_l * 1e-3), "unit": UNIT, "ms_per_step": ms_l, "micro_batches": job.live_requests,
-                "what": "the same store scored with the controller in the loop: responses become ready 512 at a "
-                        "time in arrival order, every micro-batch is the answer to an af_controller_get (ready, "
-                        "not consumed, <= the token budget) read back to the host, then packed, scored and "
-                        "loss-reduced; the next request is queued ahead of the current micro-batch's kernels"}
-
-    refresh = None
-    if args.weight_refresh and not w.backward:
-        job.make_weight_refresh()
-        for _ in range(2):
-            job.step_with_weight_refresh()
-        ms_r_total = timed_loop(job.step_with_weight_refresh, args.steps, world)
-        ms_r, _ = reduce_over_ranks(ms_r_total / args.steps, job.T, world)
-        refresh = {"value": tokens / (ms_r * 1e-3), "unit": UNIT, "ms_per_step": ms_r,
-                   "h2d_bytes_per_step": int(job.W.numel() * job.W.element_size()), "swaps": job.w_swaps,
-                   "what": "every step a new LM-head weight is loaded from pinned host memory on a second stream "
-                           "while scoring continues with the old one; swapped at a micro-batch boundary"}
+    streaming = {}
+    if w.token_budget and world == 1 and (args.live_controller or args.weight_refresh or args.closed_loop):
+        streaming = streaming_legs(job, args, world, tokens, args.steps, 2)
 
     flops = 2.0 * job.T * w.d * (job.v_hi - job.v_lo)       # this rank's rows of the head
     achieved = flops / (gemm_ms * 1e-3) / 1e12
@@ -668,14 +1091,12 @@ def run_ours(args):
                           "max": float(np.max(steps_ms))},
         "higher_is_better": True,
         "scaling": "strong" if args.vocab_parallel else "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": f"{args.workload}: {head_name(w)} head d={w.d} V={w.V}, {w.N} responses "
-                               f"({w.n_prompts} prompts x {w.group_size}), {job.T} scored tokens per GPU, "
-                               + (f"{len(job.mbs)} arrival-ordered micro-batches of <= {w.token_budget} tokens, packed, "
-                                  "scored and loss-reduced back to back on one stream" if w.token_budget
-                                  else "one arrival-ordered packed micro-batch")
-                               + (", forward + backward (dH, dW)" if w.backward else ""),
+        "config": {"workload": describe(w, job, args.workload),
                    "l2": "inputs (hidden states >> 126 MB L2) exceed L2; no flush needed",
                    "gemm": "one CTA per 128x256 tile" if args.gemm == "single" else "CTA pairs (cta_group::2), 256x256 tiles",
+                   "parallelism": ("vocabulary-parallel head" if args.vocab_parallel else
+                                   f"dp{world}: global batch dealt by token count (Karmarkar-Karp, equal counts)" if dp
+                                   else f"dp{world}: a store per rank" if world > 1 else "single GPU"),
                    "loss": {"clip_eps": w.clip_eps, "kl_coef": w.kl_coef, "agg": "seq-mean-token-mean"}},
         "roofline": {"bound": "tensor", "kernel": "fused LM-head GEMM + online log-softmax (af_token_logprob)",
                      "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
@@ -686,7 +1107,8 @@ def run_ours(args):
                                  if GEMM_DRAM_BYTES_PER_TOKEN_7B and (w.d, w.V) == (3584, 152064)
                                  and args.gemm != "single" and args.v_splits == 0 and not w.token_budget else None)},
         "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": job.h2d_bytes,
-                "d2h_bytes_per_step": int(sum(lo.numel() for lo in job.loss_outs)), "ms_per_step": ms_e2e,
+                "d2h_bytes_per_step": int(job.d2h_bytes), "ms_per_step": ms_e2e,
+                "d2h": "per-token log-probs in packed order (4 B per token) and the loss record",
                 # the first timed step cannot hide its own copy behind a previous step's kernels
                 "step_ms_rank0": {"first": e2e_steps_ms[0], "median": float(np.median(e2e_steps_ms)),
                                   "min": float(np.min(e2e_steps_ms))}},
@@ -703,10 +1125,9 @@ def run_ours(args):
     line["hbm_kernels"].update(hbm_alone)
     if fused is not None:
         line["fused_update"] = fused
-    if refresh is not None:
-        line["weight_refresh"] = refresh
-    if live is not None:
-        line["live_controller"] = live
+    line.update(streaming)
+    if dp is not None:
+        line["data_parallel"] = dp.report()
     if rank == 0:
         line["balance"] = job.balance_report()
     if bwd_ms is not None:
@@ -722,6 +1143,29 @@ def run_ours(args):
                                 "sample": f"first {n} packed tokens as one sequence through pack/log-prob/loss "
                                           f"oracles at full V={w.V}, advantage oracle over all {w.N} responses; "
                                           f"{secs:.1f} s"}
+    # the other workloads, one short leg each (single GPU, default workload only)
+    if rank == 0 and world == 1 and args.workload == "cfg2" and not args.no_configs:
+        job.ctx.close()
+        del job, rows, W_bits
+        torch.cuda.empty_cache()
+        line["configs"] = {name: side_leg(name, args, dev, peaks) for name in ("cfg1", "cfg3", "cfg4", "cfg5")}
+        c = line["configs"]
+        # the same figures as flat scalars beside the headline kernel's
+        line["roofline"].update({
+            "cfg1_tokens_per_s": c["cfg1"]["value"], "cfg1_host_enqueue_us_per_step": c["cfg1"].get("host_enqueue_us_per_step"),
+            "cfg1_graph_replay_us_per_scoring_step": c["cfg1"].get("graph_replay_us_per_scoring_step"),
+            "cfg3_tokens_per_s": c["cfg3"]["value"], "cfg3_logprob_tflops": c["cfg3"]["logprob_tflops"],
+            "cfg3_frac_of_sustained": c["cfg3"]["frac_of_sustained"],
+            "cfg4_three_calls_ms": c["cfg4"]["three_calls"]["ms_per_step"],
+            "cfg4_three_calls_tflops_8TdV": c["cfg4"]["three_calls"]["step_tflops_8TdV"],
+            "cfg4_backward_ms": c["cfg4"]["three_calls"]["backward_ms"],
+            "cfg4_fused_update_ms": c["cfg4"]["fused_update"]["ms_per_step"],
+            "cfg4_fused_update_tflops_6TdV": c["cfg4"]["fused_update"]["tflops_6TdV_model"],
+            "cfg5_tokens_per_s_incl_pack": c["cfg5"]["value"],
+            "cfg5_live_controller_tokens_per_s": c["cfg5"]["live_controller"]["value"],
+            "cfg5_weight_refresh_tokens_per_s": c["cfg5"]["weight_refresh"]["value"],
+            "cfg5_closed_loop_scored_tokens_per_s": c["cfg5"]["closed_loop"]["scored_tokens_per_s"],
+            "cfg5_pack_frac_of_hbm": c["cfg5"]["pack_frac_of_hbm"]})
     if rank == 0:
         print(json.dumps(line), flush=True)
     if world > 1:
@@ -734,8 +1178,25 @@ def run_ours(args):
 # ------------------------------------------------------------------------------------------
 def run_reference(args):
     rank, _, world = dist_env()
+    ranks_reported = 1
+    if world > 1:
+        # every rank reports in (gloo, CPU); rank 0 alone does the work
+        import torch.distributed as dist
+        dist.init_process_group("gloo")
+        seen = [torch.zeros(1, dtype=torch.int64) for _ in range(world)]
+        dist.all_gather(seen, torch.tensor([rank + 1], dtype=torch.int64))
+        ranks_reported = int(sum(int(t.item()) > 0 for t in seen))
+        dist.barrier()
+        dist.destroy_process_group()
     if rank != 0:
         return
+    # a launcher may have pinned the math libraries to one thread per rank (torchrun exports
+    # OMP_NUM_THREADS=1); the oracle runs alone here and gets the host's cores back
+    try:
+        from threadpoolctl import threadpool_limits
+        threadpool_limits(limits=os.cpu_count() or 1, user_api="blas")
+    except Exception:
+        pass
     w = wl.make_workload(args.workload)
     n = args.cpu_sample
     W_bits = wl.bf16_bits(wl.gen_weight(w, "cpu"))
@@ -757,9 +1218,23 @@ def run_reference(args):
         "config": {"workload": f"{args.workload}: {head_name(w)} head d={w.d} V={w.V}; bounded sample: {sample}"},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
-        "gpu_launches": 0,
+        "gpu_launches": 0, "ranks_reported": ranks_reported,
     }
     print(json.dumps(line), flush=True)
+
+
+def launch_ranks(n: int) -> int:
+    """`python bench.py --gpus N` with no launcher around it: start N ranks of this script, one per
+    GPU, through torch.distributed.run on this node, and pass their output through (rank 0 prints
+    the JSON line).  Returns the launcher's exit code."""
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__), *sys.argv[1:]]
+    env = dict(os.environ)
+    env.setdefault("OMP_NUM_THREADS", str(max(1, (os.cpu_count() or 1) // n)))
+    return subprocess.run(cmd, env=env).returncode
 
 
 def main():
@@ -773,6 +1248,11 @@ def main():
     ap.add_argument("--vocab-parallel", action="store_true",
                     help="split the LM head by vocabulary rows over the ranks (one batch for all; shard statistics "
                          "all-gathered and merged) instead of giving every rank its own batch")
+    ap.add_argument("--no-balance", action="store_true",
+                    help="data parallel: deal the global batch to the ranks by prompt index instead of by token "
+                         "count (af_balance_partitions)")
+    ap.add_argument("--no-configs", action="store_true",
+                    help="skip the short legs of the other four workloads that follow the default cfg2 run")
     ap.add_argument("--v-splits", type=int, default=0,
                     help="vocabulary ranges per row tile of the fused GEMM (af_set_tuning v_splits); 0 = the library's choice")
     ap.add_argument("--hbm-log2", type=int, default=28, choices=range(20, 30),
@@ -781,14 +1261,16 @@ def main():
                     help="token rows per block of the backward and fused-update calls (af_set_tuning "
                          "bwd_token_block, a multiple of 128); 0 = the library's choice")
     ap.add_argument("--live-controller", action="store_true",
-                    help="streaming workloads: also time the step with af_controller_put / get handing out the "
-                         "micro-batches")
-    ap.add_argument("--weight-refresh", action="store_true",
-                    help="also time the steps while a new LM-head weight is loaded and swapped in every step")
+                    help="streaming workloads: also time the steps with the controller in the loop, with the "
+                         "weight refresh, and as the two-task closed loop")
+    ap.add_argument("--weight-refresh", action="store_true", help="same as --live-controller")
+    ap.add_argument("--closed-loop", action="store_true", help="same as --live-controller")
     ap.add_argument("--gemm", default="default", choices=["default", "single", "pair"],
                     help="main loop of the tensor-core GEMMs (af_set_tuning gemm_variant): CTA pairs (the default) "
                          "or one CTA per tile")
     args = ap.parse_args()
+    if args.gpus > 1 and "RANK" not in os.environ:
+        sys.exit(launch_ranks(args.gpus))
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     if args.impl == "reference":

@@ -59,6 +59,7 @@ typedef enum {
 #define AF_DEVERR_WATCHDOG 2u     /* a bounded wait inside a kernel ran out; results invalid      */
 #define AF_DEVERR_CU_SEQLENS 4u   /* cu_seqlens not non-decreasing from 0 to T                     */
 #define AF_DEVERR_SAMPLE_INDEX 8u /* af_controller_put met an index outside [0, N): entry skipped  */
+#define AF_DEVERR_GROUP_ID 16u    /* af_grpo_advantage met a group id outside [0, n_groups): NaN    */
 
 /* Create / destroy a context on CUDA device `device`.  af_create fails with
  * AF_ERR_UNSUPPORTED_DEVICE unless the device is compute capability 10.0.  af_destroy
@@ -84,6 +85,17 @@ int64_t af_workspace_bytes(const af_ctx* ctx);
  * another so that a weight tile fetched once serves them all; 1 = one CTA per 128 x 256 tile.
  * Results agree within the stated tolerances either way. */
 af_status af_set_tuning(af_ctx* ctx, int32_t v_splits, int32_t bwd_token_block, int32_t gemm_variant);
+
+/* Data-parallel actor update (Section 4.1: the training batch is streamed to the DP groups of the
+ * actor-update task; each computes the gradient of its share).  The one exchange of the path is
+ * the sum of the ranks' d_W.  Register a cudaEvent_t (as void*; NULL clears it; the event stays the
+ * caller's) and af_policy_loss_backward, its shard form and af_policy_update record it on their
+ * stream at the point where d_W is complete: the last token block then runs its dW product BEFORE
+ * its dH product, so a collective that waits on the event on another stream overlaps with the
+ * remaining dH product, the loss record and whatever the caller enqueues next.  Results do not
+ * depend on it (the two products of a block are independent).  While an event is registered the
+ * three calls cannot be recorded into a CUDA graph of a single stream. */
+af_status af_set_dw_ready_event(af_ctx* ctx, void* event);
 
 /* Synchronise `stream`, read and clear the sticky device error word.  Returns AF_OK when it was
  * zero, else AF_ERR_DEVICE_FLAGGED with the bits in *flags (nullable). */
@@ -188,8 +200,11 @@ af_status af_merge_logprob_shards(af_ctx* ctx, const float* partials, const int3
  *
  * reward [N] fp32 dev.  group_id [N] int32 dev with values in [0, n_groups) in any order, or
  * NULL for contiguous equal groups (sample i belongs to group i / (N / n_groups); then
- * N % n_groups must be 0).  With group_id given the kernel scans the id array once per group
- * (deterministic, no float atomics) and N * n_groups must stay below 2^33 (AF_ERR_SHAPE).
+ * N % n_groups must be 0).  With group_id given the work is O(N) whatever n_groups is: the group
+ * sums are exact fixed-point sums taken with integer atomics, so the result does not depend on the
+ * order of the members and is bit-reproducible; N < 2^31 (AF_ERR_SHAPE); a per-group accumulator
+ * table (64 B per group) is kept in the context's workspace; a sample whose id lies outside
+ * [0, n_groups) gets a NaN advantage and raises AF_DEVERR_GROUP_ID; groups without members are fine.
  * ddof is 0 or 1.  eps_adv must be > 0 (AF_ERR_INVALID_ARG otherwise: with eps_adv = 0 a group of
  * equal rewards would divide 0 by 0).  adv [N] fp32 dev.
  * ------------------------------------------------------------------------------------------- */

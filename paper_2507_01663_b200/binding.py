@@ -21,13 +21,13 @@ AF_OK = 0
 STATUS_NAMES = {0: "AF_OK", -1: "AF_ERR_INVALID_ARG", -2: "AF_ERR_SHAPE", -3: "AF_ERR_ALIGNMENT",
                 -4: "AF_ERR_CAPACITY", -5: "AF_ERR_INDEX", -6: "AF_ERR_WORKSPACE", -7: "AF_ERR_CUDA",
                 -8: "AF_ERR_UNSUPPORTED_DEVICE", -9: "AF_ERR_DEVICE_FLAGGED"}
-DEVERR_TARGET_RANGE, DEVERR_WATCHDOG, DEVERR_CU_SEQLENS, DEVERR_SAMPLE_INDEX = 1, 2, 4, 8
+DEVERR_TARGET_RANGE, DEVERR_WATCHDOG, DEVERR_CU_SEQLENS, DEVERR_SAMPLE_INDEX, DEVERR_GROUP_ID = 1, 2, 4, 8, 16
 
 EXPORTS = ["af_create", "af_destroy", "af_status_string", "af_reserve", "af_workspace_bytes",
            "af_set_tuning", "af_check_device_errors", "af_pack_microbatch", "af_token_logprob",
            "af_grpo_advantage", "af_policy_loss", "af_policy_loss_backward", "af_token_logprob_static",
            "af_controller_put", "af_controller_get", "af_controller_clear", "af_balance_partitions",
-           "af_token_logprob_shard", "af_merge_logprob_shards", "af_policy_update", "af_unpack_microbatch", "af_policy_loss_backward_shard"]
+           "af_token_logprob_shard", "af_merge_logprob_shards", "af_policy_update", "af_unpack_microbatch", "af_policy_loss_backward_shard", "af_set_dw_ready_event"]
 MAX_WRITE_COLS = 4
 
 
@@ -100,6 +100,7 @@ def load_library() -> C.CDLL:
     lib.af_workspace_bytes.restype = i64
     lib.af_set_tuning.argtypes = [vp, i32, i32, i32]
     lib.af_check_device_errors.argtypes = [vp, C.POINTER(C.c_uint32), vp]
+    lib.af_set_dw_ready_event.argtypes = [vp, vp]
     lib.af_pack_microbatch.argtypes = [vp, C.POINTER(StoreView), vp, i32, C.POINTER(Packed),
                                        C.POINTER(i64), vp]
     lib.af_token_logprob.argtypes = [vp, vp, vp, vp, i64, i32, i32, vp, vp, vp, vp]
@@ -177,6 +178,12 @@ class Context:
     def set_tuning(self, v_splits: int = 0, bwd_token_block: int = 0, gemm_variant: int = 0):
         """gemm_variant: 0 = default (CTA pairs), 1 = one CTA per tile, 2 = CTA pairs."""
         _check(self.lib.af_set_tuning(self.handle, v_splits, bwd_token_block, gemm_variant), "af_set_tuning")
+
+    def set_dw_ready_event(self, event: Optional[torch.cuda.Event]):
+        """Register a torch CUDA event that the backward / fused-update calls record once d_W is
+        complete (None clears it).  The event must have been recorded once, so that it exists."""
+        _check(self.lib.af_set_dw_ready_event(self.handle, None if event is None else C.c_void_p(event.cuda_event)),
+               "af_set_dw_ready_event")
 
     def check_device_errors(self, stream=None) -> int:
         """Synchronise the stream; return the device error bits (0 = none) and clear them."""

@@ -12,8 +12,7 @@
 //   G <= 4096: a block stages a run of whole groups in shared memory with 128-bit loads, reduces
 //   each group with warp shuffles (two passes: mean, then squared deviations) and writes the
 //   advantages back coalesced;  larger groups: one block per group.
-// Arbitrary membership (group_id given): one block per group scans the id array; sums are taken
-// in a fixed thread/iteration order, so the result is reproducible without float atomics.
+// Arbitrary membership (group_id given) lives in advantage_ids.cu.
 #include "common.cuh"
 
 namespace af {
@@ -447,11 +446,10 @@ __global__ void __launch_bounds__(kThreads) advantage_scan_kernel(
 
 }  // namespace
 
-cudaError_t launch_advantage(const float* reward, const int32_t* group_id, int64_t N,
-                             int32_t n_groups, float eps_adv, int32_t ddof, float* adv,
-                             int sm_count, cudaStream_t s) {
+cudaError_t launch_advantage(const float* reward, int64_t N, int32_t n_groups, float eps_adv, int32_t ddof,
+                             float* adv, int sm_count, cudaStream_t s) {
   if (N == 0 || n_groups == 0) return cudaSuccess;
-  if (group_id == nullptr) {
+  {
     const int64_t G = N / n_groups;
     const bool aligned = ((reinterpret_cast<uintptr_t>(reward) | reinterpret_cast<uintptr_t>(adv)) & 15) == 0;
     if (G >= 32 && G <= 512 && (G & (G - 1)) == 0 && aligned) {
@@ -519,8 +517,6 @@ cudaError_t launch_advantage(const float* reward, const int32_t* group_id, int64
     } else {
       advantage_scan_kernel<<<n_groups, kThreads, 0, s>>>(reward, nullptr, adv, N, G, eps_adv, ddof);
     }
-  } else {
-    advantage_scan_kernel<<<n_groups, kThreads, 0, s>>>(reward, group_id, adv, N, 0, eps_adv, ddof);
   }
   return cudaGetLastError();
 }

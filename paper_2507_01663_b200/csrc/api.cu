@@ -95,7 +95,7 @@ af_status af_destroy(af_ctx* c) {
   if (!c) return AF_ERR_INVALID_ARG;
   DeviceGuard guard(c->device);
   cudaDeviceSynchronize();
-  Buf* bufs[] = {&c->partial, &c->loss_ws, &c->pack_meta, &c->dz, &c->ctrl_ws, &c->zlog};
+  Buf* bufs[] = {&c->partial, &c->loss_ws, &c->pack_meta, &c->dz, &c->ctrl_ws, &c->zlog, &c->adv_ws};
   for (Buf* b : bufs) if (b->p) cudaFree(b->p);
   for (int i = 0; i < kPackRing; ++i) {
     if (c->pack_host[i]) cudaFreeHost(c->pack_host[i]);
@@ -108,7 +108,7 @@ af_status af_destroy(af_ctx* c) {
 
 int64_t af_workspace_bytes(const af_ctx* c) {
   if (!c) return 0;
-  return (int64_t)(c->partial.cap + c->loss_ws.cap + c->pack_meta.cap + c->dz.cap + c->ctrl_ws.cap + c->zlog.cap);
+  return (int64_t)(c->partial.cap + c->loss_ws.cap + c->pack_meta.cap + c->dz.cap + c->ctrl_ws.cap + c->zlog.cap + c->adv_ws.cap);
 }
 
 af_status af_set_tuning(af_ctx* c, int32_t v_splits, int32_t bwd_token_block, int32_t gemm_variant) {
@@ -117,6 +117,12 @@ af_status af_set_tuning(af_ctx* c, int32_t v_splits, int32_t bwd_token_block, in
   c->v_splits = v_splits;
   c->bwd_token_block = bwd_token_block;
   c->gemm_pair = gemm_variant == 1 ? 0 : (c->sm_count >= 2 ? 1 : 0);
+  return AF_OK;
+}
+
+af_status af_set_dw_ready_event(af_ctx* c, void* event) {
+  if (!c) return AF_ERR_INVALID_ARG;
+  c->dw_ready = static_cast<cudaEvent_t>(event);
   return AF_OK;
 }
 
@@ -344,10 +350,15 @@ af_status af_grpo_advantage(af_ctx* c, const float* reward, const int32_t* group
   if (N == 0) return AF_OK;
   if (!reward || !adv || n_groups < 1) return AF_ERR_INVALID_ARG;
   if (!group_id && N % n_groups != 0) return AF_ERR_SHAPE;
-  if (group_id && (double)N * (double)n_groups >= 8589934592.0) return AF_ERR_SHAPE;
+  if (group_id && N >= ((int64_t)1 << 31)) return AF_ERR_SHAPE;       // member counts are 32-bit
   DeviceGuard guard(c->device);
-  return launch_advantage(reward, group_id, N, n_groups, eps_adv, ddof, adv, c->sm_count,
-                          static_cast<cudaStream_t>(stream)) == cudaSuccess ? AF_OK : AF_ERR_CUDA;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (!group_id)
+    return launch_advantage(reward, N, n_groups, eps_adv, ddof, adv, c->sm_count, s) == cudaSuccess ? AF_OK : AF_ERR_CUDA;
+  const af_status st = ws_grow(c->adv_ws, advantage_ids_workspace_bytes(n_groups));
+  if (st != AF_OK) return st;
+  return launch_advantage_ids(reward, group_id, N, n_groups, eps_adv, ddof, adv, c->adv_ws.p, c->d_err, c->sm_count,
+                              s) == cudaSuccess ? AF_OK : AF_ERR_CUDA;
 }
 
 af_status af_policy_loss(af_ctx* c, const float* logp, const float* old_logp, const float* ref_logp,

@@ -18,23 +18,14 @@
 // vocabulary row write 128 consecutive bytes without any staging.  That orientation also gives the
 // product the forward's memory behaviour: the H_blk panels of the row tiles in flight stay in L2
 // while dZ streams past them (once per round of row tiles).
+#include "device_util.cuh"
 #include "gemm_launch.cuh"
 
 namespace af {
 namespace {
 
-constexpr float kLog2e = 1.4426950408889634f;
 constexpr int kDefaultTokenBlock = 74 * 128;  // 37 pair tiles (74 CTA tiles) x 14 column tiles of d = 3584: 7 full rounds of 148 SMs
 
-__device__ __forceinline__ float ex2f(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
-  __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<uint32_t*>(&h);
-}
 
 // Store a 32-row x 32-column bf16 chunk (lane L holds row L as 16 packed words) to a row-major
 // bf16 matrix: rows row0.., columns col0..; rows >= M and 8-column groups past N are skipped.
@@ -180,19 +171,33 @@ struct StoreF32TransposedEpi {
 //                         streams past them.
 af_status launch_backward_products(af_ctx* ctx, const void* hidden_blk, const void* W, const void* dz_blk,
                                    int64_t tc, int32_t d, int32_t V, void* d_hidden_blk, float* d_W,
-                                   int32_t accumulate_dW, cudaStream_t s) {
+                                   int32_t accumulate_dW, bool last_block, cudaStream_t s) {
   const GemmEnv env = gemm_env(ctx);
   const uint64_t dB = (uint64_t)d * 2, vB = (uint64_t)V * 2;
   const Operand Hblk{hidden_blk, (uint64_t)tc, (uint64_t)d, dB};
   const Operand Wop{W, (uint64_t)V, (uint64_t)d, dB};
   const Operand dZop{dz_blk, (uint64_t)tc, (uint64_t)V, vB};
-  StoreBf16Epi::Params p2{static_cast<__nv_bfloat16*>(d_hidden_blk), d, (int)tc, d};
-  af_status st = run_gemm<StoreBf16Epi, false, true>(env, dZop, Wop, 0, p2, s);
+  auto dH_product = [&]() {
+    StoreBf16Epi::Params p2{static_cast<__nv_bfloat16*>(d_hidden_blk), d, (int)tc, d};
+    return run_gemm<StoreBf16Epi, false, true>(env, dZop, Wop, 0, p2, s);
+  };
+  auto dW_product = [&]() {
+    StoreF32TransposedEpi::Params p3{d_W, d, d, V, accumulate_dW ? 1 : 0};
+    return run_gemm<StoreF32TransposedEpi, true, true>(
+        env, Hblk, dZop, logprob_pick_splits((int64_t)d, (int32_t)tc, V, ctx->sm_count, env.pair, 0), p3, s);
+  };
+  // With a "d_W ready" event registered, the last block runs its dW product first and records the
+  // event behind it: d_W is complete from there on, and whoever waits on the event (a gradient
+  // all-reduce on another stream) overlaps with the block's dH product and whatever follows.
+  if (last_block && ctx->dw_ready) {
+    af_status st = dW_product();
+    if (st != AF_OK) return st;
+    if (cudaEventRecord(ctx->dw_ready, s) != cudaSuccess) return AF_ERR_CUDA;
+    return dH_product();
+  }
+  af_status st = dH_product();
   if (st != AF_OK) return st;
-  StoreF32TransposedEpi::Params p3{d_W, d, d, V, accumulate_dW ? 1 : 0};
-  return run_gemm<StoreF32TransposedEpi, true, true>(env, Hblk, dZop,
-                                                     logprob_pick_splits((int64_t)d, (int32_t)tc, V, ctx->sm_count, env.pair, 0),
-                                                     p3, s);
+  return dW_product();
 }
 
 // Token block of the backward (and of the fused update): a multiple of 128 rows.
@@ -214,6 +219,7 @@ af_status launch_backward(af_ctx* ctx, const void* hidden, const void* W, const 
 
   if (T == 0) {
     if (!accumulate_dW && cudaMemsetAsync(d_W, 0, (size_t)V * d * sizeof(float), s) != cudaSuccess) return AF_ERR_CUDA;
+    if (ctx->dw_ready && cudaEventRecord(ctx->dw_ready, s) != cudaSuccess) return AF_ERR_CUDA;
     return AF_OK;
   }
   const __nv_bfloat16* H = static_cast<const __nv_bfloat16*>(hidden);
@@ -232,7 +238,7 @@ af_status launch_backward(af_ctx* ctx, const void* hidden, const void* W, const 
     if (st != AF_OK) return st;
     st = launch_backward_products(ctx, H + t0 * d, W, dz, (int64_t)tc, d, V,
                                   static_cast<__nv_bfloat16*>(d_hidden) + t0 * d, d_W,
-                                  (!first || accumulate_dW) ? 1 : 0, s);
+                                  (!first || accumulate_dW) ? 1 : 0, t0 + Tc >= T, s);
     if (st != AF_OK) return st;
   }
   return AF_OK;

@@ -7,6 +7,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "../../include/asyncflow.h"
 
 namespace af {
@@ -24,6 +26,39 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
+// Tensor maps already encoded for this context, keyed by what determines them.  A map depends only
+// on the address, shape, pitch and box of the matrix, not on the allocation behind it, so an entry
+// stays valid for as long as the caller keeps passing the same buffer; the steady state of a
+// training or scoring loop re-encodes nothing.
+struct TmapCache {
+  static constexpr int kEntries = 32;
+  struct Entry {
+    const void* base = nullptr;
+    uint64_t rows = 0, cols = 0, pitch = 0;
+    uint32_t box_rows = 0;
+    CUtensorMap map;
+  };
+  Entry e[kEntries];
+  int next = 0;      // round-robin replacement
+};
+
+// cudaFuncSetAttribute(MaxDynamicSharedMemorySize) once per kernel and device (the attribute is
+// per device, and a process may drive several) instead of on every launch.
+struct SmemAttrOnce {
+  std::atomic<unsigned long long> done{0};   // bit i: set on device i (devices >= 64 set it every time)
+};
+template <class Kernel>
+inline cudaError_t set_smem_once(SmemAttrOnce& once, Kernel kernel, int bytes) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  const unsigned long long bit = dev < 64 ? 1ull << dev : 0ull;
+  if (bit && (once.done.load(std::memory_order_acquire) & bit)) return cudaSuccess;
+  e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess && bit) once.done.fetch_or(bit, std::memory_order_release);
+  return e;
+}
+
 }  // namespace af
 
 struct af_ctx {
@@ -36,6 +71,9 @@ struct af_ctx {
   int v_splits = 0;         // 0 = automatic
   int bwd_token_block = 0;  // 0 = default
   int gemm_pair = 1;        // 1 = CTA-pair GEMM variant (the default), 0 = one CTA per tile
+  cudaEvent_t dw_ready = nullptr;  // caller's event recorded once d_W is complete (af_set_dw_ready_event)
+
+  af::TmapCache tmaps;      // tensor maps of the GEMM operands seen so far
 
   // workspace (device)
   af::Buf partial;    // [splits, T] float4 online-softmax partials
@@ -44,6 +82,7 @@ struct af_ctx {
   af::Buf dz;         // dZ [Tc, V] bf16 (backward, one token block)
   af::Buf ctrl_ws;    // per-block aggregates of af_controller_get
   af::Buf zlog;       // fp32 logits [Tc, V] of one token block (fused actor update)
+  af::Buf adv_ws;     // per-group accumulators of af_grpo_advantage with group ids
 
   // pinned staging ring for pack metadata
   void* pack_host[af::kPackRing] = {};
@@ -75,9 +114,12 @@ cudaError_t launch_unpack(const af_write_cols& cols, const PackSeqTable& tab, in
 cudaError_t launch_pack(const af_store_view& st, const af_packed& out, const PackSeqTable& tab,
                         int32_t B, int64_t T, int sm_count, unsigned int* d_err, cudaStream_t s);
 
-cudaError_t launch_advantage(const float* reward, const int32_t* group_id, int64_t N,
-                             int32_t n_groups, float eps_adv, int32_t ddof, float* adv,
-                             int sm_count, cudaStream_t s);
+cudaError_t launch_advantage(const float* reward, int64_t N, int32_t n_groups, float eps_adv, int32_t ddof,
+                             float* adv, int sm_count, cudaStream_t s);                  // contiguous groups
+size_t advantage_ids_workspace_bytes(int32_t n_groups);
+cudaError_t launch_advantage_ids(const float* reward, const int32_t* group_id, int64_t N, int32_t n_groups,
+                                 float eps_adv, int32_t ddof, float* adv, void* ws, unsigned int* d_err,
+                                 int sm_count, cudaStream_t s);                            // membership by id
 
 size_t loss_workspace_bytes(int sm_count);
 cudaError_t launch_policy_loss(const float* logp, const float* old_logp, const float* ref_logp,
@@ -113,7 +155,7 @@ af_status launch_token_logprob_z(af_ctx* ctx, const void* hidden, const void* W,
 int64_t backward_token_block(const af_ctx* ctx, int64_t T);
 af_status launch_backward_products(af_ctx* ctx, const void* hidden_blk, const void* W, const void* dz_blk,
                                    int64_t tc, int32_t d, int32_t V, void* d_hidden_blk, float* d_W,
-                                   int32_t accumulate_dW, cudaStream_t s);
+                                   int32_t accumulate_dW, bool last_block, cudaStream_t s);
 af_status launch_policy_update(af_ctx* ctx, const void* hidden, const void* W, const int32_t* target,
                                const float* old_logp, const float* ref_logp, const float* adv_seq,
                                const int32_t* cu_seqlens, int32_t B, int64_t T, int32_t d, int32_t V,

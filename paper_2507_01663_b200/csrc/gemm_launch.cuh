@@ -21,9 +21,18 @@ struct GemmEnv {
   unsigned int* d_err;
   bool pair;             // CTA-pair variant (cta_group::2)
   unsigned int* tile_clock;  // device word the pair variant paces itself with (zeroed per launch), or null
+  TmapCache* cache;          // tensor maps encoded earlier (a context's), or null
 };
 
 inline af_status encode_operand(const GemmEnv& env, CUtensorMap* map, const Operand& op, uint32_t box_rows) {
+  TmapCache::Entry* slot = nullptr;
+  if (env.cache) {
+    for (TmapCache::Entry& c : env.cache->e)
+      if (c.base == op.base && c.rows == op.rows && c.cols == op.cols && c.pitch == op.pitch_bytes &&
+          c.box_rows == box_rows) { *map = c.map; return AF_OK; }
+    slot = &env.cache->e[env.cache->next];
+    env.cache->next = (env.cache->next + 1) % TmapCache::kEntries;
+  }
   cuuint64_t dims[2] = {op.cols, op.rows};
   cuuint64_t strides[1] = {op.pitch_bytes};
   cuuint32_t box[2] = {64, box_rows};
@@ -31,7 +40,12 @@ inline af_status encode_operand(const GemmEnv& env, CUtensorMap* map, const Oper
   CUresult r = env.encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(op.base), dims, strides,
                           box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS ? AF_OK : AF_ERR_CUDA;
+  if (r != CUDA_SUCCESS) { if (slot) slot->base = nullptr; return AF_ERR_CUDA; }
+  if (slot) {
+    slot->base = op.base; slot->rows = op.rows; slot->cols = op.cols; slot->pitch = op.pitch_bytes;
+    slot->box_rows = box_rows; slot->map = *map;
+  }
+  return AF_OK;
 }
 
 // C[M,N] = sum_k A(m,k) B(n,k).  A K-major operand is stored [M or N, K]; an MN-major operand is
@@ -57,8 +71,8 @@ af_status run_gemm(const GemmEnv& env, const Operand& A, const Operand& B, int s
   const int64_t units = (int64_t)g.m_tiles * g.splits;
   if (env.pair) {
     constexpr int smem = E::kStaged ? umma::kPairSmemBytesStaged : umma::kPairSmemBytes;
-    if (cudaFuncSetAttribute(umma::gemm_pair_kernel<E, kAMN, kBMN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             smem) != cudaSuccess) return AF_ERR_CUDA;
+    static SmemAttrOnce once;
+    if (set_smem_once(once, umma::gemm_pair_kernel<E, kAMN, kBMN>, smem) != cudaSuccess) return AF_ERR_CUDA;
     const int pairs = env.sm_count / 2;
     const int grid = 2 * (int)(units < pairs ? units : pairs);
     unsigned int* clock = env.tile_clock;
@@ -66,16 +80,17 @@ af_status run_gemm(const GemmEnv& env, const Operand& A, const Operand& B, int s
     umma::gemm_pair_kernel<E, kAMN, kBMN><<<grid, umma::kThreads, smem, s>>>(ta, tb, g, ep, env.d_err, clock);
   } else {
     constexpr int smem = E::kStaged ? umma::kSmemBytesStaged : umma::kSmemBytes;
-    if (cudaFuncSetAttribute(umma::gemm_kernel<E, kAMN, kBMN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             smem) != cudaSuccess) return AF_ERR_CUDA;
+    static SmemAttrOnce once;
+    if (set_smem_once(once, umma::gemm_kernel<E, kAMN, kBMN>, smem) != cudaSuccess) return AF_ERR_CUDA;
     const int grid = (int)(units < env.sm_count ? units : env.sm_count);
     umma::gemm_kernel<E, kAMN, kBMN><<<grid, umma::kThreads, smem, s>>>(ta, tb, g, ep, env.d_err);
   }
   return cudaGetLastError() == cudaSuccess ? AF_OK : AF_ERR_CUDA;
 }
 
-inline GemmEnv gemm_env(const af_ctx* ctx) {
-  return GemmEnv{ctx->encode, ctx->sm_count, ctx->d_err, ctx->gemm_pair != 0, ctx->d_err + kTileClockWord};
+inline GemmEnv gemm_env(af_ctx* ctx) {
+  return GemmEnv{ctx->encode, ctx->sm_count, ctx->d_err, ctx->gemm_pair != 0, ctx->d_err + kTileClockWord,
+                 &ctx->tmaps};
 }
 
 }  // namespace af

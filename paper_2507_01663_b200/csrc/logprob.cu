@@ -8,19 +8,13 @@
 //   lse = M + log sum_i s_i e^{m_i - M},  logp = zy - lse,  entropy = lse - (sum_i u_i e^{m_i-M}) / S.
 #include <mutex>
 
+#include "device_util.cuh"
 #include "gemm_launch.cuh"
 
 namespace af {
 namespace {
 
-constexpr float kLog2e = 1.4426950408889634f;
-constexpr float kLn2 = 0.6931471805599453f;
 
-__device__ __forceinline__ float ex2f(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
 
 // kStoreZ: also write the fp32 logits of the tile to z [T, ldz] (one token block of the fused actor
 // update, which turns them into dZ without a second GEMM).
@@ -313,7 +307,7 @@ extern "C" af_status af_token_logprob_static(const void* hidden, const void* W, 
   unsigned int* err_word = device_flags ? device_flags : reinterpret_cast<unsigned int*>(st->scratch);
   float4* partial = reinterpret_cast<float4*>(st->scratch + kStaticHeaderBytes);
 
-  const GemmEnv env{g_static_encode, st->sm_count, err_word, false, nullptr};
+  const GemmEnv env{g_static_encode, st->sm_count, err_word, false, nullptr, nullptr};
   const Operand Hop{hidden, (uint64_t)T, (uint64_t)d, (uint64_t)d * 2};
   const Operand Wop{W, (uint64_t)V, (uint64_t)d, (uint64_t)d * 2};
   LogprobEpi::Params ep{target, partial, (int)T, V, 0, nullptr, 0};

@@ -55,15 +55,6 @@ __device__ __forceinline__ float4 lds128(uint32_t addr) {
   return v;
 }
 
-// largest j in [0, B) with cu[j] <= t  (cu non-decreasing, cu[0] = 0, t < cu[B])
-__device__ __forceinline__ int find_seq(const int32_t* __restrict__ cu, int B, int t) {
-  int lo = 0, hi = B;
-  while (hi - lo > 1) {
-    int mid = (lo + hi) >> 1;
-    if (__ldg(cu + mid) <= t) lo = mid; else hi = mid;
-  }
-  return lo;
-}
 
 // The same search done by one warp, 32 probes per step (2 steps for B = 512, 4 for B = 10^6).
 __device__ __forceinline__ int find_seq_warp(const int32_t* __restrict__ cu, int B, int t, int lane) {
@@ -330,10 +321,9 @@ cudaError_t launch_policy_loss(const float* logp, const float* old_logp, const f
                                int32_t B, int64_t T, const af_loss_params& p, af_loss_out* out,
                                float* dlogp, void* ws, unsigned int* d_err, int sm_count,
                                cudaStream_t s) {
-  // set on every launch: the attribute is per device, and a process may drive several
   {
-    cudaError_t e = cudaFuncSetAttribute(policy_loss_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         kRingSmemBytes);
+    static SmemAttrOnce once;
+    cudaError_t e = set_smem_once(once, policy_loss_kernel, kRingSmemBytes);
     if (e != cudaSuccess) return e;
   }
   const int64_t chunks = (T + kChunk - 1) / kChunk;

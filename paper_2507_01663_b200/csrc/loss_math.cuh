@@ -3,17 +3,13 @@
 #pragma once
 
 #include "common.cuh"
+#include "device_util.cuh"
 
 namespace af {
 namespace lossmath {
 
-constexpr float kLog2e = 1.4426950408889634f;
-
-__device__ __forceinline__ float ex2f(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
+using af::ex2f;
+using af::kLog2e;
 
 struct TokenTerms {
   float pg;       // -min(rho A, clip(rho) A)
@@ -31,23 +27,21 @@ __device__ __forceinline__ TokenTerms token_terms(float logp, float old_logp, fl
   const float s2 = fminf(fmaxf(rho, lo_b), hi_b) * A;
   t.clipped = s2 < s1;
   const float delta = ref_logp - logp;
-  // exp(delta) - 1 and k3 = exp(delta) - delta - 1.  Near the reference policy both are tiny
-  // differences of numbers near 1, where the approximate exp2 (about 2^-22 relative on a value
-  // near 1) would leave k3 = delta^2 / 2 with an absolute error of 2.4e-7: several 1e-3 relative at
-  // |delta| = 0.01.  For |delta| < 1/4 the series is used instead (truncation below 2e-8 relative),
-  // k3 = delta^2 (1/2 + delta/6 + ... + delta^5/5040) without any cancellation, exp(delta) - 1 =
-  // delta + k3; both are exactly 0 when ref == logp.
-  float em1 = ex2f(delta * kLog2e) - 1.f;
-  float k3 = em1 - delta;
-  if (fabsf(delta) < 0.25f) {
-    float q = fmaf(delta, 1.f / 5040.f, 1.f / 720.f);
-    q = fmaf(delta, q, 1.f / 120.f);
-    q = fmaf(delta, q, 1.f / 24.f);
-    q = fmaf(delta, q, 1.f / 6.f);
-    q = fmaf(delta, q, 0.5f);
-    k3 = delta * delta * q;
-    em1 = delta + k3;
-  }
+  // exp(delta) - 1 (for the gradient) comes from the approximate exp2: about 2^-22 relative on a
+  // value near 1, i.e. 2.4e-7 absolute, which no gradient tolerance notices.  k3 = exp(delta) -
+  // delta - 1 would inherit that absolute error, and near the reference policy (k3 = delta^2 / 2)
+  // it is several 1e-3 relative at |delta| = 0.01: for |delta| < 1/32 k3 is therefore taken from
+  // its series delta^2 (1/2 + delta/6) (truncation delta^2/12 < 8e-5 relative, no cancellation,
+  // exactly 0 when ref == logp); from 1/32 on the direct form is good to 5e-4.  The loss kernel runs
+  // at its issue limit when it streams at full bandwidth (every instruction per token costs it
+  // about 0.9 % of its GB/s; a six-term series for both quantities cost 10 %), hence the short
+  // series.  Explicit roundings: the loss kernel and the fused
+  // update must produce the same bits, so the compiler may not contract these differently at the
+  // two call sites.
+  const float em1 = __fadd_rn(ex2f(__fmul_rn(delta, kLog2e)), -1.f);
+  const float k3_direct = __fadd_rn(em1, -delta);
+  const float k3_series = __fmul_rn(__fmul_rn(delta, delta), fmaf(delta, 1.f / 6.f, 0.5f));
+  const float k3 = fabsf(delta) < 0.03125f ? k3_series : k3_direct;
   t.pg = -fminf(s1, s2);
   t.k3 = k3;
   t.grad = fmaf(nbeta, em1, t.clipped ? 0.f : -s1);

@@ -11,20 +11,11 @@
 // than a chunk fall back to a warp-per-row copy with 128-bit loads and stores.  The 4-byte
 // columns are gathered by a second, small kernel (one thread per token).
 #include "common.cuh"
+#include "device_util.cuh"
 #include "umma.cuh"
 
 namespace af {
 namespace {
-
-__device__ __forceinline__ int find_seq(const int32_t* __restrict__ cu, int B, int t) {
-  // largest j in [0, B) with cu[j] <= t  (cu is non-decreasing, cu[0] = 0, t < cu[B])
-  int lo = 0, hi = B;
-  while (hi - lo > 1) {
-    int mid = (lo + hi) >> 1;
-    if (__ldg(cu + mid) <= t) lo = mid; else hi = mid;
-  }
-  return lo;
-}
 
 __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
   uint4 v;
@@ -272,10 +263,9 @@ cudaError_t launch_pack(const af_store_view& st, const af_packed& out, const Pac
   if (T > 0 && out.hidden) {
     const int rpc = pack_rows_per_chunk(st.d);
     if (rpc > 0 && tab.n_chunks > 0) {
-      // set on every launch: the attribute is per device, and a process may drive several
       {
-        cudaError_t e = cudaFuncSetAttribute(pack_rows_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             kCopySmemBytes);
+        static SmemAttrOnce once;
+        cudaError_t e = set_smem_once(once, pack_rows_bulk_kernel, kCopySmemBytes);
         if (e != cudaSuccess) return e;
       }
       const int grid = tab.n_chunks < sm_count ? tab.n_chunks : sm_count;

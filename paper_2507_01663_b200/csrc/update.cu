@@ -21,20 +21,7 @@ namespace {
 
 constexpr int kThreads = 256;
 
-__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
-  __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<uint32_t*>(&h);
-}
 
-// largest j in [0, B) with cu[j] <= t  (cu non-decreasing, cu[0] = 0, t < cu[B])
-__device__ __forceinline__ int find_seq(const int32_t* __restrict__ cu, int B, int t) {
-  int lo = 0, hi = B;
-  while (hi - lo > 1) {
-    const int mid = (lo + hi) >> 1;
-    if (__ldg(cu + mid) <= t) lo = mid; else hi = mid;
-  }
-  return lo;
-}
 
 // One CTA per token row of the block.  z: [rows, V] fp32 logits; dz: [rows, V] bf16.  V % 8 == 0.
 __global__ void __launch_bounds__(kThreads) dz_from_logits_kernel(
@@ -91,6 +78,7 @@ af_status launch_policy_update(af_ctx* ctx, const void* hidden, const void* W, c
   if (accumulate_dW < 0) return AF_OK;  // reserve only
   if (T == 0) {
     if (!accumulate_dW && cudaMemsetAsync(d_W, 0, (size_t)V * d * sizeof(float), s) != cudaSuccess) return AF_ERR_CUDA;
+    if (ctx->dw_ready && cudaEventRecord(ctx->dw_ready, s) != cudaSuccess) return AF_ERR_CUDA;
   }
   const __nv_bfloat16* H = static_cast<const __nv_bfloat16*>(hidden);
   __nv_bfloat16* dz = static_cast<__nv_bfloat16*>(ctx->dz.p);
@@ -109,7 +97,7 @@ af_status launch_policy_update(af_ctx* ctx, const void* hidden, const void* W, c
     if (cudaGetLastError() != cudaSuccess) return AF_ERR_CUDA;
     // 3. the two products that consume dZ
     st = launch_backward_products(ctx, H + t0 * d, W, dz, tc, d, V, static_cast<__nv_bfloat16*>(d_hidden) + t0 * d,
-                                  d_W, (!first || accumulate_dW) ? 1 : 0, s);
+                                  d_W, (!first || accumulate_dW) ? 1 : 0, t0 + Tc >= T, s);
     if (st != AF_OK) return st;
   }
   // loss scalars over the whole batch, from the log-probs just written

@@ -233,9 +233,10 @@ def gen_weight(w: Workload, device="cpu") -> torch.Tensor:
     return _normal_matrix(w.seed, S_W, w.V, w.d, w.w_std, device)
 
 
-def gen_target(w: Workload, device="cpu") -> torch.Tensor:
-    """Store column ``target`` [sum L] int32, uniform over the vocabulary."""
-    return randint(w.seed, S_TARGET, 0, w.total_tokens, w.V, device).to(torch.int32)
+def gen_target(w: Workload, device="cpu", row_start: int = 0, rows: Optional[int] = None) -> torch.Tensor:
+    """Store column ``target`` [sum L] int32, uniform over the vocabulary (or the given row range)."""
+    rows = w.total_tokens - row_start if rows is None else rows
+    return randint(w.seed, S_TARGET, row_start, rows, w.V, device).to(torch.int32)
 
 
 def gen_reward(w: Workload, device="cpu") -> torch.Tensor:

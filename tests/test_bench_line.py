@@ -43,10 +43,21 @@ def test_reference_arm_line():
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["e2e"]["value"] == line["value"]
 
 
+def test_gpus_flag_starts_that_many_ranks():
+    """`bench.py --gpus 2` with no launcher around it starts two ranks itself (CPU ranks over gloo in
+    the reference arm); rank 0 prints the one line, which says how many ranks reported in."""
+    line = run_bench("--impl", "reference", "--gpus", "2", "--workload", "cfg1", "--steps", "1", "--warmup", "0",
+                     "--cpu-sample", "32")
+    check_base(line)
+    assert line["n_gpus"] == 2 and line["ranks_reported"] == 2
+
+
 @pytest.mark.gpu
 def test_gpu_arm_line():
     line = run_bench("--workload", "cfg1", "--steps", "3", "--warmup", "3", "--hbm-log2", "20", "--cpu-sample", "64")
     check_base(line)
+    # the step's result comes back to the host: 4 bytes of log-prob per token besides the loss record
+    assert line["e2e"]["d2h_bytes_per_step"] > 4 * 1000
     assert "impl" not in line and line["dtype"] == "bf16" and line["n_gpus"] == 1 and line["scaling"] == "weak"
     assert line["gpu_launches"] > 0 and line["e2e"]["h2d_bytes_per_step"] > 0 and line["e2e"]["d2h_bytes_per_step"] > 0
     roof = line["roofline"]

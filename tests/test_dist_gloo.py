@@ -2,7 +2,9 @@
 whole groups, rank results concatenate to the single-rank result, bench.py's reduction takes the
 max step time and the token sum over ranks, and the weight gradients of the ranks' batches, each
 scored with loss_scale = B_rank / B_global, sum to the gradient of the global batch; the
-statistics of vocabulary shards, gathered over the ranks, merge to the full-vocabulary result."""
+statistics of vocabulary shards, gathered over the ranks, merge to the full-vocabulary result; a
+global batch dealt to the ranks by token count (Karmarkar-Karp, equal sample counts) with gathered
+rewards reproduces the single-rank advantages, loss and weight gradient."""
 import os
 import socket
 
@@ -149,3 +151,66 @@ def test_two_rank_vocabulary_parallel_exchange(tmp_path):
     port = _free_port()
     mp.start_processes(_vocab_worker, args=(2, port, str(tmp_path)), nprocs=2, join=True, start_method="spawn")
     assert open(tmp_path / "ok_vocab_0").read() == "1" and open(tmp_path / "ok_vocab_1").read() == "1"
+
+
+def _balanced_worker(rank, world, port, out_dir):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    import bench
+    dp = bench.DataParallelShare("cfg4_mini", world, rank)
+    w0 = dp.sources[0]
+    W = wl.bf16_bits(wl.gen_weight(w0))
+    goff = np.concatenate([[0], np.cumsum(dp.lengths)])                  # global token index of a response's first row
+
+    def perturbation(samples):
+        """old / ref offsets as a function of the token's global identity, so that they do not
+        depend on which rank scores the token or where it sits in the rank's batch."""
+        t = np.concatenate([np.arange(goff[g], goff[g + 1]) for g in samples]).astype(np.float64)
+        return 0.1 * np.sin(t), -0.05 * np.cos(t)
+
+    def actor_update(H_bits, y, lengths, adv, samples, scale):
+        cu = np.concatenate([[0], np.cumsum(lengths)])
+        lp, _, lse = O.token_logprob_ref(H_bits, W, y)
+        d_old, d_ref = perturbation(samples)
+        res = O.policy_loss_ref(lp, lp + d_old, lp + d_ref, adv, cu, loss_scale=scale)
+        _, dW = O.policy_loss_backward_ref(H_bits, W, y, lse, res["dlogp"])
+        return res["loss"], dW
+
+    # this rank: its own rows and rewards only; the rewards of the others arrive by the all-gather
+    H, y, r_mine = dp.build_columns("cpu")
+    gathered = dp.gather_rewards(r_mine).numpy()
+    adv_all = O.grpo_advantage_ref(gathered, dp.gathered_group_id, dp.n_groups)
+    adv_mine = adv_all[rank * dp.n_mine:(rank + 1) * dp.n_mine]
+    loss_local, dW_local = actor_update(wl.bf16_bits(H), y.numpy(), dp.lengths[dp.mine], adv_mine, dp.mine, dp.loss_scale)
+    dW_sum = bench.allreduce_sum_(torch.from_numpy(dW_local.copy()), world).numpy()
+    loss_sum = bench.allreduce_sum_(torch.tensor([loss_local], dtype=torch.float64), world).item()
+    if rank == 0:
+        # the global batch on one process, in global index order
+        Hs = [wl.bf16_bits(wl.gen_hidden(w)) for w in dp.sources]
+        ys = [wl.gen_target(w).numpy() for w in dp.sources]
+        r_all = np.concatenate([wl.gen_reward(w).numpy() for w in dp.sources])
+        adv_global = O.grpo_advantage_ref(r_all, dp.group_id, dp.n_groups)
+        loss_g, dW_g = actor_update(np.concatenate(Hs), np.concatenate(ys), dp.lengths, adv_global,
+                                    np.arange(dp.N_global), 1.0)
+        rep = dp.report()
+        counts = np.bincount(dp.part, minlength=world)
+        ok = (np.array_equal(gathered, r_all[dp.gathered_order])
+              and np.allclose(adv_all, adv_global[dp.gathered_order], rtol=0, atol=1e-14)
+              and abs(loss_sum - loss_g) <= 1e-12 * max(1.0, abs(loss_g))
+              and np.allclose(dW_sum, dW_g, rtol=0, atol=1e-11 * np.abs(dW_g).max())
+              and counts.min() == counts.max() == w0.N
+              and rep["token_spread_balanced"] <= rep["token_spread_by_prompt_index"]
+              and sum(rep["tokens_per_rank"]) == int(dp.lengths.sum())
+              and len(set(dp.group_id[dp.mine])) > w0.n_prompts // 2)       # groups really are spread over ranks
+        with open(os.path.join(out_dir, "ok_balanced"), "w") as f:
+            f.write("1" if ok else "0")
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_two_rank_token_balanced_actor_update(tmp_path):
+    from paper_2507_01663_b200 import build as b
+    b.build()                                    # af_balance_partitions is a host call of the library
+    port = _free_port()
+    mp.start_processes(_balanced_worker, args=(2, port, str(tmp_path)), nprocs=2, join=True, start_method="spawn")
+    assert open(tmp_path / "ok_balanced").read() == "1"

@@ -70,6 +70,82 @@ def test_advantage_of_nearly_equal_rewards(ctx, G):
     assert np.abs(np_of(adv) - ref).max() <= ADV_TOL
 
 
+def groups_ref(r, gid, groups, eps=1e-6, ddof=0):
+    """The oracle on the given groups only (it visits every group in turn, which at 2^17 groups
+    would take hours): each group's members form a batch of one group."""
+    order = np.argsort(gid, kind="stable")
+    bounds = np.searchsorted(gid[order], np.arange(gid.max() + 2))
+    out = {}
+    for g in groups:
+        members = order[bounds[g]:bounds[g + 1]]
+        out[g] = (members, O.grpo_advantage_ref(r[members], np.zeros(len(members), np.int64), 1, eps, ddof))
+    return out
+
+
+@pytest.mark.parametrize("law", ["uniform", "bernoulli", "last_bits", "outliers"])
+def test_advantage_by_group_id_at_scale(ctx, law):
+    """2^20 responses in 2^17 shuffled groups of unequal size (some empty): O(N) work, checked
+    against the oracle on sampled groups, and the same bits on every run although the members of a
+    group meet in no fixed order."""
+    dev = device()
+    N, n_groups = 1 << 20, 1 << 17
+    # group sizes from 0 to a few dozen: ids drawn with a skew, then shuffled by construction
+    u = np_of(wl.uniform01(41, wl.S_MISC, 0, N))
+    gid = np.minimum((u ** 1.7 * n_groups).astype(np.int64), n_groups - 1)
+    if law == "uniform":
+        r = np_of(wl.uniform01(42, wl.S_REWARD, 0, N))
+    elif law == "bernoulli":
+        r = (np_of(wl.uniform01(42, wl.S_REWARD, 0, N)) < 0.3).astype(np.float32)
+    elif law == "last_bits":          # rewards that differ only in the last bits of an fp32
+        steps = np_of(wl.randint(42, wl.S_REWARD, 0, N, 40)).astype(np.float32)
+        r = (np.float32(0.3) + steps * np.spacing(np.float32(0.3))).astype(np.float32)
+    else:                             # a few huge rewards among tiny ones, both signs
+        big = np_of(wl.uniform01(43, wl.S_REWARD, 0, N)) < 0.02
+        r = np.where(big, 1.0e6, 1.0e-3 * np_of(wl.normal01(44, wl.S_REWARD, 0, N))).astype(np.float32)
+    counts = np.bincount(gid, minlength=n_groups)
+    assert counts.min() == 0 and counts.max() > 30
+    for ddof in (0, 1):
+        adv = torch.full((N,), 9.0, device=dev)
+        ctx.grpo_advantage(f32(r), i32(gid), n_groups, adv, 1e-6, ddof)
+        a = np_of(adv)
+        again = torch.full((N,), 9.0, device=dev)
+        ctx.grpo_advantage(f32(r), i32(gid), n_groups, again, 1e-6, ddof)
+        assert a.tobytes() == np_of(again).tobytes()
+        pick = sorted({int(np.argmax(counts)), int(np.argmax(counts == 1)), int(np.argmax(counts == 2)), 0, n_groups - 1}
+                      | set(np.random.default_rng(5).integers(0, n_groups, 1500).tolist()))
+        for g, (members, want) in groups_ref(r, gid, pick, 1e-6, ddof).items():
+            assert np.abs(a[members] - want).max(initial=0.0) <= ADV_TOL, (law, ddof, g)
+        assert np.isfinite(a).all()
+    assert ctx.check_device_errors() == 0
+
+
+def test_advantage_by_group_id_few_huge_groups_and_bad_ids(ctx):
+    from paper_2507_01663_b200 import binding as B
+    dev = device()
+    N = 1 << 18
+    r = np_of(wl.uniform01(45, wl.S_REWARD, 0, N))
+    gid = np_of(wl.randint(46, wl.S_MISC, 0, N, 3)).astype(np.int64)          # three groups of ~87 k members
+    adv = torch.full((N,), 9.0, device=dev)
+    ctx.grpo_advantage(f32(r), i32(gid), 3, adv)
+    ref = O.grpo_advantage_ref(r, gid, 3)
+    assert np.abs(np_of(adv) - ref).max() <= ADV_TOL
+    # one group holding everything, in one warp's worth of lanes each time
+    ctx.grpo_advantage(f32(r), i32(np.zeros(N)), 1, adv)
+    assert np.abs(np_of(adv) - O.grpo_advantage_ref(r, np.zeros(N, np.int64), 1)).max() <= ADV_TOL
+    assert ctx.check_device_errors() == 0
+    # ids outside [0, n_groups): NaN for those samples, the flag is raised, the rest is unaffected
+    bad = gid.copy()
+    bad[[5, 70000]] = [3, -1]
+    ctx.grpo_advantage(f32(r), i32(bad), 3, adv)
+    a = np_of(adv)
+    assert ctx.check_device_errors() & B.DEVERR_GROUP_ID
+    assert np.isnan(a[[5, 70000]]).all() and np.isnan(a).sum() == 2
+    keep = np.ones(N, bool)
+    keep[[5, 70000]] = False
+    ref_bad = O.grpo_advantage_ref(r[keep], gid[keep], 3)
+    assert np.abs(a[keep] - ref_bad).max() <= ADV_TOL
+
+
 def test_advantage_degenerate_groups(ctx):
     # equal rewards inside a group (also non-dyadic values) give exactly-zero-sized advantages
     r = f32([0.3] * 8 + [1.0] * 8 + [0.0] * 8 + [0.1, 0.7, 0.1, 0.7, 0.1, 0.7, 0.1, 0.7])
@@ -221,8 +297,9 @@ def test_kl_term_close_to_the_reference_policy(ctx):
             oref = O.policy_loss_ref(logp.numpy(), old.numpy(), ref.numpy(), A, cu, entropy=ent.numpy(), **kw)
             assert rel(res["kl_mean"], oref["kl_mean"]) <= LOSS_RTOL, (std, res["kl_mean"], oref["kl_mean"])
             compare_loss(res, g, oref, T)
-            # the KL part of dL/dlogp alone: advantages of zero leave nothing else
+            # the KL part of dL/dlogp alone (advantages of zero leave nothing else): exp(delta) - 1 carries
+            # the approximate exp2's 2.4e-7 absolute error, a few 1e-4 of its size at delta ~ 1e-3
             res0, g0 = run_loss(ctx, logp, old, ref, ent, np.zeros(24, np.float32), cu, **kw)
             o0 = O.policy_loss_ref(logp.numpy(), old.numpy(), ref.numpy(), np.zeros(24), cu, entropy=ent.numpy(), **kw)
-            assert np.abs(g0 - o0["dlogp"]).max() <= 1e-4 * np.abs(o0["dlogp"]).max()
+            assert np.abs(g0 - o0["dlogp"]).max() <= 1e-3 * np.abs(o0["dlogp"]).max()
     assert ctx.check_device_errors() == 0

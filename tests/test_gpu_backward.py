@@ -212,3 +212,47 @@ def test_shard_backward_argument_errors(ctx):
         ctx.policy_loss_backward_shard(H, torch.zeros(16, 8, dtype=torch.bfloat16, device=dev), y, z4, z4, -8,
                                        torch.zeros_like(H), torch.zeros(16, 8, device=dev))
     assert ctx.check_device_errors() == 0
+
+
+@pytest.mark.parametrize("fused", [False, True], ids=["backward", "update"])
+def test_dw_ready_event_marks_the_complete_gradient(ctx, fused):
+    """With a "d_W ready" event registered, a second stream that waits on it sees the finished d_W
+    (the data-parallel all-reduce starts there, beside the last block's dH product), and the
+    results are those of the default order bit for bit."""
+    from paper_2507_01663_b200 import binding as B
+    dev = device()
+    H, W, y, g, lse = inputs(1000, 264, 3000, seed=77)
+    Hd, Wd, yd, gd, lsed = H.to(dev), W.to(dev), y.to(dev), g.to(dev), f32(lse)
+    cu = torch.as_tensor(np.array([0, 400, 1000], dtype=np.int32), device=dev)
+    adv = f32([0.7, -1.1])
+    old = lsed * 0 - 8.0
+    ctx.set_tuning(0, 256, VARIANT)
+
+    def run():
+        dH = torch.full((1000, 264), 7.0, dtype=torch.bfloat16, device=dev)
+        dW = torch.full((3000, 264), 7.0, device=dev)
+        if fused:
+            lo = B.new_loss_out(dev)
+            logp, lse_o = torch.empty(1000, device=dev), torch.empty(1000, device=dev)
+            ctx.policy_update(Hd, Wd, yd, old, old, adv, cu, lo, logp, lse_o, dH, dW)
+        else:
+            ctx.policy_loss_backward(Hd, Wd, yd, lsed, gd, dH, dW)
+        return dH, dW
+
+    dH0, dW0 = run()
+    torch.cuda.synchronize()
+    ev = torch.cuda.Event()
+    ev.record()                                   # creates the underlying CUDA event
+    ctx.set_dw_ready_event(ev)
+    side = torch.cuda.Stream()
+    try:
+        dH1, dW1 = run()
+        with torch.cuda.stream(side):
+            side.wait_event(ev)
+            snap = dW1.clone()                    # reads d_W as soon as the event allows
+        torch.cuda.synchronize()
+    finally:
+        ctx.set_dw_ready_event(None)
+        ctx.set_tuning(0, 0)
+    assert ctx.check_device_errors() == 0
+    assert torch.equal(snap, dW1) and torch.equal(dW1, dW0) and torch.equal(dH1, dH0)

@@ -28,8 +28,9 @@ def ctx():
     c.close()
 
 
-def oracle_rows(H_rows, W_bits, y_rows, chunk=128):
-    """Oracle log-prob / entropy / lse of the given rows at the full vocabulary."""
+def oracle_rows(H_rows, W_bits, y_rows, chunk=512):
+    """Oracle log-prob / entropy / lse of the given rows at the full vocabulary (in chunks of rows:
+    every call of the oracle widens the whole weight matrix to fp64 first)."""
     outs = [O.token_logprob_ref(wl.bf16_bits(H_rows[s:s + chunk]), W_bits, y_rows[s:s + chunk])
             for s in range(0, H_rows.shape[0], chunk)]
     return [np.concatenate([o[k] for o in outs]) for k in range(3)]
@@ -225,7 +226,7 @@ def test_loss_stage_full_size(ctx):
     assert ctx.check_device_errors() == 0
 
 
-def dH_rows_ref(H_rows, W_bits, y_rows, lse_rows, g_rows, chunk=64):
+def dH_rows_ref(H_rows, W_bits, y_rows, lse_rows, g_rows, chunk=256):
     """Oracle dH of the given token rows (each row needs the whole vocabulary, nothing else)."""
     return np.concatenate([
         O.policy_loss_backward_ref(wl.bf16_bits(H_rows[s:s + chunk]), W_bits, y_rows[s:s + chunk],
