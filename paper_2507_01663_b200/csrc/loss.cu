@@ -4,7 +4,10 @@
 // A CTA owns a contiguous range of 2048-token chunks.  One thread feeds a ring of shared-memory
 // stages with bulk copies (TMA) of the chunk's logp / old / ref / entropy slices, up to three
 // chunks ahead, so the bytes in flight do not depend on how many threads are resident; each thread then
-// reads its 4 consecutive tokens from shared memory with one 128-bit load per column.  Warps run
+// reads two groups of 4 consecutive tokens (128 tokens apart, so that a warp's 128-bit accesses stay
+// contiguous) from shared memory with one 128-bit load per group and column.  At full bandwidth the
+// kernel runs at the SM's instruction-issue limit, so the work per thread that does not depend on
+// the token count (sequence lookup, barrier waits, loop control) is spread over 8 tokens.  Warps run
 // free of one another inside the chunk loop: a "full" mbarrier per stage announces the data, an
 // "empty" mbarrier per stage (one arrival per warp) tells the feeding thread when the stage can
 // be refilled -- there is no block-wide barrier per chunk.
@@ -25,9 +28,12 @@
 namespace af {
 namespace {
 
-constexpr int kThreads = 512;
+constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
-constexpr int kTokPerThread = 4;
+constexpr int kGroup = 4;                                 // consecutive tokens per 128-bit access
+constexpr int kGroups = 2;                                // such groups per thread, 128 tokens apart
+constexpr int kTokPerThread = kGroup * kGroups;
+constexpr int kWarpTokens = 32 * kTokPerThread;           // a warp owns 256 consecutive tokens of a chunk
 constexpr int kChunk = kThreads * kTokPerThread;          // tokens per chunk = per ring stage
 constexpr int kStages = 3;                                // ring depth: up to 3 chunks in flight
 constexpr int kColBytes = kChunk * 4;                     // one column slice of a stage
@@ -170,25 +176,33 @@ __global__ void __launch_bounds__(kThreads, 2) policy_loss_kernel(
     }
     if (!ok) continue;
 
-    const int t0 = c0 + threadIdx.x * kTokPerThread;
-    const int n = t0 < T ? ((T - t0) < kTokPerThread ? (T - t0) : kTokPerThread) : 0;
-    float lp[4], ol[4], rf[4], en[4] = {0.f, 0.f, 0.f, 0.f}, g[4];
-    if (n == 4 && vec_ok) {
-      const uint32_t src = ring + st * kStageBytes + threadIdx.x * 16;
-      const float4 a = lds128(src), b = lds128(src + kColBytes), r = lds128(src + 2 * kColBytes);
-      lp[0] = a.x; lp[1] = a.y; lp[2] = a.z; lp[3] = a.w;
-      ol[0] = b.x; ol[1] = b.y; ol[2] = b.z; ol[3] = b.w;
-      rf[0] = r.x; rf[1] = r.y; rf[2] = r.z; rf[3] = r.w;
-      if (entropy) {
-        const float4 e = lds128(src + 3 * kColBytes);
-        en[0] = e.x; en[1] = e.y; en[2] = e.z; en[3] = e.w;
+    // token of slot k of this thread: group k / 4 starts 128 tokens after the previous one
+    const int t0 = c0 + warp * kWarpTokens + lane * kGroup;
+    auto tok = [&](int k) { return t0 + (k / kGroup) * (32 * kGroup) + (k % kGroup); };
+    const int n = tok(kTokPerThread - 1) < T ? kTokPerThread : -1;      // -1: some slot lies past the end
+    float lp[kTokPerThread], ol[kTokPerThread], rf[kTokPerThread], en[kTokPerThread], g[kTokPerThread];
+#pragma unroll
+    for (int k = 0; k < kTokPerThread; ++k) en[k] = 0.f;
+    if (n == kTokPerThread && vec_ok) {
+#pragma unroll
+      for (int q = 0; q < kGroups; ++q) {
+        const uint32_t src = ring + st * kStageBytes + (uint32_t)(tok(q * kGroup) - c0) * 4u;
+        const float4 a = lds128(src), b = lds128(src + kColBytes), r = lds128(src + 2 * kColBytes);
+        lp[4 * q] = a.x; lp[4 * q + 1] = a.y; lp[4 * q + 2] = a.z; lp[4 * q + 3] = a.w;
+        ol[4 * q] = b.x; ol[4 * q + 1] = b.y; ol[4 * q + 2] = b.z; ol[4 * q + 3] = b.w;
+        rf[4 * q] = r.x; rf[4 * q + 1] = r.y; rf[4 * q + 2] = r.z; rf[4 * q + 3] = r.w;
+        if (entropy) {
+          const float4 e = lds128(src + 3 * kColBytes);
+          en[4 * q] = e.x; en[4 * q + 1] = e.y; en[4 * q + 2] = e.z; en[4 * q + 3] = e.w;
+        }
       }
     } else {
 #pragma unroll
       for (int k = 0; k < kTokPerThread; ++k) {
-        if (k < n) {
-          lp[k] = __ldg(logp + t0 + k); ol[k] = __ldg(old_logp + t0 + k); rf[k] = __ldg(ref_logp + t0 + k);
-          if (entropy) en[k] = __ldg(entropy + t0 + k);
+        const int t = tok(k);
+        if (t < T) {
+          lp[k] = __ldg(logp + t); ol[k] = __ldg(old_logp + t); rf[k] = __ldg(ref_logp + t);
+          if (entropy) en[k] = __ldg(entropy + t);
         }
       }
     }
@@ -196,7 +210,7 @@ __global__ void __launch_bounds__(kThreads, 2) policy_loss_kernel(
       __syncwarp();
       if (lane == 0) umma::mbar_arrive(empty_bar(st));
     }
-    if (n > 0) {
+    if (t0 < T) {
       int j, seq_beg, seq_end;
       if (staged) {
         // gallop forward from the previous position, then bisect: s_win[lo] <= t0 < s_win[hi]
@@ -222,8 +236,8 @@ __global__ void __launch_bounds__(kThreads, 2) policy_loss_kernel(
       float run_pg = 0.f, run_kl = 0.f;
 #pragma unroll
       for (int k = 0; k < kTokPerThread; ++k) {
-        if (k < n) {
-          const int t = t0 + k;
+        const int t = tok(k);                 // increasing in k: the thread walks forward through the sequences
+        if (t < T) {
           if (t >= seq_end) {  // run of sequence j ends: scale it once, move to the next sequence
             acc_pg += run_pg * inv_len; acc_kl += run_kl * inv_len;
             run_pg = 0.f; run_kl = 0.f;
@@ -245,11 +259,13 @@ __global__ void __launch_bounds__(kThreads, 2) policy_loss_kernel(
       }
       acc_pg += run_pg * inv_len; acc_kl += run_kl * inv_len;
       if (dlogp) {
-        if (n == 4 && vec_ok) {
-          *reinterpret_cast<float4*>(dlogp + t0) = make_float4(g[0], g[1], g[2], g[3]);
+        if (n == kTokPerThread && vec_ok) {
+#pragma unroll
+          for (int q = 0; q < kGroups; ++q)
+            *reinterpret_cast<float4*>(dlogp + tok(q * kGroup)) = make_float4(g[4 * q], g[4 * q + 1], g[4 * q + 2], g[4 * q + 3]);
         } else {
 #pragma unroll
-          for (int k = 0; k < kTokPerThread; ++k) if (k < n) dlogp[t0 + k] = g[k];
+          for (int k = 0; k < kTokPerThread; ++k) if (tok(k) < T) dlogp[tok(k)] = g[k];
         }
       }
     }
