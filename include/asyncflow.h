@@ -29,6 +29,8 @@
  *     memory and wait on an event of their own; they cannot be recorded.  Nothing is claimed for
  *     af_token_logprob_static.
  *   - Only compute capability 10.0 devices are accepted.  There is no CPU path.
+ *   - Every entry point that enqueues work opens an NVTX range named after itself (a no-op unless
+ *     a profiler that reads NVTX is attached).
  */
 #ifndef ASYNCFLOW_H_
 #define ASYNCFLOW_H_

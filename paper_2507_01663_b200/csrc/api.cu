@@ -7,6 +7,8 @@
 #include <new>
 #include <vector>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "common.cuh"
 
 namespace af {
@@ -22,6 +24,13 @@ af_status ws_grow(Buf& b, size_t bytes) {
 
 namespace {
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// A named range around every entry point that enqueues work, for timelines of a profiler that
+// understands NVTX (header-only: without such a tool attached the calls do nothing).
+struct NvtxRange {
+  explicit NvtxRange(const char* name) { nvtxRangePushA(name); }
+  ~NvtxRange() { nvtxRangePop(); }
+};
 
 struct DeviceGuard {
   int prev = -1;
@@ -127,6 +136,7 @@ af_status af_set_dw_ready_event(af_ctx* c, void* event) {
 }
 
 af_status af_check_device_errors(af_ctx* c, uint32_t* flags, void* stream) {
+  NvtxRange range("af_check_device_errors");
   if (!c) return AF_ERR_INVALID_ARG;
   DeviceGuard guard(c->device);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -149,6 +159,7 @@ static size_t pack_meta_bytes(int32_t B) {
 
 af_status af_reserve(af_ctx* c, int64_t max_T, int32_t max_B, int32_t d, int32_t V,
                      int32_t with_backward) {
+  NvtxRange range("af_reserve");
   if (!c || max_T < 0 || max_B < 0 || d < 1 || V < 1) return AF_ERR_INVALID_ARG;
   if (max_T >= ((int64_t)1 << 31)) return AF_ERR_SHAPE;
   DeviceGuard guard(c->device);
@@ -244,6 +255,7 @@ static af_status stage_sequence_table(af_ctx* c, const int64_t* tok_offset_host,
 
 af_status af_pack_microbatch(af_ctx* c, const af_store_view* store, const int32_t* idx_host,
                              int32_t B, const af_packed* out, int64_t* T_out, void* stream) {
+  NvtxRange range("af_pack_microbatch");
   if (!c || !store || !out || B < 0 || (B > 0 && !idx_host) || !store->tok_offset_host ||
       !out->cu_seqlens || store->n_samples < 0 || store->d < 1)
     return AF_ERR_INVALID_ARG;
@@ -271,13 +283,15 @@ af_status af_pack_microbatch(af_ctx* c, const af_store_view* store, const int32_
 af_status af_unpack_microbatch(af_ctx* c, const int64_t* tok_offset_host, int64_t n_samples, const int32_t* idx_host,
                                int32_t B, const af_write_cols* cols, const af_controller_view* table,
                                uint32_t column_bits, int64_t* T_out, void* stream) {
+  NvtxRange range("af_unpack_microbatch");
   if (!c || !tok_offset_host || n_samples < 0 || B < 0 || (B > 0 && !idx_host) || !cols || cols->n_cols < 0 ||
       cols->n_cols > AF_MAX_WRITE_COLS)
     return AF_ERR_INVALID_ARG;
   if (table && (table->n_samples != n_samples || (n_samples > 0 && !table->ready))) return AF_ERR_INVALID_ARG;
   // a sample may be listed once: two writers of one row would have no defined order
   try {
-    std::vector<int32_t> sorted(idx_host, idx_host + B);
+    std::vector<int32_t>& sorted = c->idx_scratch;     // the context's buffer: allocates only when it grows
+    sorted.assign(idx_host, idx_host + B);
     std::sort(sorted.begin(), sorted.end());
     if (std::adjacent_find(sorted.begin(), sorted.end()) != sorted.end()) return AF_ERR_INVALID_ARG;
   } catch (...) {   // no exception may cross the C boundary (the copy of the list could not be allocated)
@@ -309,6 +323,7 @@ af_status af_unpack_microbatch(af_ctx* c, const int64_t* tok_offset_host, int64_
 af_status af_token_logprob(af_ctx* c, const void* hidden, const void* W, const int32_t* target,
                            int64_t T, int32_t d, int32_t V, float* logp, float* entropy, float* lse,
                            void* stream) {
+  NvtxRange range("af_token_logprob");
   if (!c || T < 0 || d < 1 || V < 1) return AF_ERR_INVALID_ARG;
   if (T == 0) return AF_OK;
   if (!hidden || !W || !target || !logp) return AF_ERR_INVALID_ARG;
@@ -322,6 +337,7 @@ af_status af_token_logprob(af_ctx* c, const void* hidden, const void* W, const i
 af_status af_token_logprob_shard(af_ctx* c, const void* hidden, const void* W_shard, const int32_t* target,
                                  int64_t T, int32_t d, int32_t V_shard, int32_t v_offset, float* partial_out,
                                  void* stream) {
+  NvtxRange range("af_token_logprob_shard");
   if (!c || T < 0 || d < 1 || V_shard < 1 || v_offset < 0) return AF_ERR_INVALID_ARG;
   if (T == 0) return AF_OK;
   if (!hidden || !W_shard || !target || !partial_out) return AF_ERR_INVALID_ARG;
@@ -334,6 +350,7 @@ af_status af_token_logprob_shard(af_ctx* c, const void* hidden, const void* W_sh
 
 af_status af_merge_logprob_shards(af_ctx* c, const float* partials, const int32_t* target, int32_t R, int64_t T,
                                   int32_t V_total, float* logp, float* entropy, float* lse, void* stream) {
+  NvtxRange range("af_merge_logprob_shards");
   if (!c || T < 0 || R < 1 || V_total < 1) return AF_ERR_INVALID_ARG;
   if (T == 0) return AF_OK;
   if (!partials || !target || !logp) return AF_ERR_INVALID_ARG;
@@ -346,6 +363,7 @@ af_status af_merge_logprob_shards(af_ctx* c, const float* partials, const int32_
 
 af_status af_grpo_advantage(af_ctx* c, const float* reward, const int32_t* group_id, int64_t N,
                             int32_t n_groups, float eps_adv, int32_t ddof, float* adv, void* stream) {
+  NvtxRange range("af_grpo_advantage");
   if (!c || N < 0 || n_groups < 0 || (ddof != 0 && ddof != 1) || !(eps_adv > 0.f)) return AF_ERR_INVALID_ARG;
   if (N == 0) return AF_OK;
   if (!reward || !adv || n_groups < 1) return AF_ERR_INVALID_ARG;
@@ -365,6 +383,7 @@ af_status af_policy_loss(af_ctx* c, const float* logp, const float* old_logp, co
                          const float* entropy, const float* adv_seq, const int32_t* cu_seqlens,
                          int32_t B, int64_t T, const af_loss_params* params, af_loss_out* out,
                          float* dlogp, void* stream) {
+  NvtxRange range("af_policy_loss");
   if (!c || !params || !out || !cu_seqlens || B < 0 || T < 0) return AF_ERR_INVALID_ARG;
   if (T > 0 && (!logp || !old_logp || !ref_logp || !adv_seq || B < 1)) return AF_ERR_INVALID_ARG;
   if (params->agg_mode != 0 && params->agg_mode != 1) return AF_ERR_INVALID_ARG;
@@ -378,6 +397,7 @@ af_status af_policy_loss(af_ctx* c, const float* logp, const float* old_logp, co
 af_status af_policy_loss_backward(af_ctx* c, const void* hidden, const void* W, const int32_t* target,
                                   const float* lse, const float* dlogp, int64_t T, int32_t d, int32_t V,
                                   void* d_hidden, float* d_W, int32_t accumulate_dW, void* stream) {
+  NvtxRange range("af_policy_loss_backward");
   if (!c || T < 0 || d < 1 || V < 1) return AF_ERR_INVALID_ARG;
   if (!hidden || !W || !target || !lse || !dlogp || !d_hidden || !d_W) {
     if (T > 0 || !d_W) return AF_ERR_INVALID_ARG;
@@ -394,6 +414,7 @@ af_status af_policy_loss_backward_shard(af_ctx* c, const void* hidden, const voi
                                         const float* lse, const float* dlogp, int64_t T, int32_t d, int32_t V_shard,
                                         int32_t v_offset, void* d_hidden_partial, float* d_W_shard,
                                         int32_t accumulate_dW, void* stream) {
+  NvtxRange range("af_policy_loss_backward_shard");
   if (!c || T < 0 || d < 1 || V_shard < 1 || v_offset < 0) return AF_ERR_INVALID_ARG;
   if (!hidden || !W_shard || !target || !lse || !dlogp || !d_hidden_partial || !d_W_shard) {
     if (T > 0 || !d_W_shard) return AF_ERR_INVALID_ARG;
@@ -416,6 +437,7 @@ af_status af_policy_update(af_ctx* c, const void* hidden, const void* W, const i
                            const int32_t* cu_seqlens, int32_t B, int64_t T, int32_t d, int32_t V,
                            const af_loss_params* params, af_loss_out* out, float* logp, float* entropy, float* lse,
                            float* dlogp, void* d_hidden, float* d_W, int32_t accumulate_dW, void* stream) {
+  NvtxRange range("af_policy_update");
   if (!c || !params || !out || !cu_seqlens || B < 0 || T < 0 || d < 1 || V < 1 || !d_W) return AF_ERR_INVALID_ARG;
   if (T > 0 && (!hidden || !W || !target || !old_logp || !ref_logp || !adv_seq || !logp || !lse || !d_hidden || B < 1))
     return AF_ERR_INVALID_ARG;
@@ -431,6 +453,7 @@ af_status af_policy_update(af_ctx* c, const void* hidden, const void* W, const i
 
 af_status af_controller_put(af_ctx* c, const af_controller_view* table, const int32_t* idx, int64_t n,
                             uint32_t column_bits, void* stream) {
+  NvtxRange range("af_controller_put");
   if (!c || !table_ok(table) || n < 0 || (n > 0 && !idx)) return AF_ERR_INVALID_ARG;
   if (table->n_samples >= ((int64_t)1 << 31)) return AF_ERR_SHAPE;
   DeviceGuard guard(c->device);
@@ -441,6 +464,7 @@ af_status af_controller_put(af_ctx* c, const af_controller_view* table, const in
 af_status af_controller_get(af_ctx* c, const af_controller_view* table, uint32_t column_mask, uint32_t task_bit,
                             int32_t max_samples, int64_t token_budget, int32_t* out_idx, af_get_result* out,
                             void* stream) {
+  NvtxRange range("af_controller_get");
   if (!c || !table_ok(table) || !out || max_samples < 0 || (max_samples > 0 && !out_idx)) return AF_ERR_INVALID_ARG;
   if (task_bit == 0 || (task_bit & (task_bit - 1)) != 0) return AF_ERR_INVALID_ARG;
   if (token_budget > 0 && !table->length && table->n_samples > 0) return AF_ERR_INVALID_ARG;
@@ -453,6 +477,7 @@ af_status af_controller_get(af_ctx* c, const af_controller_view* table, uint32_t
 
 af_status af_controller_clear(af_ctx* c, const af_controller_view* table, uint32_t column_bits, uint32_t task_bits,
                               void* stream) {
+  NvtxRange range("af_controller_clear");
   if (!c || !table_ok(table)) return AF_ERR_INVALID_ARG;
   DeviceGuard guard(c->device);
   return launch_controller_clear(*table, column_bits, task_bits, c->sm_count,

@@ -8,6 +8,7 @@
 #include <stdint.h>
 
 #include <atomic>
+#include <vector>
 
 #include "../../include/asyncflow.h"
 
@@ -74,6 +75,7 @@ struct af_ctx {
   cudaEvent_t dw_ready = nullptr;  // caller's event recorded once d_W is complete (af_set_dw_ready_event)
 
   af::TmapCache tmaps;      // tensor maps of the GEMM operands seen so far
+  std::vector<int32_t> idx_scratch;  // host copy of an index list (duplicate check of the write-back); grows, never shrinks
 
   // workspace (device)
   af::Buf partial;    // [splits, T] float4 online-softmax partials
