@@ -197,6 +197,41 @@ def test_streaming_store_full_size(ctx):
         assert r["n_tokens"] == int(w.lengths[m].sum()) and np.isfinite(r["loss"]) and 0 <= r["clip_frac"] <= 1
 
 
+def test_closed_streaming_loop_full_size():
+    """cfg5 through the benchmark's two-task loop (controller get -> pack -> log-prob -> write-back with
+    status bits; get on those bits -> pack -> log-prob -> loss; weight swap at an iteration boundary):
+    the column actor inference wrote back against the oracle on sampled store rows, every sample
+    served once per task, every loss record finite with nothing clipped."""
+    import bench
+    w = wl.make_workload("cfg5")
+    dev = device()
+    job = bench.ScoringJob(w, dev)
+    try:
+        job.make_closed_loop()
+        scored = job.step_closed_loop(refresh_weights=True)
+        torch.cuda.synchronize()
+        assert scored == 2 * w.total_tokens and job.ctx.check_device_errors() == 0 and job.w_swaps == 1
+        col = job.cl_old_col
+        assert bool(torch.isfinite(col).all())
+        rows = sample_rows(w.tok_offset, w.total_tokens, N_ROWS_MB, seed=11)
+        rt = torch.as_tensor(rows, device=dev)
+        o_logp, _, _ = oracle_rows(job.store["hidden"][rt].cpu(), wl.bf16_bits(job.W), np_of(job.store["target"][rt]))
+        assert np.abs(np_of(col[rt]) - o_logp).max() <= LOGP_TOL
+        both = job.COL_RESPONSE | job.COL_OLD_LOGP
+        assert bool((job.cl_tab["ready"] == both).all())
+        assert bool((job.cl_tab["consumed"] == (job.TASK_INFER | job.TASK_UPDATE)).all())
+        for task in (job.TASK_INFER, job.TASK_UPDATE):
+            seen = np.concatenate([mb for t, mb in job.cl_history if t == task])
+            assert np.array_equal(np.sort(seen), np.arange(w.N))
+        for _, mb in job.cl_history:
+            assert int(w.lengths[mb].sum()) <= w.token_budget or len(mb) == 1
+        records = [job.B.read_loss_out(lo) for lo in job.cl_loss_outs[:job.cl_loss_count]]
+        assert sum(r["n_tokens"] for r in records) == w.total_tokens
+        assert all(np.isfinite(r["loss"]) and r["clip_frac"] == 0.0 for r in records)
+    finally:
+        job.ctx.close()
+
+
 def test_loss_stage_full_size(ctx):
     """The loss kernel alone at 1.1 M tokens against the oracle, on generator-made inputs."""
     from paper_2507_01663_b200 import binding as B
