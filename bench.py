@@ -117,6 +117,16 @@ def head_name(w) -> str:
     return {(3584, 152064): "Qwen2.5-7B-shaped", (5120, 152064): "Qwen2.5-32B-shaped"}.get((w.d, w.V), "synthetic")
 
 
+# Set by --dp-single-rank: run the data-parallel exchanges (reward all-gather, overlapped dW
+# all-reduce) through a process group of ONE rank, so that their code path -- NCCL calls, streams,
+# events -- runs on a single GPU.
+EXCHANGE_WITH_ONE_RANK = False
+
+
+def exchanging(world: int) -> bool:
+    return world > 1 or EXCHANGE_WITH_ONE_RANK
+
+
 def dist_env():
     return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
 
@@ -192,7 +202,7 @@ class DataParallelShare:
 
     def gather_rewards(self, mine: torch.Tensor) -> torch.Tensor:
         """All ranks' reward slices back to back (rank-major): 4 bytes per response cross the links."""
-        if self.world == 1:
+        if not exchanging(self.world):
             return mine
         import torch.distributed as dist
         out = torch.empty(self.N_global, dtype=mine.dtype, device=mine.device)
@@ -224,7 +234,7 @@ def allreduce_sum_(t: torch.Tensor, world: int) -> torch.Tensor:
     """Actor update under data parallelism: every rank scores its own prompts with
     loss_scale = B_rank / B_global, so the weight gradients of the ranks ADD UP to the gradient of
     the global batch; the one exchange of the path is this sum (NCCL on GPUs, gloo in CPU tests)."""
-    if world > 1:
+    if exchanging(world):
         import torch.distributed as dist
         dist.all_reduce(t, op=dist.ReduceOp.SUM)
     return t
@@ -309,7 +319,7 @@ class ScoringJob:
         if w.backward:
             self.d_hidden = torch.empty(cap_T, w.d, dtype=torch.bfloat16, device=device)
             self.d_W = torch.empty(w.V, w.d, device=device)
-            if world > 1 and not vocab_parallel:
+            if exchanging(world) and not vocab_parallel:
                 # the gradient all-reduce runs on its own stream, started by the event the backward
                 # records as soon as d_W is complete (its last block runs the dW product first)
                 self.overlap_dw = True
@@ -339,7 +349,7 @@ class ScoringJob:
         """The one exchange of a data-parallel actor update.  With the overlap set up, the all-reduce
         waits for the backward's "d_W complete" event on the communication stream and runs beside
         the last block's dH product; the compute stream waits for it only before d_W is next written."""
-        if self.world == 1:
+        if not exchanging(self.world):
             return
         if not self.overlap_dw:
             allreduce_sum_(self.d_W, self.world)
@@ -1018,16 +1028,25 @@ def run_ours(args):
         raise RuntimeError("bench.py needs a CUDA device (there is no CPU path)")
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
+    global EXCHANGE_WITH_ONE_RANK
+    EXCHANGE_WITH_ONE_RANK = bool(args.dp_single_rank) and world == 1
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
+    elif EXCHANGE_WITH_ONE_RANK:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        with socket.socket() as sk:
+            sk.bind(("127.0.0.1", 0))
+            os.environ.setdefault("MASTER_PORT", str(sk.getsockname()[1]))
+        dist.init_process_group("nccl", rank=0, world_size=1, device_id=dev)
     variant = {"default": 0, "single": 1, "pair": 2}[args.gemm]
     base = wl.make_workload(args.workload)
     # data parallel: the global batch (one draw of the workload per rank) is dealt to the ranks by
     # token count; a streaming store stays whole on its rank; vocabulary parallel: one batch, the
     # head split by rows
     dp = None
-    if world > 1 and not args.vocab_parallel and not base.token_budget:
+    if exchanging(world) and not args.vocab_parallel and not base.token_budget:
         dp = DataParallelShare(args.workload, world, rank, balance=not args.no_balance)
     w = rank_workload(args.workload, 0 if args.vocab_parallel else rank)
     job = ScoringJob(w, dev, variant, world, args.v_splits, args.vocab_parallel, rank, args.bwd_token_block, dp)
@@ -1184,7 +1203,7 @@ def run_ours(args):
             "cfg5_pack_frac_of_hbm": fig("cfg5", "pack_frac_of_hbm")})
     if rank == 0:
         print(json.dumps(line), flush=True)
-    if world > 1:
+    if exchanging(world):
         import torch.distributed as dist
         dist.destroy_process_group()
 
@@ -1267,6 +1286,10 @@ def main():
     ap.add_argument("--no-balance", action="store_true",
                     help="data parallel: deal the global batch to the ranks by prompt index instead of by token "
                          "count (af_balance_partitions)")
+    ap.add_argument("--dp-single-rank", action="store_true",
+                    help="one GPU: run the data-parallel code path (split, reward all-gather, advantages by group "
+                         "id, dW all-reduce started by the backward's event on a second stream) through a process "
+                         "group of one rank")
     ap.add_argument("--no-configs", action="store_true",
                     help="skip the short legs of the other four workloads that follow the default cfg2 run")
     ap.add_argument("--v-splits", type=int, default=0,

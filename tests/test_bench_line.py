@@ -68,3 +68,19 @@ def test_gpu_arm_line():
     assert set(clocks) >= {"sm_mhz", "sm_max_mhz", "reasons"}
     assert set(line["hbm_kernels"]) >= {"pack_microbatch", "policy_loss", "grpo_advantage", "controller_get"}
     assert line["step_ms_rank0"]["min"] <= line["step_ms_rank0"]["median"] <= line["step_ms_rank0"]["max"]
+
+
+@pytest.mark.gpu
+def test_data_parallel_code_path_with_a_process_group_of_one_rank():
+    """The exchanges of the data-parallel step -- NCCL all-gather of rewards, advantages by group id, the
+    dW all-reduce started by the backward's "d_W ready" event on a second stream -- run on one GPU
+    through a process group of one rank (where they change no value)."""
+    import math
+    line = run_bench("--workload", "cfg4_mini", "--dp-single-rank", "--steps", "3", "--warmup", "3", "--hbm-log2", "20",
+                     "--cpu-sample", "64")
+    check_base(line)
+    dp = line["data_parallel"]
+    assert dp["ranks"] == 1 and dp["responses_per_rank"] == 32 and sum(dp["tokens_per_rank"]) == 1024
+    assert line["config"]["parallelism"].startswith("dp1")
+    assert math.isfinite(line["loss"]) and math.isfinite(line["fused_update"]["loss"])
+    assert line["backward"]["ms"] > 0
