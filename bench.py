@@ -976,7 +976,7 @@ def streaming_legs(job, args, world: int, tokens: int, steps: int, warmup: int) 
 def side_leg(name: str, args, dev, peaks, steps: int = 5, warmup: int = 3) -> dict:
     """A short timed leg of another workload on one GPU (its own buffers, its own clock record)."""
     w = wl.make_workload(name)
-    job = ScoringJob(w, dev, {"default": 0, "single": 1, "pair": 2}[args.gemm])
+    job = ScoringJob(w, dev, {"default": 0, "single": 1, "pair": 2, "die": 3}[args.gemm])
     out = {"workload": describe(w, job, name), "steps": steps, "warmup": warmup}
     for _ in range(warmup):
         job.step()
@@ -1040,7 +1040,7 @@ def run_ours(args):
             sk.bind(("127.0.0.1", 0))
             os.environ.setdefault("MASTER_PORT", str(sk.getsockname()[1]))
         dist.init_process_group("nccl", rank=0, world_size=1, device_id=dev)
-    variant = {"default": 0, "single": 1, "pair": 2}[args.gemm]
+    variant = {"default": 0, "single": 1, "pair": 2, "die": 3}[args.gemm]
     base = wl.make_workload(args.workload)
     # data parallel: the global batch (one draw of the workload per rank) is dealt to the ranks by
     # token count; a streaming store stays whole on its rank; vocabulary parallel: one batch, the
@@ -1304,7 +1304,7 @@ def main():
                          "weight refresh, and as the two-task closed loop")
     ap.add_argument("--weight-refresh", action="store_true", help="same as --live-controller")
     ap.add_argument("--closed-loop", action="store_true", help="same as --live-controller")
-    ap.add_argument("--gemm", default="default", choices=["default", "single", "pair"],
+    ap.add_argument("--gemm", default="default", choices=["default", "single", "pair", "die"],
                     help="main loop of the tensor-core GEMMs (af_set_tuning gemm_variant): CTA pairs (the default) "
                          "or one CTA per tile")
     args = ap.parse_args()

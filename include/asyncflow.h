@@ -82,11 +82,18 @@ int64_t af_workspace_bytes(const af_ctx* ctx);
 /* Tuning knobs of the fused LM-head kernels (0 keeps the default): `v_splits` = number of
  * vocabulary ranges one token tile is split into across CTAs; `bwd_token_block` = tokens per
  * backward block, a multiple of 128 (scratch is proportional to it); `gemm_variant` selects the
- * main loop of every tensor-core GEMM of the context: 2 (and 0, the default) = CTA pairs -- two
- * SMs share one 256 x 256 tile, each staging half of the weight tile, and the pairs pace one
- * another so that a weight tile fetched once serves them all; 1 = one CTA per 128 x 256 tile.
+ * main loop of every tensor-core GEMM of the context: 0 (the default) and 3 = CTA pairs -- two
+ * SMs share one 256 x 256 tile, each staging half of the weight tile, the pairs pace one another
+ * so that a weight tile fetched once serves them all, and the row tiles are dealt to the pairs by
+ * the die they run on (see af_die_split), so that a hidden-state panel occupies one half of L2
+ * only; 2 = CTA pairs dealt without regard to dies; 1 = one CTA per 128 x 256 tile.
  * Results agree within the stated tolerances either way. */
 af_status af_set_tuning(af_ctx* ctx, int32_t v_splits, int32_t bwd_token_block, int32_t gemm_variant);
+
+/* How af_create found the SMs split over the two dies of the part (each die has its own half of
+ * L2): the number of SMs that share a die with the first SM probed, and the rest.  Both 0 when the
+ * latency measurement behind it was not clear-cut (then work is dealt without regard to dies). */
+af_status af_die_split(const af_ctx* ctx, int32_t* die0_sms, int32_t* die1_sms);
 
 /* Data-parallel actor update (Section 4.1: the training batch is streamed to the DP groups of the
  * actor-update task; each computes the gradient of its share).  The one exchange of the path is

@@ -27,7 +27,7 @@ EXPORTS = ["af_create", "af_destroy", "af_status_string", "af_reserve", "af_work
            "af_set_tuning", "af_check_device_errors", "af_pack_microbatch", "af_token_logprob",
            "af_grpo_advantage", "af_policy_loss", "af_policy_loss_backward", "af_token_logprob_static",
            "af_controller_put", "af_controller_get", "af_controller_clear", "af_balance_partitions",
-           "af_token_logprob_shard", "af_merge_logprob_shards", "af_policy_update", "af_unpack_microbatch", "af_policy_loss_backward_shard", "af_set_dw_ready_event"]
+           "af_token_logprob_shard", "af_merge_logprob_shards", "af_policy_update", "af_unpack_microbatch", "af_policy_loss_backward_shard", "af_set_dw_ready_event", "af_die_split"]
 MAX_WRITE_COLS = 4
 
 
@@ -101,6 +101,7 @@ def load_library() -> C.CDLL:
     lib.af_set_tuning.argtypes = [vp, i32, i32, i32]
     lib.af_check_device_errors.argtypes = [vp, C.POINTER(C.c_uint32), vp]
     lib.af_set_dw_ready_event.argtypes = [vp, vp]
+    lib.af_die_split.argtypes = [vp, C.POINTER(i32), C.POINTER(i32)]
     lib.af_pack_microbatch.argtypes = [vp, C.POINTER(StoreView), vp, i32, C.POINTER(Packed),
                                        C.POINTER(i64), vp]
     lib.af_token_logprob.argtypes = [vp, vp, vp, vp, i64, i32, i32, vp, vp, vp, vp]
@@ -176,7 +177,8 @@ class Context:
         return int(self.lib.af_workspace_bytes(self.handle))
 
     def set_tuning(self, v_splits: int = 0, bwd_token_block: int = 0, gemm_variant: int = 0):
-        """gemm_variant: 0 = default (CTA pairs), 1 = one CTA per tile, 2 = CTA pairs."""
+        """gemm_variant: 0 = default (CTA pairs, row tiles dealt by die), 1 = one CTA per tile, 2 = CTA
+        pairs dealt without regard to dies, 3 = same as 0."""
         _check(self.lib.af_set_tuning(self.handle, v_splits, bwd_token_block, gemm_variant), "af_set_tuning")
 
     def set_dw_ready_event(self, event: Optional[torch.cuda.Event]):
@@ -184,6 +186,12 @@ class Context:
         complete (None clears it).  The event must have been recorded once, so that it exists."""
         _check(self.lib.af_set_dw_ready_event(self.handle, None if event is None else C.c_void_p(event.cuda_event)),
                "af_set_dw_ready_event")
+
+    def die_split(self):
+        """(SMs on the first die, SMs on the other) as measured at creation; (0, 0) if unclear."""
+        a, b = C.c_int32(0), C.c_int32(0)
+        _check(self.lib.af_die_split(self.handle, C.byref(a), C.byref(b)), "af_die_split")
+        return int(a.value), int(b.value)
 
     def check_device_errors(self, stream=None) -> int:
         """Synchronise the stream; return the device error bits (0 = none) and clear them."""

@@ -90,8 +90,11 @@ af_status af_create(af_ctx** out, int device) {
     return AF_ERR_CUDA;
   }
   c->encode = reinterpret_cast<EncodeTiledFn>(fn);
-  if (cudaMalloc(&c->d_err, 256) != cudaSuccess) { c->d_err = nullptr; cudaGetLastError(); af_destroy(c); return AF_ERR_WORKSPACE; }
-  if (cudaMemset(c->d_err, 0, 256) != cudaSuccess) { af_destroy(c); return AF_ERR_CUDA; }
+  if (cudaMalloc(&c->d_err, kDeviceBlockBytes) != cudaSuccess) { c->d_err = nullptr; cudaGetLastError(); af_destroy(c); return AF_ERR_WORKSPACE; }
+  if (cudaMemset(c->d_err, 0, kDeviceBlockBytes) != cudaSuccess) { af_destroy(c); return AF_ERR_CUDA; }
+  // which SMs share a die (for die-aware dealing of GEMM row tiles); 0 when the measurement is unclear
+  if (!measure_die_map(c->sm_count, reinterpret_cast<unsigned char*>(c->d_err) + kDieTableByte, &c->die0_sms)) c->die0_sms = 0;
+  c->die_aware = 1;
   af_status st = ws_grow(c->loss_ws, loss_workspace_bytes(c->sm_count));
   if (st == AF_OK && cudaMemset(c->loss_ws.p, 0, c->loss_ws.cap) != cudaSuccess) st = AF_ERR_CUDA;
   if (st == AF_OK) st = ws_grow(c->ctrl_ws, controller_workspace_bytes(c->sm_count));
@@ -120,12 +123,20 @@ int64_t af_workspace_bytes(const af_ctx* c) {
   return (int64_t)(c->partial.cap + c->loss_ws.cap + c->pack_meta.cap + c->dz.cap + c->ctrl_ws.cap + c->zlog.cap + c->adv_ws.cap);
 }
 
+af_status af_die_split(const af_ctx* c, int32_t* die0_sms, int32_t* die1_sms) {
+  if (!c || !die0_sms || !die1_sms) return AF_ERR_INVALID_ARG;
+  *die0_sms = c->die0_sms;
+  *die1_sms = c->die0_sms > 0 ? c->sm_count - c->die0_sms : 0;
+  return AF_OK;
+}
+
 af_status af_set_tuning(af_ctx* c, int32_t v_splits, int32_t bwd_token_block, int32_t gemm_variant) {
-  if (!c || v_splits < 0 || bwd_token_block < 0 || gemm_variant < 0 || gemm_variant > 2) return AF_ERR_INVALID_ARG;
+  if (!c || v_splits < 0 || bwd_token_block < 0 || gemm_variant < 0 || gemm_variant > 3) return AF_ERR_INVALID_ARG;
   if (bwd_token_block % 128 != 0) return AF_ERR_SHAPE;
   c->v_splits = v_splits;
   c->bwd_token_block = bwd_token_block;
   c->gemm_pair = gemm_variant == 1 ? 0 : (c->sm_count >= 2 ? 1 : 0);
+  c->die_aware = gemm_variant == 2 ? 0 : 1;      // 0 and 3: by die where the die map was measured; 2: plain dealing
   return AF_OK;
 }
 
@@ -165,7 +176,8 @@ af_status af_reserve(af_ctx* c, int64_t max_T, int32_t max_B, int32_t d, int32_t
   DeviceGuard guard(c->device);
   af_status st = AF_OK;
   if (max_T > 0) {
-    const int S = logprob_pick_splits(max_T, d, V, c->sm_count, c->gemm_pair != 0, c->v_splits);
+    const int S = logprob_pick_splits(max_T, d, V, c->sm_count, c->gemm_pair != 0, c->v_splits,
+                                      c->gemm_pair && c->die_aware ? c->die0_sms / 2 : 0);
     // smaller batches may pick up to 8 ranges whatever their size, and more than 8 only while
     // there are at most 8 units per worker
     size_t need = (size_t)(S > 8 ? S : 8) * (size_t)max_T;

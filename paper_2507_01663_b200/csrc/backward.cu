@@ -184,7 +184,7 @@ af_status launch_backward_products(af_ctx* ctx, const void* hidden_blk, const vo
   auto dW_product = [&]() {
     StoreF32TransposedEpi::Params p3{d_W, d, d, V, accumulate_dW ? 1 : 0};
     return run_gemm<StoreF32TransposedEpi, true, true>(
-        env, Hblk, dZop, logprob_pick_splits((int64_t)d, (int32_t)tc, V, ctx->sm_count, env.pair, 0), p3, s);
+        env, Hblk, dZop, logprob_pick_splits((int64_t)d, (int32_t)tc, V, ctx->sm_count, env.pair, 0, 0), p3, s);
   };
   // With a "d_W ready" event registered, the last block runs its dW product first and records the
   // event behind it: d_W is complete from there on, and whoever waits on the event (a gradient
@@ -234,7 +234,7 @@ af_status launch_backward(af_ctx* ctx, const void* hidden, const void* W, const 
     // 1. dZ block:  Z = H_blk W^T, both K-major
     DzEpi::Params p1{target + t0, lse + t0, dlogp + t0, dz, (int)tc, V, v_offset};
     st = run_gemm<DzEpi, false, false>(env, Hblk, Wop,
-                                       logprob_pick_splits((int64_t)tc, d, V, ctx->sm_count, env.pair, ctx->v_splits), p1, s);
+                                       logprob_pick_splits((int64_t)tc, d, V, ctx->sm_count, env.pair, ctx->v_splits, env.die0_pairs), p1, s);
     if (st != AF_OK) return st;
     st = launch_backward_products(ctx, H + t0 * d, W, dz, (int64_t)tc, d, V,
                                   static_cast<__nv_bfloat16*>(d_hidden) + t0 * d, d_W,

@@ -15,7 +15,10 @@
 namespace af {
 
 constexpr int kPackRing = 8;  // pinned staging slots for af_pack_microbatch metadata
-constexpr int kTileClockWord = 16;  // word of the context's 256-byte device block used as the GEMM tile clock
+constexpr int kDeviceBlockBytes = 1024;  // the context's small device block: error word, tile clock, rank slots
+constexpr int kTileClockWord = 16;  // word of that block used as the GEMM tile clock
+constexpr int kDieCounterWord = 17;  // two words behind the clock: the per-die rank counters of a GEMM launch
+constexpr int kDieTableByte = 512;   // 256 bytes of that block: die (0 / 1) of every SM id, measured at af_create
 
 struct Buf {
   void* p = nullptr;
@@ -66,12 +69,14 @@ struct af_ctx {
   int device = 0;
   int sm_count = 0;
   af::EncodeTiledFn encode = nullptr;
-  unsigned int* d_err = nullptr;  // 256-byte device block: word 0 = sticky error word, word kTileClockWord = tile clock
+  unsigned int* d_err = nullptr;  // kDeviceBlockBytes device block: word 0 = sticky error word, then clock and rank slots
 
   // tuning
   int v_splits = 0;         // 0 = automatic
   int bwd_token_block = 0;  // 0 = default
   int gemm_pair = 1;        // 1 = CTA-pair GEMM variant (the default), 0 = one CTA per tile
+  int die_aware = 0;        // pair variant: deal row tiles to pairs by the die they run on
+  int die0_sms = 0;         // SMs on the die of the first SM probed (0: the measurement was not clear-cut; no die-aware dealing)
   cudaEvent_t dw_ready = nullptr;  // caller's event recorded once d_W is complete (af_set_dw_ready_event)
 
   af::TmapCache tmaps;      // tensor maps of the GEMM operands seen so far
@@ -97,6 +102,9 @@ struct af_ctx {
 namespace af {
 
 af_status ws_grow(Buf& b, size_t bytes);
+
+// Measures which SMs share a die (device table of 256 bytes indexed by SM id); false if unclear.
+bool measure_die_map(int sm_count, unsigned char* d_table, int* die0_sms);
 
 // ---- launchers (each returns the cudaGetLastError of its launches) --------------------------
 struct PackSeqTable {     // device views into ctx->pack_meta for one call
@@ -139,7 +147,7 @@ cudaError_t launch_controller_get(const af_controller_view& v, uint32_t mask, ui
                                   int64_t token_budget, int32_t* out_idx, af_get_result* out, void* ws,
                                   int sm_count, cudaStream_t s);
 
-int logprob_pick_splits(int64_t T, int32_t d, int32_t V, int sm_count, bool pair, int requested);
+int logprob_pick_splits(int64_t T, int32_t d, int32_t V, int sm_count, bool pair, int requested, int die0_pairs);
 af_status launch_token_logprob(af_ctx* ctx, const void* hidden, const void* W,
                                const int32_t* target, int64_t T, int32_t d, int32_t V,
                                float* logp, float* entropy, float* lse, cudaStream_t s);

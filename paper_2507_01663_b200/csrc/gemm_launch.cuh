@@ -22,7 +22,27 @@ struct GemmEnv {
   bool pair;             // CTA-pair variant (cta_group::2)
   unsigned int* tile_clock;  // device word the pair variant paces itself with (zeroed per launch), or null
   TmapCache* cache;          // tensor maps encoded earlier (a context's), or null
+  const unsigned char* die_of_sm;  // measured die of every SM id, or null
+  int die0_pairs;            // > 0: deal row tiles to pairs by die; CTA pairs the first die hosts
 };
+
+// Die-aware dealing of a pair GEMM's units (see umma::PairWork): can the first rows0 row tiles go to
+// the n0 pairs of one die and the rest to the others without any pair needing more rounds of units
+// than plain dealing would?  rows0 is looked for near m_tiles * n0 / pairs.  Returns 0 if not.
+inline int die_split_rows(int64_t m_tiles, int64_t splits, int64_t pairs, int64_t n0) {
+  const int64_t n1 = pairs - n0, units = m_tiles * splits;
+  if (n0 <= 0 || n1 <= 0 || units < pairs || m_tiles < 2) return 0;
+  const int64_t plain_rounds = (units + pairs - 1) / pairs;
+  const int64_t guess = (m_tiles * n0 + pairs / 2) / pairs;
+  int64_t best_rows = 0, best_rounds = INT64_MAX;
+  for (int64_t r0 = guess - 2; r0 <= guess + 2; ++r0) {
+    if (r0 < 1 || r0 >= m_tiles) continue;
+    const int64_t a = (r0 * splits + n0 - 1) / n0, b = ((m_tiles - r0) * splits + n1 - 1) / n1;
+    const int64_t rounds = a > b ? a : b;
+    if (rounds < best_rounds) { best_rounds = rounds; best_rows = r0; }
+  }
+  return best_rows > 0 && best_rounds <= plain_rounds ? (int)best_rows : 0;
+}
 
 inline af_status encode_operand(const GemmEnv& env, CUtensorMap* map, const Operand& op, uint32_t box_rows) {
   TmapCache::Entry* slot = nullptr;
@@ -68,6 +88,8 @@ af_status run_gemm(const GemmEnv& env, const Operand& A, const Operand& B, int s
   g.n_tiles = (int)((N + umma::kBN - 1) / umma::kBN);
   g.splits = splits > 0 && splits < g.n_tiles ? splits : g.n_tiles;
   g.k_blocks = (int)((K + umma::kBK - 1) / umma::kBK);
+  g.die0_pairs = 0;
+  g.die0_rows = 0;
   const int64_t units = (int64_t)g.m_tiles * g.splits;
   if (env.pair) {
     constexpr int smem = E::kStaged ? umma::kPairSmemBytesStaged : umma::kPairSmemBytes;
@@ -76,8 +98,14 @@ af_status run_gemm(const GemmEnv& env, const Operand& A, const Operand& B, int s
     const int pairs = env.sm_count / 2;
     const int grid = 2 * (int)(units < pairs ? units : pairs);
     unsigned int* clock = env.tile_clock;
-    if (clock && cudaMemsetAsync(clock, 0, sizeof(unsigned int), s) != cudaSuccess) return AF_ERR_CUDA;
-    umma::gemm_pair_kernel<E, kAMN, kBMN><<<grid, umma::kThreads, smem, s>>>(ta, tb, g, ep, env.d_err, clock);
+    // die-aware dealing when every SM pair gets a CTA pair and it costs no extra round of units
+    const int rows0 = env.die0_pairs > 0 && env.die_of_sm && clock && units >= pairs
+                          ? die_split_rows(g.m_tiles, g.splits, pairs, env.die0_pairs) : 0;
+    const bool by_die = rows0 > 0;
+    if (by_die) { g.die0_pairs = env.die0_pairs; g.die0_rows = rows0; }
+    if (clock && cudaMemsetAsync(clock, 0, (by_die ? 3 : 1) * sizeof(unsigned int), s) != cudaSuccess) return AF_ERR_CUDA;
+    umma::gemm_pair_kernel<E, kAMN, kBMN><<<grid, umma::kThreads, smem, s>>>(ta, tb, g, ep, env.d_err, clock,
+                                                                             by_die ? clock + 1 : nullptr, env.die_of_sm);
   } else {
     constexpr int smem = E::kStaged ? umma::kSmemBytesStaged : umma::kSmemBytes;
     static SmemAttrOnce once;
@@ -90,7 +118,8 @@ af_status run_gemm(const GemmEnv& env, const Operand& A, const Operand& B, int s
 
 inline GemmEnv gemm_env(af_ctx* ctx) {
   return GemmEnv{ctx->encode, ctx->sm_count, ctx->d_err, ctx->gemm_pair != 0, ctx->d_err + kTileClockWord,
-                 &ctx->tmaps};
+                 &ctx->tmaps, reinterpret_cast<const unsigned char*>(ctx->d_err) + kDieTableByte,
+                 ctx->die_aware && ctx->die0_sms > 0 ? ctx->die0_sms / 2 : 0};
 }
 
 }  // namespace af

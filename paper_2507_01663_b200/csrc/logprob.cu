@@ -128,23 +128,29 @@ __global__ void __launch_bounds__(256) merge_partials_kernel(
 // vocabulary over ceil(workers / S) row tiles whose hidden-state panels should stay L2-resident
 // while W streams past once, which rules out small S for wide hidden sizes.  More than 8 ranges are
 // only allowed while S * T stays small (partials buffer).
-int logprob_pick_splits(int64_t T, int32_t d, int32_t V, int sm_count, bool pair, int requested) {
+int logprob_pick_splits(int64_t T, int32_t d, int32_t V, int sm_count, bool pair, int requested, int die0_pairs) {
   const int tile_rows = pair ? umma::kPairBM : umma::kBM;
   const int workers = pair ? (sm_count / 2 > 0 ? sm_count / 2 : 1) : (sm_count > 0 ? sm_count : 1);
   const int64_t m_tiles = (T + tile_rows - 1) / tile_rows;
   const int n_tiles = (V + umma::kBN - 1) / umma::kBN;
   if (requested > 0) return requested < n_tiles ? requested : n_tiles;
   if (m_tiles < 1) return 1;
-  // bytes of hidden-state rows kept in L2: pairs sharing a row tile may sit on different dies, each
-  // of which then caches the panel in its own half of L2, so pairs get the smaller budget
+  // bytes of hidden-state rows kept in L2.  Pairs sharing a row tile may sit on different dies, each
+  // of which then caches the panel in its own half of L2, so pairs get the smaller budget; with the
+  // row tiles dealt by die a panel lives in one half only and the budget holds per die, i.e. for the
+  // row tiles half of the pairs keep alive
   const int64_t kPanelBudget = pair ? (48ll << 20) : (72ll << 20);
+  const bool by_die = pair && die0_pairs > 0 && die0_pairs < workers;
   const int64_t max_units_many = (int64_t)workers * 8;
   int best = 1;
   double best_cost = 1e300;
   for (int S = 1; S <= 32 && S <= n_tiles; ++S) {
     const int64_t units = m_tiles * S;
     if (S > 8 && units > max_units_many) break;
-    int64_t alive = (workers + S - 1) / S;
+    // by die only where the launch will really deal that way (no extra round of units)
+    const int die_workers = die0_pairs > workers - die0_pairs ? die0_pairs : workers - die0_pairs;
+    const int fit_workers = by_die && die_split_rows(m_tiles, S, workers, die0_pairs) > 0 ? die_workers : workers;
+    int64_t alive = (fit_workers + S - 1) / S;
     if (alive > m_tiles) alive = m_tiles;
     const bool fits = alive * tile_rows * (int64_t)d * 2 <= kPanelBudget;
     const int64_t grid = units < workers ? units : workers;
@@ -161,7 +167,7 @@ af_status launch_token_logprob_z(af_ctx* ctx, const void* hidden, const void* W,
                                  float* logp, float* entropy, float* lse, float* z, cudaStream_t s) {
   if (T == 0) return AF_OK;
   const GemmEnv env = gemm_env(ctx);
-  const int S = logprob_pick_splits(T, d, V, ctx->sm_count, env.pair, ctx->v_splits);
+  const int S = logprob_pick_splits(T, d, V, ctx->sm_count, env.pair, ctx->v_splits, env.die0_pairs);
   af_status st = ws_grow(ctx->partial, (size_t)S * (size_t)T * sizeof(float4));
   if (st != AF_OK) return st;
   const Operand Hop{hidden, (uint64_t)T, (uint64_t)d, (uint64_t)d * 2};
@@ -193,7 +199,7 @@ af_status launch_token_logprob_shard(af_ctx* ctx, const void* hidden, const void
                                      int32_t v_offset, float* partial_out, cudaStream_t s) {
   if (T == 0) return AF_OK;
   const GemmEnv env = gemm_env(ctx);
-  const int S = logprob_pick_splits(T, d, V_shard, ctx->sm_count, env.pair, ctx->v_splits);
+  const int S = logprob_pick_splits(T, d, V_shard, ctx->sm_count, env.pair, ctx->v_splits, env.die0_pairs);
   af_status st = ws_grow(ctx->partial, (size_t)S * (size_t)T * sizeof(float4));
   if (st != AF_OK) return st;
   const Operand Hop{hidden, (uint64_t)T, (uint64_t)d, (uint64_t)d * 2};
@@ -302,12 +308,12 @@ extern "C" af_status af_token_logprob_static(const void* hidden, const void* W, 
   if (d % 8 != 0 || (reinterpret_cast<uintptr_t>(hidden) & 15u) || (reinterpret_cast<uintptr_t>(W) & 15u))
     return AF_ERR_ALIGNMENT;
 
-  int S = logprob_pick_splits(T, d, V, st->sm_count, false, 0);
+  int S = logprob_pick_splits(T, d, V, st->sm_count, false, 0, 0);
   if ((int64_t)S * T > kStaticPartialSlots) S = (int)(kStaticPartialSlots / T);
   unsigned int* err_word = device_flags ? device_flags : reinterpret_cast<unsigned int*>(st->scratch);
   float4* partial = reinterpret_cast<float4*>(st->scratch + kStaticHeaderBytes);
 
-  const GemmEnv env{g_static_encode, st->sm_count, err_word, false, nullptr, nullptr};
+  const GemmEnv env{g_static_encode, st->sm_count, err_word, false, nullptr, nullptr, nullptr, 0};
   const Operand Hop{hidden, (uint64_t)T, (uint64_t)d, (uint64_t)d * 2};
   const Operand Wop{W, (uint64_t)V, (uint64_t)d, (uint64_t)d * 2};
   LogprobEpi::Params ep{target, partial, (int)T, V, 0, nullptr, 0};

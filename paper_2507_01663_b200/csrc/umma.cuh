@@ -190,6 +190,8 @@ struct GemmShape {
   int m_tiles, n_tiles; // ceil(M/128), ceil(N/256)
   int splits;           // S: n-tile ranges per m_tile
   int k_blocks;         // ceil(K/64)
+  int die0_pairs;       // pair kernel only: > 0 = deal the row tiles by die; the number of CTA pairs the first die hosts
+  int die0_rows;        // ... and the number of row tiles (the first ones) those pairs share among themselves
 };
 __device__ __forceinline__ int split_begin(const GemmShape& g, int s) {
   return (int)(((long long)g.n_tiles * s) / g.splits);
@@ -441,12 +443,46 @@ __device__ __forceinline__ void mma_commit_pair(uint32_t bar) {
       ::"r"(bar), "h"((unsigned short)3) : "memory");
 }
 
+__device__ __forceinline__ uint32_t ld_shared_cluster_u32(uint32_t cluster_addr) {
+  uint32_t v;
+  asm volatile("ld.shared::cluster.u32 %0, [%1];" : "=r"(v) : "r"(cluster_addr) : "memory");
+  return v;
+}
+
+// Which units a pair processes.  Plain dealing: the pair of rank r takes units r, r + n_pairs, ...
+// (unit u = row tile u / S, vocabulary range u % S).  Die-aware dealing: the B200 is two dies, each
+// with its own half of L2, and a line that SMs of both dies read is kept in both halves; the A panel
+// of a row tile therefore costs L2 space twice when the pairs working on its S ranges sit on
+// different dies.  Here ranks [0, n0) -- the pairs that run on the first die, which they learn from a
+// measured table of SM ids -- share the first rows0 row tiles among themselves and the other ranks
+// the rest, so a panel lives in one half of L2 only.  Ranks are handed out by atomic counters and are
+// a permutation of 0 .. n_pairs - 1 whatever the table says, so every unit is processed exactly once in
+// either mode; only the cache behaviour depends on the table being right.
+struct PairWork {
+  int first, step, end, base_unit;     // units base_unit + first, base_unit + first + step, ... below base_unit + end
+};
+__device__ __forceinline__ PairWork pair_work(const GemmShape& g, int rank, int n_pairs) {
+  const int total = g.m_tiles * g.splits;
+  const int n0 = g.die0_pairs, n1 = n_pairs - n0;
+  if (n0 <= 0 || n1 <= 0) return PairWork{rank, n_pairs, total, 0};
+  const int rows0 = g.die0_rows;                 // chosen by the host: in proportion to the pairs, rounds balanced
+  if (rank < n0) return PairWork{rank, n0, rows0 * g.splits, 0};
+  return PairWork{rank - n0, n1, (g.m_tiles - rows0) * g.splits, rows0 * g.splits};
+}
+// most units any pair processes in this launch
+__device__ __forceinline__ int pair_work_most(const GemmShape& g, int n_pairs) {
+  const PairWork a = pair_work(g, 0, n_pairs), b = pair_work(g, n_pairs - 1, n_pairs);
+  const int ua = (a.end + a.step - 1) / a.step, ub = (b.end + b.step - 1) / b.step;
+  return ua > ub ? ua : ub;
+}
+
 // Work decomposition of the pair kernel: a unit is one 256-row tile times a range of B tiles;
-// pair p processes units p, p + n_pairs, ...
+// see PairWork for which units a pair processes.
 template <class E, bool kAMN = false, bool kBMN = false>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-                 const GemmShape g, const typename E::Params ep, unsigned int* d_err, unsigned int* tile_clock) {
+                 const GemmShape g, const typename E::Params ep, unsigned int* d_err, unsigned int* tile_clock,
+                 unsigned int* die_counters, const unsigned char* die_of_sm) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles = (raw + 1023u) & ~1023u;
@@ -459,10 +495,11 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
   uint8_t* const epi_stage_base = smem_raw + (bars + 256u - raw);
   volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(smem_raw + (tmem_slot - raw));
   __shared__ int abort_flag;
+  __shared__ uint32_t s_pair_rank;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();          // 0 = leader
-  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+  const int n_pairs = gridDim.x >> 1;
   if (threadIdx.x == 0) {
     abort_flag = 0;
     for (int s = 0; s < kPairStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
@@ -470,6 +507,25 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     fence_mbar_init();
     tma_prefetch_desc(&tmap_a);
     tma_prefetch_desc(&tmap_b);
+    // The pair's rank in the work assignment.  With die-aware dealing the leader looks its SM up in
+    // the table and takes the next rank of that die from the die's counter (the host zeroed both);
+    // should the die already be full -- a table that does not match where the pairs really run -- it
+    // takes one of the other die's: n_pairs claimants for n0 + n1 = n_pairs ranks, so that always works.
+    uint32_t r = (uint32_t)(blockIdx.x >> 1);
+    if (rank == 0 && g.die0_pairs > 0 && g.die0_pairs < n_pairs && die_counters != nullptr && die_of_sm != nullptr) {
+      uint32_t smid;
+      asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+      const uint32_t n0 = (uint32_t)g.die0_pairs, n1 = (uint32_t)n_pairs - n0;
+      uint32_t die = smid < 256u ? (uint32_t)die_of_sm[smid] & 1u : 0u;
+      uint32_t idx = atomicAdd(die_counters + die, 1u);
+      if (idx >= (die ? n1 : n0)) {
+        die ^= 1u;
+        idx = atomicAdd(die_counters + die, 1u);
+        if (idx >= (die ? n1 : n0)) { abort_flag = 1; idx = 0; }     // cannot happen; never run with a duplicate rank
+      }
+      r = die ? n0 + idx : idx;
+    }
+    s_pair_rank = r;
   }
   if (warp == 1) {
     tmem_alloc_pair(tmem_slot, kTmemCols);
@@ -480,8 +536,9 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
   cluster_sync_all();       // the peer's barriers exist before anything is signalled across CTAs
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot_ptr;
-
-  const int total_units = g.m_tiles * g.splits;     // m_tiles counts 256-row tiles here
+  // both CTAs work from the leader's rank
+  const int pair = (int)ld_shared_cluster_u32(map_to_cta(smem_u32(&s_pair_rank), 0));
+  const PairWork work = pair_work(g, pair, n_pairs);  // m_tiles counts 256-row tiles here
 
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer (both CTAs)
@@ -508,11 +565,12 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
       int to_next_tick = 0;                                         // K blocks until the next tick
       const unsigned long long patience = kClockPatienceNs + kClockPatiencePerKBlockNs * (unsigned long long)tick_len;
       // most ticks any pair starts in this launch
-      const unsigned long long most_kb = (unsigned long long)((total_units + n_pairs - 1) / n_pairs) *
+      const unsigned long long most_kb = (unsigned long long)pair_work_most(g, n_pairs) *
                                          (unsigned long long)((g.n_tiles + g.splits - 1) / g.splits) *
                                          (unsigned long long)g.k_blocks;
       const unsigned int clock_most = (unsigned int)((most_kb + tick_len - 1) / tick_len);
-      for (int u = pair; u < total_units && ok; u += n_pairs) {
+      for (int q = work.first; q < work.end && ok; q += work.step) {
+        const int u = work.base_unit + q;
         const int m_tile = u / g.splits, s = u % g.splits;
         const int nb = split_begin(g, s), ne = split_begin(g, s + 1);
         const int m0 = m_tile * kPairBM + (int)rank * kBM;          // this CTA's 128 rows of A
@@ -575,8 +633,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
       constexpr uint32_t idesc = instr_desc_bf16_f32(kPairBM, kBN, kAMN, kBMN);
       constexpr uint64_t a_step = kAMN ? (2048 >> 4) : 2, b_step = kBMN ? (2048 >> 4) : 2;
       int stage = 0; uint32_t phase = 0; uint32_t tile_count = 0; bool ok = true;
-      for (int u = pair; u < total_units && ok; u += n_pairs) {
-        const int s = u % g.splits;
+      for (int q = work.first; q < work.end && ok; q += work.step) {
+        const int s = (work.base_unit + q) % g.splits;
         const int nb = split_begin(g, s), ne = split_begin(g, s + 1);
         for (int nt = nb; nt < ne && ok; ++nt, ++tile_count) {
           const uint32_t acc = tile_count & 1u, acc_phase = (tile_count >> 1) & 1u;
@@ -609,7 +667,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     uint32_t tile_count = 0; bool ok = true;
     typename E::State st;
     uint8_t* const stage = E::kStaged ? epi_stage_base + (warp - 2) * kEpiStageBytes : nullptr;
-    for (int u = pair; u < total_units && ok; u += n_pairs) {
+    for (int q = work.first; q < work.end && ok; q += work.step) {
+      const int u = work.base_unit + q;
       const int m_tile = u / g.splits, s = u % g.splits;
       const int nb = split_begin(g, s), ne = split_begin(g, s + 1);
       const int row = m_tile * kPairBM + row_in_tile;

@@ -164,12 +164,12 @@ def _fixed_total_lengths(seed, n, lo, hi, total):
 def make_workload(name: str, seed_offset: int = 0) -> Workload:
     """The five evaluation workloads (``cfg1`` .. ``cfg5``) and reduced test variants (``*_mini``).
 
-    ``cfg4_mid`` is a profiling-sized actor-update batch (a few GB on the device).  Mini variants keep the structure (group sizes, length law, ragged tails) at sizes a CPU
+    ``cfg2_mid`` and ``cfg4_mid`` are profiling-sized forward and actor-update batches (a few GB on the device).  Mini variants keep the structure (group sizes, length law, ragged tails) at sizes a CPU
     oracle evaluates in seconds; their V is deliberately not a multiple of the GEMM tile.
     ``seed_offset`` derives an independent draw of the same shape (one per data-parallel rank).
     """
     base = {"cfg1": 0, "cfg2": 1, "cfg3": 2, "cfg4": 3, "cfg5": 4,
-            "cfg2_mini": 11, "cfg3_mini": 12, "cfg4_mini": 13, "cfg5_mini": 14, "cfg4_mid": 23}
+            "cfg2_mini": 11, "cfg3_mini": 12, "cfg4_mini": 13, "cfg5_mini": 14, "cfg4_mid": 23, "cfg2_mid": 21}
     if name not in base:
         raise KeyError(name)
     sd = base[name] + seed_offset
@@ -185,6 +185,8 @@ def make_workload(name: str, seed_offset: int = 0) -> Workload:
     if name == "cfg5":
         return Workload(name, sd, 3584, 152064, 64, 64, _pareto_lengths(sd, 4096, 128, 1.5, 16384),
                         "bernoulli:0.3", token_budget=32768)
+    if name == "cfg2_mid":   # the 7B head on a profiling-sized forward batch (about 65 k tokens, a few GB on the device)
+        return Workload(name, sd, 3584, 152064, 4, 8, _uniform_lengths(sd, 32, 1024, 3072), "bernoulli:0.3")
     if name == "cfg4_mid":   # one backward token block at the 7B hidden size, a quarter-size vocabulary
         return Workload(name, sd, 3584, 32768, 2, 8, _fixed_total_lengths(sd, 16, 64, 1024, 9472),
                         "bernoulli:0.5", backward=True)

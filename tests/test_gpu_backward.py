@@ -256,3 +256,22 @@ def test_dw_ready_event_marks_the_complete_gradient(ctx, fused):
         ctx.set_tuning(0, 0)
     assert ctx.check_device_errors() == 0
     assert torch.equal(snap, dW1) and torch.equal(dW1, dW0) and torch.equal(dH1, dH0)
+
+
+def test_backward_with_die_aware_dealing(ctx):
+    """gemm_variant 3 on the backward's three products (the dZ and dH products have enough units for
+    the mode to switch on at this size): dense against the oracle."""
+    if VARIANT != 2:
+        pytest.skip("one run is enough: the test selects its own variant")
+    dev = device()
+    T, d, V = 12000, 264, 2048
+    H, W, y, g, lse = inputs(T, d, V, seed=91)
+    dH = torch.full((T, d), 7.0, dtype=torch.bfloat16, device=dev)
+    dW = torch.full((V, d), 7.0, device=dev)
+    ctx.set_tuning(0, 0, 3)
+    ctx.policy_loss_backward(H.to(dev), W.to(dev), y.to(dev), f32(lse), g.to(dev), dH, dW)
+    flags = ctx.check_device_errors()
+    ctx.set_tuning(0, 0)
+    assert flags == 0
+    dH_ref, dW_ref = O.policy_loss_backward_ref(wl.bf16_bits(H), wl.bf16_bits(W), y.numpy(), lse, g.numpy())
+    compare(np_of(dH.float()), np_of(dW), dH_ref, dW_ref)

@@ -333,8 +333,10 @@ def test_vocabulary_parallel_head_full_size(ctx):
     assert np.abs(np_of(logp[rt]) - o_logp).max() <= LOGP_TOL
     assert np.abs(np_of(ent[rt]) - o_ent).max() <= LOGP_TOL
     assert np.abs(np_of(lse[rt]) - o_lse).max() <= LOGP_TOL
+    # the two CUDA paths sum the vocabulary in different groupings (fp32, approximate exp2): a loose
+    # consistency check beside the oracle comparison above
     for got, ref in zip((logp, ent, lse), one):
-        assert float((got - ref).abs().max()) <= 1e-4
+        assert float((got - ref).abs().max()) <= 3e-4
     # exactly one shard holds every token's target
     assert bool((torch.isfinite(partials[:, :, 3]).sum(0) == 1).all())
 

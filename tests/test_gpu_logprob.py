@@ -313,3 +313,24 @@ def test_shard_argument_errors(ctx):
     ctx.merge_logprob_shards(part, y, 8, out)
     assert ctx.check_device_errors() == B.DEVERR_TARGET_RANGE
     assert torch.isnan(out[1]) and not torch.isnan(out[0])
+
+
+def test_die_aware_dealing_of_row_tiles(ctx):
+    """gemm_variant 3: the pairs claim ranks by the SM they run on and each half of the chip shares its
+    own row tiles.  Every unit must still be processed exactly once: all rows against the oracle,
+    at sizes with several units per pair (the mode switches itself off below that), on ragged shapes."""
+    for T, d, V, splits in [(40000, 64, 1024, 0), (50001, 72, 1500, 2), (38400, 128, 520, 0)]:
+        H, W, y = random_case(T, d, V, seed=T)
+        dev = device()
+        logp, ent, lse = (torch.full((T,), 9.0, device=dev) for _ in range(3))
+        ctx.set_tuning(splits, 0, 3)
+        ctx.token_logprob(H.to(dev), W.to(dev), y.to(dev), logp, ent, lse)
+        again = torch.full((T,), 9.0, device=dev)
+        ctx.token_logprob(H.to(dev), W.to(dev), y.to(dev), again)
+        flags = ctx.check_device_errors()
+        ctx.set_tuning(0, 0)
+        assert flags == 0
+        want = O.token_logprob_ref(wl.bf16_bits(H), wl.bf16_bits(W), y.numpy())
+        for got, ref in zip((logp, ent, lse), want):
+            assert np.abs(np_of(got) - ref).max() <= LOGP_TOL
+        assert torch.equal(again, logp)              # the claimed ranks may differ between launches, the bits may not
