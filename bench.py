@@ -1112,7 +1112,11 @@ def run_ours(args):
         "scaling": "strong" if args.vocab_parallel else "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": describe(w, job, args.workload),
                    "l2": "inputs (hidden states >> 126 MB L2) exceed L2; no flush needed",
-                   "gemm": "one CTA per 128x256 tile" if args.gemm == "single" else "CTA pairs (cta_group::2), 256x256 tiles",
+                   "gemm": "one CTA per 128x256 tile" if args.gemm == "single" else
+                           "CTA pairs (cta_group::2), 256x256 tiles" + (", dealt without regard to dies" if args.gemm == "pair"
+                                                                        else ", row tiles dealt by die"),
+                   "die_split_sms": list(job.ctx.die_split()),
+                   "l2_bytes": int(torch.cuda.get_device_properties(dev).L2_cache_size),
                    "parallelism": ("vocabulary-parallel head" if args.vocab_parallel else
                                    f"dp{world}: global batch dealt by token count (Karmarkar-Karp, equal counts)" if dp
                                    else f"dp{world}: a store per rank" if world > 1 else "single GPU"),

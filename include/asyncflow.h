@@ -91,8 +91,11 @@ int64_t af_workspace_bytes(const af_ctx* ctx);
 af_status af_set_tuning(af_ctx* ctx, int32_t v_splits, int32_t bwd_token_block, int32_t gemm_variant);
 
 /* How af_create found the SMs split over the two dies of the part (each die has its own half of
- * L2): the number of SMs that share a die with the first SM probed, and the rest.  Both 0 when the
- * latency measurement behind it was not clear-cut (then work is dealt without regard to dies). */
+ * L2): the number of SMs that share a die with the first SM probed, and the rest.  When the latency
+ * measurement behind it was not clear-cut after several attempts (then work is dealt without regard
+ * to dies), *die0_sms is 0 and *die1_sms is minus the reason: 1 a CUDA call failed, 2 SM ids out of
+ * range or repeated, 3 an SM between the two groups, 4 an SM pair straddling the dies, 5 a lopsided
+ * split. */
 af_status af_die_split(const af_ctx* ctx, int32_t* die0_sms, int32_t* die1_sms);
 
 /* Data-parallel actor update (Section 4.1: the training batch is streamed to the DP groups of the

@@ -93,7 +93,8 @@ af_status af_create(af_ctx** out, int device) {
   if (cudaMalloc(&c->d_err, kDeviceBlockBytes) != cudaSuccess) { c->d_err = nullptr; cudaGetLastError(); af_destroy(c); return AF_ERR_WORKSPACE; }
   if (cudaMemset(c->d_err, 0, kDeviceBlockBytes) != cudaSuccess) { af_destroy(c); return AF_ERR_CUDA; }
   // which SMs share a die (for die-aware dealing of GEMM row tiles); 0 when the measurement is unclear
-  if (!measure_die_map(c->sm_count, reinterpret_cast<unsigned char*>(c->d_err) + kDieTableByte, &c->die0_sms)) c->die0_sms = 0;
+  if (!measure_die_map(c->sm_count, reinterpret_cast<unsigned char*>(c->d_err) + kDieTableByte, &c->die0_sms,
+                       &c->die_map_reason)) c->die0_sms = 0;
   c->die_aware = 1;
   af_status st = ws_grow(c->loss_ws, loss_workspace_bytes(c->sm_count));
   if (st == AF_OK && cudaMemset(c->loss_ws.p, 0, c->loss_ws.cap) != cudaSuccess) st = AF_ERR_CUDA;
@@ -126,7 +127,7 @@ int64_t af_workspace_bytes(const af_ctx* c) {
 af_status af_die_split(const af_ctx* c, int32_t* die0_sms, int32_t* die1_sms) {
   if (!c || !die0_sms || !die1_sms) return AF_ERR_INVALID_ARG;
   *die0_sms = c->die0_sms;
-  *die1_sms = c->die0_sms > 0 ? c->sm_count - c->die0_sms : 0;
+  *die1_sms = c->die0_sms > 0 ? c->sm_count - c->die0_sms : -c->die_map_reason;
   return AF_OK;
 }
 

@@ -77,6 +77,7 @@ struct af_ctx {
   int gemm_pair = 1;        // 1 = CTA-pair GEMM variant (the default), 0 = one CTA per tile
   int die_aware = 0;        // pair variant: deal row tiles to pairs by the die they run on
   int die0_sms = 0;         // SMs on the die of the first SM probed (0: the measurement was not clear-cut; no die-aware dealing)
+  int die_map_reason = 0;   // why not, if so (see diemap.cu)
   cudaEvent_t dw_ready = nullptr;  // caller's event recorded once d_W is complete (af_set_dw_ready_event)
 
   af::TmapCache tmaps;      // tensor maps of the GEMM operands seen so far
@@ -104,7 +105,7 @@ namespace af {
 af_status ws_grow(Buf& b, size_t bytes);
 
 // Measures which SMs share a die (device table of 256 bytes indexed by SM id); false if unclear.
-bool measure_die_map(int sm_count, unsigned char* d_table, int* die0_sms);
+bool measure_die_map(int sm_count, unsigned char* d_table, int* die0_sms, int* reason);
 
 // ---- launchers (each returns the cudaGetLastError of its launches) --------------------------
 struct PackSeqTable {     // device views into ctx->pack_meta for one call

@@ -60,11 +60,11 @@ __global__ void __launch_bounds__(32) die_probe_kernel(const unsigned* buf, unsi
 
 }  // namespace
 
-// Fills table[smid] = 0 / 1 (device, kMaxSmid bytes) and *die0_sms; returns false (table untouched)
-// when the measurement is not clear-cut, in which case the caller deals the work without regard to dies.
-bool measure_die_map(int sm_count, unsigned char* d_table, int* die0_sms) {
-  *die0_sms = 0;
-  if (sm_count < 4 || sm_count > kMaxSmid) return false;
+namespace {
+// One measurement.  Returns 0 and fills `table` / *die0_sms, or the reason it is not clear-cut:
+// 1 a CUDA call failed, 2 an SM id out of range or seen twice, 3 an SM between the two groups,
+// 4 an SM pair straddling the dies, 5 a lopsided split.
+int measure_once(int sm_count, std::vector<unsigned char>& table, int* die0_sms) {
   unsigned *buf = nullptr, *scratch = nullptr;
   const size_t buf_bytes = (size_t)kAddr * kStrideWords * 4 + 4096;
   const size_t scratch_words = 1 + (size_t)sm_count * (1 + kAddr);
@@ -81,14 +81,14 @@ bool measure_die_map(int sm_count, unsigned char* d_table, int* die0_sms) {
   } while (false);
   if (buf) cudaFree(buf);
   if (scratch) cudaFree(scratch);
-  if (!ok) { cudaGetLastError(); return false; }
+  if (!ok) { cudaGetLastError(); return 1; }
 
   const unsigned* smid = host.data() + 1;
   const unsigned* lat = host.data() + 1 + sm_count;
   // every SM id below kMaxSmid, each seen once
   std::vector<int> block_of(kMaxSmid, -1);
   for (int b = 0; b < sm_count; ++b) {
-    if (smid[b] >= (unsigned)kMaxSmid || block_of[smid[b]] >= 0) return false;
+    if (smid[b] >= (unsigned)kMaxSmid || block_of[smid[b]] >= 0) return 2;
     block_of[smid[b]] = b;
   }
   std::vector<double> mean(kAddr, 0.0);
@@ -107,12 +107,12 @@ bool measure_die_map(int sm_count, unsigned char* d_table, int* die0_sms) {
       s += zb * (lat[k] - mean[k]);
       nb += zb * zb;
     }
-    if (!(nb > 0.0) || !(norm0 > 0.0)) return false;
+    if (!(nb > 0.0) || !(norm0 > 0.0)) return 3;
     dot[b] = s / std::sqrt(nb * norm0);
     weakest = std::min(weakest, std::fabs(dot[b]));
   }
-  if (weakest < 0.15) return false;                          // some SM sits between the two groups: no clear split
-  std::vector<unsigned char> table(kMaxSmid, 0);
+  if (weakest < 0.15) return 3;                              // some SM sits between the two groups: no clear split
+  table.assign(kMaxSmid, 0);
   int n0 = 0;
   for (int b = 0; b < sm_count; ++b) {
     const unsigned char die = dot[b] > 0.0 ? 0 : 1;          // die 0 = the die of the first block's SM
@@ -121,11 +121,31 @@ bool measure_die_map(int sm_count, unsigned char* d_table, int* die0_sms) {
   }
   // SM pairs (ids 2k, 2k+1) host CTA pairs: they must not straddle the dies, and both dies must be there
   for (int k = 0; 2 * k + 1 < kMaxSmid; ++k)
-    if (block_of[2 * k] >= 0 && block_of[2 * k + 1] >= 0 && table[2 * k] != table[2 * k + 1]) return false;
-  if (n0 % 2 != 0 || n0 < sm_count / 4 || n0 > 3 * sm_count / 4) return false;
-  if (cudaMemcpy(d_table, table.data(), kMaxSmid, cudaMemcpyHostToDevice) != cudaSuccess) { cudaGetLastError(); return false; }
+    if (block_of[2 * k] >= 0 && block_of[2 * k + 1] >= 0 && table[2 * k] != table[2 * k + 1]) return 4;
+  if (n0 % 2 != 0 || n0 < sm_count / 4 || n0 > 3 * sm_count / 4) return 5;
   *die0_sms = n0;
-  return true;
+  return 0;
+}
+}  // namespace
+
+// Fills table[smid] = 0 / 1 (device, kMaxSmid bytes) and *die0_sms.  The measurement is repeated a few
+// times if it does not come out clear-cut (another process on the GPU, a profiler's instrumentation);
+// if it never does, returns false with *reason set (table untouched) and the caller deals the work
+// without regard to dies.
+bool measure_die_map(int sm_count, unsigned char* d_table, int* die0_sms, int* reason) {
+  *die0_sms = 0;
+  *reason = 1;
+  if (sm_count < 4 || sm_count > kMaxSmid) return false;
+  std::vector<unsigned char> table;
+  for (int attempt = 0; attempt < 4; ++attempt) {
+    int n0 = 0;
+    *reason = measure_once(sm_count, table, &n0);
+    if (*reason != 0) continue;
+    if (cudaMemcpy(d_table, table.data(), kMaxSmid, cudaMemcpyHostToDevice) != cudaSuccess) { cudaGetLastError(); *reason = 1; return false; }
+    *die0_sms = n0;
+    return true;
+  }
+  return false;
 }
 
 }  // namespace af

@@ -140,6 +140,11 @@ int logprob_pick_splits(int64_t T, int32_t d, int32_t V, int sm_count, bool pair
   // row tiles dealt by die a panel lives in one half only and the budget holds per die, i.e. for the
   // row tiles half of the pairs keep alive
   const int64_t kPanelBudget = pair ? (48ll << 20) : (72ll << 20);
+  // by die: the panels of the die with more pairs.  Its half of L2 also holds the home copies of
+  // about half of the other die's panels and the weight tiles in flight; 19 row tiles of the 7B
+  // head (34.9 MB) stream W once per wave, 20 (36.7 MB, on a part whose dies have 70 and 78 SMs)
+  // tripled the DRAM reads
+  const int64_t kDiePanelBudget = 36ll << 20;
   const bool by_die = pair && die0_pairs > 0 && die0_pairs < workers;
   const int64_t max_units_many = (int64_t)workers * 8;
   int best = 1;
@@ -149,10 +154,11 @@ int logprob_pick_splits(int64_t T, int32_t d, int32_t V, int sm_count, bool pair
     if (S > 8 && units > max_units_many) break;
     // by die only where the launch will really deal that way (no extra round of units)
     const int die_workers = die0_pairs > workers - die0_pairs ? die0_pairs : workers - die0_pairs;
-    const int fit_workers = by_die && die_split_rows(m_tiles, S, workers, die0_pairs) > 0 ? die_workers : workers;
+    const bool die_here = by_die && die_split_rows(m_tiles, S, workers, die0_pairs) > 0;
+    const int fit_workers = die_here ? die_workers : workers;
     int64_t alive = (fit_workers + S - 1) / S;
     if (alive > m_tiles) alive = m_tiles;
-    const bool fits = alive * tile_rows * (int64_t)d * 2 <= kPanelBudget;
+    const bool fits = alive * tile_rows * (int64_t)d * 2 <= (die_here ? kDiePanelBudget : kPanelBudget);
     const int64_t grid = units < workers ? units : workers;
     double cost = (double)((units + grid - 1) / grid) * (double)((n_tiles + S - 1) / S);
     cost *= 1.0 + 0.002 * S;                          // partials written and merged per range
