@@ -41,12 +41,14 @@ from paper_2507_01663_b200 import workloads as wl  # noqa: E402
 METRIC = "scored tokens/sec (logprob+GRPO loss) at Qwen-7B head; % dense-BF16 peak"
 UNIT = "tokens/s"
 KERNELS_PER_STEP = 7  # advantage, pack table fetch, pack columns, pack rows (bulk copy), fused LM-head GEMM, partial merge, loss
-# DRAM bytes per scored token of the fused LM-head kernel (dram__bytes_read + dram__bytes_write of
-# one ncu capture of the CTA-pair kernel at T = 65536, d = 3584, V = 152064 with the three
-# vocabulary ranges the library picks at the bench size: 13.752 GB + 8.5 MB; traffic grows with the
-# number of waves of row tiles, i.e. in proportion to T).  Valid for the 7B head shape only; None whenever the kernel
-# or its work decomposition has changed since the counters were taken.
-GEMM_DRAM_BYTES_PER_TOKEN_7B = (13.752132e9 + 8.53e6) / 65536
+# DRAM bytes per scored token of the fused LM-head kernel (dram__bytes_read of one ncu capture of the
+# CTA-pair kernel, row tiles dealt by die, two vocabulary ranges -- what the library picks at the
+# bench size -- on `--workload cfg2_mid --v-splits 2`: T = 62989, d = 3584, V = 152064; 8.306 and
+# 8.838 GB for two launches on a part with 70 + 78 SMs per die, 8.46-8.47 GB on one with 72 + 76; writes
+# are 7-10 MB; traffic grows with the number of waves of row tiles, i.e. in proportion to T).  Valid
+# for the 7B head shape and the default kernel only; None whenever the kernel or its work
+# decomposition has changed since the counters were taken.
+GEMM_DRAM_BYTES_PER_TOKEN_7B = (8.572e9 + 8.5e6) / 62989
 BWD_TOKEN_BLOCK = 9472  # the library's default backward block (3 GEMM launches per block)
 
 
@@ -1128,7 +1130,8 @@ def run_ours(args):
                      "kernel_ms": gemm_ms,
                      "traffic": (GEMM_DRAM_BYTES_PER_TOKEN_7B * job.T
                                  if GEMM_DRAM_BYTES_PER_TOKEN_7B and (w.d, w.V) == (3584, 152064)
-                                 and args.gemm != "single" and args.v_splits == 0 and not w.token_budget else None)},
+                                 and args.gemm in ("default", "die") and args.v_splits == 0 and not w.token_budget
+                                 and job.ctx.die_split()[0] > 0 else None)},
         "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": job.h2d_bytes,
                 "d2h_bytes_per_step": int(job.d2h_bytes), "ms_per_step": ms_e2e,
                 "d2h": "per-token log-probs in packed order (4 B per token) and the loss record",

@@ -140,10 +140,9 @@ int logprob_pick_splits(int64_t T, int32_t d, int32_t V, int sm_count, bool pair
   // row tiles dealt by die a panel lives in one half only and the budget holds per die, i.e. for the
   // row tiles half of the pairs keep alive
   const int64_t kPanelBudget = pair ? (48ll << 20) : (72ll << 20);
-  // by die: the panels of the die with more pairs.  Its half of L2 also holds the home copies of
-  // about half of the other die's panels and the weight tiles in flight; 19 row tiles of the 7B
-  // head (34.9 MB) stream W once per wave, 20 (36.7 MB, on a part whose dies have 70 and 78 SMs)
-  // tripled the DRAM reads
+  // by die: the panels of the die with more pairs.  Its half of L2 also holds lines of the other
+  // die's panels and the weight tiles in flight; 19 and 20 row tiles of the 7B head (34.9 and
+  // 36.7 MB, parts with 72 + 76 and 70 + 78 SMs) stream W once per wave, which sets this budget
   const int64_t kDiePanelBudget = 36ll << 20;
   const bool by_die = pair && die0_pairs > 0 && die0_pairs < workers;
   const int64_t max_units_many = (int64_t)workers * 8;
