@@ -136,14 +136,18 @@ bool measure_die_map(int sm_count, unsigned char* d_table, int* die0_sms, int* r
   *die0_sms = 0;
   *reason = 1;
   if (sm_count < 4 || sm_count > kMaxSmid) return false;
-  std::vector<unsigned char> table;
-  for (int attempt = 0; attempt < 4; ++attempt) {
-    int n0 = 0;
-    *reason = measure_once(sm_count, table, &n0);
-    if (*reason != 0) continue;
-    if (cudaMemcpy(d_table, table.data(), kMaxSmid, cudaMemcpyHostToDevice) != cudaSuccess) { cudaGetLastError(); *reason = 1; return false; }
-    *die0_sms = n0;
-    return true;
+  try {
+    std::vector<unsigned char> table;
+    for (int attempt = 0; attempt < 4; ++attempt) {
+      int n0 = 0;
+      *reason = measure_once(sm_count, table, &n0);
+      if (*reason != 0) continue;
+      if (cudaMemcpy(d_table, table.data(), kMaxSmid, cudaMemcpyHostToDevice) != cudaSuccess) { cudaGetLastError(); *reason = 1; return false; }
+      *die0_sms = n0;
+      return true;
+    }
+  } catch (...) {       // host allocation failed: no exception may reach the C boundary
+    *reason = 1;
   }
   return false;
 }

@@ -334,3 +334,14 @@ def test_die_aware_dealing_of_row_tiles(ctx):
         for got, ref in zip((logp, ent, lse), want):
             assert np.abs(np_of(got) - ref).max() <= LOGP_TOL
         assert torch.equal(again, logp)              # the claimed ranks may differ between launches, the bits may not
+
+
+def test_die_split_measured_at_creation(ctx):
+    """The latency probe behind die-aware dealing: either a clean split of the SMs into two dies (even
+    counts that add up to the SM count, neither die tiny) or a stated reason for having none."""
+    a, b = ctx.die_split()
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    if a > 0:
+        assert a + b == sms and a % 2 == 0 and b % 2 == 0 and min(a, b) >= sms // 4
+    else:
+        assert a == 0 and -5 <= b <= -1
