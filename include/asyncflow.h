@@ -90,6 +90,14 @@ int64_t af_workspace_bytes(const af_ctx* ctx);
  * Results agree within the stated tolerances either way. */
 af_status af_set_tuning(af_ctx* ctx, int32_t v_splits, int32_t bwd_token_block, int32_t gemm_variant);
 
+/* Self-test of the bounded waits (the paper has no counterpart; failure handling of this library).
+ * Every wait inside the kernels gives up after a time limit, sets AF_DEVERR_WATCHDOG and lets the
+ * kernel return; nothing traps or spins without bound.  This call runs that same wait for one warp
+ * on a barrier nobody arrives at, with a limit of one millisecond, synchronises `stream` and returns
+ * how long the warp waited (microseconds, nullable).  Afterwards af_check_device_errors reports (and
+ * clears) AF_DEVERR_WATCHDOG, and the context is as usable as before. */
+af_status af_selftest_bounded_wait(af_ctx* ctx, uint32_t* waited_us, void* stream);
+
 /* How af_create found the SMs split over the two dies of the part (each die has its own half of
  * L2): the number of SMs that share a die with the first SM probed, and the rest.  When the latency
  * measurement behind it was not clear-cut after several attempts (then work is dealt without regard

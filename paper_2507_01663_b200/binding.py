@@ -27,7 +27,7 @@ EXPORTS = ["af_create", "af_destroy", "af_status_string", "af_reserve", "af_work
            "af_set_tuning", "af_check_device_errors", "af_pack_microbatch", "af_token_logprob",
            "af_grpo_advantage", "af_policy_loss", "af_policy_loss_backward", "af_token_logprob_static",
            "af_controller_put", "af_controller_get", "af_controller_clear", "af_balance_partitions",
-           "af_token_logprob_shard", "af_merge_logprob_shards", "af_policy_update", "af_unpack_microbatch", "af_policy_loss_backward_shard", "af_set_dw_ready_event", "af_die_split"]
+           "af_token_logprob_shard", "af_merge_logprob_shards", "af_policy_update", "af_unpack_microbatch", "af_policy_loss_backward_shard", "af_set_dw_ready_event", "af_die_split", "af_selftest_bounded_wait"]
 MAX_WRITE_COLS = 4
 
 
@@ -102,6 +102,7 @@ def load_library() -> C.CDLL:
     lib.af_check_device_errors.argtypes = [vp, C.POINTER(C.c_uint32), vp]
     lib.af_set_dw_ready_event.argtypes = [vp, vp]
     lib.af_die_split.argtypes = [vp, C.POINTER(i32), C.POINTER(i32)]
+    lib.af_selftest_bounded_wait.argtypes = [vp, C.POINTER(C.c_uint32), vp]
     lib.af_pack_microbatch.argtypes = [vp, C.POINTER(StoreView), vp, i32, C.POINTER(Packed),
                                        C.POINTER(i64), vp]
     lib.af_token_logprob.argtypes = [vp, vp, vp, vp, i64, i32, i32, vp, vp, vp, vp]
@@ -192,6 +193,13 @@ class Context:
         a, b = C.c_int32(0), C.c_int32(0)
         _check(self.lib.af_die_split(self.handle, C.byref(a), C.byref(b)), "af_die_split")
         return int(a.value), int(b.value)
+
+    def selftest_bounded_wait(self, stream=None) -> int:
+        """Run the library's bounded wait on a barrier nobody arrives at (limit: 1 ms); returns the
+        microseconds the warp waited.  Leaves DEVERR_WATCHDOG set for check_device_errors."""
+        us = C.c_uint32(0)
+        _check(self.lib.af_selftest_bounded_wait(self.handle, C.byref(us), _stream(stream)), "af_selftest_bounded_wait")
+        return int(us.value)
 
     def check_device_errors(self, stream=None) -> int:
         """Synchronise the stream; return the device error bits (0 = none) and clear them."""

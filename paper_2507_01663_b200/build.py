@@ -14,7 +14,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libasyncflow.so")
-SOURCES = ["api.cu", "pack.cu", "advantage.cu", "advantage_ids.cu", "loss.cu", "logprob.cu", "backward.cu", "controller.cu", "update.cu", "diemap.cu"]
+SOURCES = ["api.cu", "pack.cu", "advantage.cu", "advantage_ids.cu", "loss.cu", "logprob.cu", "backward.cu", "controller.cu", "update.cu", "diemap.cu", "selftest.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 

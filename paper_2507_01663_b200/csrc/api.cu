@@ -124,6 +124,19 @@ int64_t af_workspace_bytes(const af_ctx* c) {
   return (int64_t)(c->partial.cap + c->loss_ws.cap + c->pack_meta.cap + c->dz.cap + c->ctrl_ws.cap + c->zlog.cap + c->adv_ws.cap);
 }
 
+af_status af_selftest_bounded_wait(af_ctx* c, uint32_t* waited_us, void* stream) {
+  if (!c) return AF_ERR_INVALID_ARG;
+  DeviceGuard guard(c->device);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  unsigned int* d_us = c->d_err + 20;           // a spare word of the context's device block
+  if (launch_bounded_wait_selftest(c->d_err, d_us, s) != cudaSuccess) return AF_ERR_CUDA;
+  unsigned int us = 0;
+  if (cudaMemcpyAsync(&us, d_us, sizeof(us), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+      cudaStreamSynchronize(s) != cudaSuccess) return AF_ERR_CUDA;
+  if (waited_us) *waited_us = us;
+  return AF_OK;
+}
+
 af_status af_die_split(const af_ctx* c, int32_t* die0_sms, int32_t* die1_sms) {
   if (!c || !die0_sms || !die1_sms) return AF_ERR_INVALID_ARG;
   *die0_sms = c->die0_sms;

@@ -107,6 +107,9 @@ af_status ws_grow(Buf& b, size_t bytes);
 // Measures which SMs share a die (device table of 256 bytes indexed by SM id); false if unclear.
 bool measure_die_map(int sm_count, unsigned char* d_table, int* die0_sms, int* reason);
 
+// One warp waits (at most a millisecond) on a barrier nobody arrives at; sets AF_DEVERR_WATCHDOG.
+cudaError_t launch_bounded_wait_selftest(unsigned int* d_err, unsigned int* waited_us, cudaStream_t s);
+
 // ---- launchers (each returns the cudaGetLastError of its launches) --------------------------
 struct PackSeqTable {     // device views into ctx->pack_meta for one call
   const int64_t* src_row; // [B] first store row of sequence j

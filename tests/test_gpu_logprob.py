@@ -345,3 +345,15 @@ def test_die_split_measured_at_creation(ctx):
         assert a + b == sms and a % 2 == 0 and b % 2 == 0 and min(a, b) >= sms // 4
     else:
         assert a == 0 and -5 <= b <= -1
+
+
+def test_a_wait_that_nothing_satisfies_ends_by_itself(ctx):
+    """Failure detection on the device: the bounded wait every kernel uses gives up after its limit
+    (one millisecond here), raises the watchdog flag and returns; the context then works as before."""
+    from paper_2507_01663_b200 import binding as B
+    assert ctx.check_device_errors() == 0
+    waited = ctx.selftest_bounded_wait()
+    assert 900 <= waited <= 50000                    # the limit, plus at most a scheduling hiccup
+    assert ctx.check_device_errors() == B.DEVERR_WATCHDOG
+    assert ctx.check_device_errors() == 0            # read clears it
+    check(ctx, *random_case(300, 64, 520, seed=3))   # and scoring still matches the oracle
