@@ -478,7 +478,10 @@ class ScoringJob:
             ms = avg_ms(lambda: c.grpo_advantage(r[:n_id], ids, n_id // G, a[:n_id]), n=5)
             gbs = 36.0 * n_id / ms / 1e6
             out["grpo_advantage_" + label] = {"responses": n_id, "groups": n_id // G, "bytes_per_response": 36, "ms": ms,
-                                              "gbs": gbs, "frac": gbs / peak_gbs}
+                                              "gbs": gbs, "frac": gbs / peak_gbs,
+                                              "bound": "integer atomics on a table of 64 B per group (537 MB here, beyond "
+                                                       "L2): read-modify-write of accumulator lines, not streaming; "
+                                                       "microseconds at workload sizes (N <= 4096)"}
         del r, a, ids
         # controller: one read request against a 2^log2_n-sample status table (12 B read per sample:
         # ready, consumed, length) that hands out the first 4096 eligible samples

@@ -165,7 +165,7 @@ def test_captured_step_replays_on_new_data(ctx, name, variant):
 def test_replay_of_a_launch_bound_scoring_step(ctx):
     """At the smallest workload the scoring step (advantage, log-prob, loss) runs for a few tens of
     microseconds on the device and the host's launches take longer than that.  The replay must give
-    the plain calls' results bit for bit; the two timings are printed, not asserted (a shared box can
+    the plain calls' results bit for bit; the two timings are printed, not asserted (a shared machine can
     disturb either loop; timing belongs to the benchmark)."""
     w = wl.make_workload("cfg1")
     first, _ = data_sets(w)
