@@ -71,8 +71,10 @@ af_status af_destroy(af_ctx* ctx);
 const char* af_status_string(af_status s);
 
 /* Pre-size the workspace for micro-batches of up to max_T tokens and max_B sequences at head
- * shape (d, V).  with_backward != 0 also reserves the scratch of af_policy_loss_backward, and
- * with_backward == 2 that of af_policy_update too.  Synchronous (allocates). */
+ * shape (d, V), and for af_grpo_advantage by group id with up to max_B groups (pass the number of
+ * stored responses as max_B if advantages are taken over the whole store).  with_backward != 0
+ * also reserves the scratch of af_policy_loss_backward, and with_backward == 2 that of
+ * af_policy_update too.  Synchronous (allocates). */
 af_status af_reserve(af_ctx* ctx, int64_t max_T, int32_t max_B, int32_t d, int32_t V,
                      int32_t with_backward);
 
@@ -223,7 +225,8 @@ af_status af_merge_logprob_shards(af_ctx* ctx, const float* partials, const int3
  * N % n_groups must be 0).  With group_id given the work is O(N) whatever n_groups is: the group
  * sums are exact fixed-point sums taken with integer atomics, so the result does not depend on the
  * order of the members and is bit-reproducible; N < 2^31 (AF_ERR_SHAPE); a per-group accumulator
- * table (64 B per group) is kept in the context's workspace; a sample whose id lies outside
+ * table (64 B per group) is kept in the context's workspace (grown on demand, or ahead of time by
+ * af_reserve for max_B groups); a sample whose id lies outside
  * [0, n_groups) gets a NaN advantage and raises AF_DEVERR_GROUP_ID; groups without members are fine.
  * ddof is 0 or 1.  eps_adv must be > 0 (AF_ERR_INVALID_ARG otherwise: with eps_adv = 0 a group of
  * equal rewards would divide 0 by 0).  adv [N] fp32 dev.

@@ -202,6 +202,9 @@ af_status af_reserve(af_ctx* c, int64_t max_T, int32_t max_B, int32_t d, int32_t
   }
   st = ws_grow(c->pack_meta, pack_meta_bytes(max_B));
   if (st != AF_OK) return st;
+  // af_grpo_advantage by group id: one accumulator per group, and a batch has at most one group per response
+  st = ws_grow(c->adv_ws, advantage_ids_workspace_bytes(max_B));
+  if (st != AF_OK) return st;
   if (with_backward) {
     // sizes are recomputed (and grown if needed) by the backward call itself
     st = launch_backward(c, nullptr, nullptr, nullptr, nullptr, nullptr, max_T, d, V, nullptr, nullptr,

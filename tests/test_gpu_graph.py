@@ -203,3 +203,36 @@ def test_replay_of_a_launch_bound_scoring_step(ctx):
     for k, v in want.items():
         assert torch.equal(getattr(st, k), v), k
     assert ctx.check_device_errors() == 0
+
+
+def test_advantage_by_group_id_is_recordable_right_after_reserve(ctx):
+    """The per-group accumulators of the id path belong to what af_reserve sizes: a context that has
+    never taken advantages by id records the call without growing its workspace, and the replay on
+    new rewards agrees with the oracle and, bit for bit, with the plain call."""
+    w = wl.make_workload("cfg5_mini")
+    dev = device()
+    ctx.reserve(w.total_tokens, w.N, w.d, w.V, with_backward=0)
+    reserved = ctx.workspace_bytes()
+    order = np.random.default_rng(5).permutation(w.N)
+    gid_host = np.asarray(w.group_id, dtype=np.int32)[order]
+    gid = torch.as_tensor(gid_host, device=dev)
+    reward = torch.empty(w.N, device=dev)
+    adv = torch.empty(w.N, device=dev)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        ctx.grpo_advantage(reward, gid, w.n_prompts, adv)
+    assert ctx.workspace_bytes() == reserved
+    for flip in (False, True):
+        r = wl.gen_reward(w).numpy()[order]
+        r = (1.0 - r) if flip else r
+        reward.copy_(torch.as_tensor(r))
+        adv.fill_(9.0)
+        graph.replay()
+        torch.cuda.synchronize()
+        replayed = adv.clone()
+        assert np.abs(np_of(replayed) - O.grpo_advantage_ref(r, gid_host, w.n_prompts)).max() <= ADV_TOL
+        adv.fill_(9.0)
+        ctx.grpo_advantage(reward, gid, w.n_prompts, adv)
+        torch.cuda.synchronize()
+        assert torch.equal(adv, replayed)
+    assert ctx.check_device_errors() == 0
