@@ -40,7 +40,7 @@ from paper_2507_01663_b200 import workloads as wl  # noqa: E402
 
 METRIC = "scored tokens/sec (logprob+GRPO loss) at Qwen-7B head; % dense-BF16 peak"
 UNIT = "tokens/s"
-KERNELS_PER_STEP = 7  # advantage, pack table fetch, pack columns, pack rows (bulk copy), fused LM-head GEMM, partial merge, loss
+KERNELS_PER_STEP = 6  # advantage, pack table fetch, pack (rows by bulk copy + the 4-byte columns), fused LM-head GEMM, partial merge, loss
 # DRAM bytes per scored token of the fused LM-head kernel (dram__bytes_read of one ncu capture of the
 # CTA-pair kernel, row tiles dealt by die, two vocabulary ranges -- what the library picks at the
 # bench size -- on `--workload cfg2_mid --v-splits 2`: T = 62989, d = 3584, V = 152064; 8.306 and

@@ -9,7 +9,8 @@
 // per CTA through a ring of shared-memory stages: no payload byte passes through a register, and
 // the number of bytes in flight does not depend on how many threads are resident.  Rows wider
 // than a chunk fall back to a warp-per-row copy with 128-bit loads and stores.  The 4-byte
-// columns are gathered by a second, small kernel (one thread per token).
+// columns are gathered one thread per token, by the other warps of the same CTAs (a kernel of its
+// own only on the fallback path).
 #include "common.cuh"
 #include "device_util.cuh"
 #include "umma.cuh"
@@ -109,14 +110,46 @@ struct ChunkCursor {
   }
 };
 
-// One CTA per SM, one working thread per CTA.  CTA b moves the contiguous chunk range
-// [n_chunks b / grid, n_chunks (b+1) / grid).
-__global__ void __launch_bounds__(32, 1) pack_rows_bulk_kernel(
+// The 4-byte columns of a packed micro-batch and what their gather needs of the sequence table.
+struct PackCols {
+  const int32_t* s_target; const float* s_old; const float* s_ref; const float* s_adv;
+  int32_t* o_target; float* o_old; float* o_ref; float* o_adv; int32_t* o_seq; int32_t* o_cu;
+  const int64_t* src_row; const int32_t* cu; const int32_t* idx;
+  int B, T;
+};
+// Items first, first + stride, ...: item i is packed token i (its columns and sequence id), and for
+// i <= B also cu_seqlens[i] and the advantage of sequence i.
+__device__ __forceinline__ void gather_cols(const PackCols& c, int64_t first, int64_t stride) {
+  for (int64_t i = first; i < c.T || i <= c.B; i += stride) {
+    if (i <= c.B) c.o_cu[i] = __ldg(c.cu + i);
+    if (i < c.B && c.o_adv) c.o_adv[i] = __ldg(c.s_adv + __ldg(c.idx + i));
+    if (i < c.T) {
+      const int j = find_seq(c.cu, c.B, (int)i);
+      const int64_t srow = __ldg(c.src_row + j) + (i - __ldg(c.cu + j));
+      if (c.o_target) c.o_target[i] = __ldg(c.s_target + srow);
+      if (c.o_old) c.o_old[i] = __ldg(c.s_old + srow);
+      if (c.o_ref) c.o_ref[i] = __ldg(c.s_ref + srow);
+      if (c.o_seq) c.o_seq[i] = j;
+    }
+  }
+}
+
+// One CTA per SM.  Its first thread moves the contiguous chunk range
+// [n_chunks b / grid, n_chunks (b+1) / grid) of the hidden column through the ring; warps 1 .. 7
+// meanwhile gather the 4-byte columns (grid-stride over the tokens), so that a micro-batch is packed
+// by one launch and the small columns cost no launch or drain of their own.
+constexpr int kBulkThreads = 256;
+__global__ void __launch_bounds__(kBulkThreads, 1) pack_rows_bulk_kernel(
     const uint8_t* __restrict__ src, uint8_t* __restrict__ dst, const int64_t* __restrict__ src_row,
     const int32_t* __restrict__ cu, const int32_t* __restrict__ chunk_cu, int B, int n_chunks,
-    int rows_per_chunk, int row_bytes, unsigned int* d_err) {
+    int rows_per_chunk, int row_bytes, unsigned int* d_err, const PackCols cols) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ int abort_flag;
+  if (threadIdx.x >= 32) {
+    constexpr int kColThreads = kBulkThreads - 32;
+    gather_cols(cols, (int64_t)blockIdx.x * kColThreads + (threadIdx.x - 32), (int64_t)gridDim.x * kColThreads);
+    return;
+  }
   if (threadIdx.x != 0) return;
   const uint32_t raw = umma::smem_u32(smem_raw);
   const uint32_t ring = (raw + 127u) & ~127u;
@@ -161,26 +194,8 @@ __global__ void __launch_bounds__(32, 1) pack_rows_bulk_kernel(
 }
 
 // One thread per packed token for the 4-byte columns; the first B threads also gather adv.
-__global__ void __launch_bounds__(256) pack_cols_kernel(
-    const int32_t* __restrict__ s_target, const float* __restrict__ s_old,
-    const float* __restrict__ s_ref, const float* __restrict__ s_adv,
-    int32_t* __restrict__ o_target, float* __restrict__ o_old, float* __restrict__ o_ref,
-    float* __restrict__ o_adv, int32_t* __restrict__ o_seq, int32_t* __restrict__ o_cu,
-    const int64_t* __restrict__ src_row, const int32_t* __restrict__ cu,
-    const int32_t* __restrict__ idx, int B, int T) {
-  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < T || i <= B; i += stride) {
-    if (i <= B) o_cu[i] = __ldg(cu + i);
-    if (i < B && o_adv) o_adv[i] = __ldg(s_adv + __ldg(idx + i));
-    if (i < T) {
-      const int j = find_seq(cu, B, (int)i);
-      const int64_t srow = __ldg(src_row + j) + (i - __ldg(cu + j));
-      if (o_target) o_target[i] = __ldg(s_target + srow);
-      if (o_old) o_old[i] = __ldg(s_old + srow);
-      if (o_ref) o_ref[i] = __ldg(s_ref + srow);
-      if (o_seq) o_seq[i] = j;
-    }
-  }
+__global__ void __launch_bounds__(256) pack_cols_kernel(const PackCols c) {
+  gather_cols(c, (int64_t)blockIdx.x * blockDim.x + threadIdx.x, (int64_t)gridDim.x * blockDim.x);
 }
 
 // The inverse for results: one thread per packed token writes up to four 4-byte columns to the
@@ -251,34 +266,32 @@ int pack_rows_per_chunk(int32_t d) {
 
 cudaError_t launch_pack(const af_store_view& st, const af_packed& out, const PackSeqTable& tab,
                         int32_t B, int64_t T, int sm_count, unsigned int* d_err, cudaStream_t s) {
+  const PackCols cols{st.target, st.old_logp, st.ref_logp, st.adv, out.target, out.old_logp, out.ref_logp,
+                      out.adv_seq, out.seq_id, out.cu_seqlens, tab.src_row, tab.cu, tab.idx, B, (int)T};
+  const int rpc = pack_rows_per_chunk(st.d);
+  if (T > 0 && out.hidden && rpc > 0 && tab.n_chunks > 0) {
+    // the usual case: one launch moves the hidden rows and gathers the small columns
+    static SmemAttrOnce once;
+    cudaError_t e = set_smem_once(once, pack_rows_bulk_kernel, kCopySmemBytes);
+    if (e != cudaSuccess) return e;
+    const int grid = tab.n_chunks < sm_count ? tab.n_chunks : sm_count;
+    pack_rows_bulk_kernel<<<grid, kBulkThreads, kCopySmemBytes, s>>>(
+        (const uint8_t*)st.hidden, (uint8_t*)out.hidden, tab.src_row, tab.cu, tab.chunk_cu, B,
+        tab.n_chunks, rpc, st.d * 2, d_err, cols);
+    return cudaGetLastError();
+  }
   {
     int64_t items = T > (int64_t)B + 1 ? T : (int64_t)B + 1;
     int blocks = (int)((items + 255) / 256);
     if (blocks > sm_count * 8) blocks = sm_count * 8;
-    pack_cols_kernel<<<blocks, 256, 0, s>>>(st.target, st.old_logp, st.ref_logp, st.adv,
-                                            out.target, out.old_logp, out.ref_logp, out.adv_seq,
-                                            out.seq_id, out.cu_seqlens, tab.src_row, tab.cu,
-                                            tab.idx, B, (int)T);
+    pack_cols_kernel<<<blocks, 256, 0, s>>>(cols);
   }
-  if (T > 0 && out.hidden) {
-    const int rpc = pack_rows_per_chunk(st.d);
-    if (rpc > 0 && tab.n_chunks > 0) {
-      {
-        static SmemAttrOnce once;
-        cudaError_t e = set_smem_once(once, pack_rows_bulk_kernel, kCopySmemBytes);
-        if (e != cudaSuccess) return e;
-      }
-      const int grid = tab.n_chunks < sm_count ? tab.n_chunks : sm_count;
-      pack_rows_bulk_kernel<<<grid, 32, kCopySmemBytes, s>>>(
-          (const uint8_t*)st.hidden, (uint8_t*)out.hidden, tab.src_row, tab.cu, tab.chunk_cu, B,
-          tab.n_chunks, rpc, st.d * 2, d_err);
-    } else {
-      const int words = st.d / 8;
-      int64_t blocks = (T + 7) / 8;  // 8 warps per block
-      if (blocks > sm_count * 8) blocks = sm_count * 8;
-      pack_rows_kernel<<<(int)blocks, 256, 0, s>>>((const uint4*)st.hidden, (uint4*)out.hidden,
-                                                   tab.src_row, tab.cu, B, (int)T, words);
-    }
+  if (T > 0 && out.hidden) {   // rows wider than a chunk
+    const int words = st.d / 8;
+    int64_t blocks = (T + 7) / 8;  // 8 warps per block
+    if (blocks > sm_count * 8) blocks = sm_count * 8;
+    pack_rows_kernel<<<(int)blocks, 256, 0, s>>>((const uint4*)st.hidden, (uint4*)out.hidden,
+                                                 tab.src_row, tab.cu, B, (int)T, words);
   }
   return cudaGetLastError();
 }
