@@ -40,7 +40,8 @@ from paper_2507_01663_b200 import workloads as wl  # noqa: E402
 
 METRIC = "scored tokens/sec (logprob+GRPO loss) at Qwen-7B head; % dense-BF16 peak"
 UNIT = "tokens/s"
-KERNELS_PER_STEP = 6  # advantage, pack table fetch, pack (rows by bulk copy + the 4-byte columns), fused LM-head GEMM, partial merge, loss
+KERNELS_PER_MICROBATCH = 4  # pack (rows by bulk copy + the 4-byte columns), fused LM-head GEMM, partial merge, loss
+PACK_INLINE_SEQS = 512      # beyond this many sequences a pack also launches the fetch of its sequence table
 # DRAM bytes per scored token of the fused LM-head kernel (dram__bytes_read of one ncu capture of the
 # CTA-pair kernel, row tiles dealt by die, two vocabulary ranges -- what the library picks at the
 # bench size -- on `--workload cfg2_mid --v-splits 2`: T = 62989, d = 3584, V = 152064; 8.306 and
@@ -333,8 +334,9 @@ class ScoringJob:
         self.e2e_logp_host = None
         self.ctx.reserve(cap_T, cap_B, w.d, w.V, with_backward=2 if w.backward else False)
         self.gemm_events, self.pack_events, self.bwd_events = [], [], []
-        per_mb = KERNELS_PER_STEP - 1 + (3 * -(-cap_T // BWD_TOKEN_BLOCK) if w.backward else 0)
-        self.launches_per_step = 1 + per_mb * len(self.mbs)
+        per_mb = KERNELS_PER_MICROBATCH + (3 * -(-cap_T // BWD_TOKEN_BLOCK) if w.backward else 0)
+        self.launches_per_step = (1 + per_mb * len(self.mbs)                      # 1: the advantage kernel
+                                  + sum(len(mb) > PACK_INLINE_SEQS for mb in self.mbs))
 
     def advantages(self, reward=None):
         """Group-normalised advantages of this rank's responses (into self.adv)."""
@@ -442,7 +444,7 @@ class ScoringJob:
         nbytes = 2.0 * t_mb * (2 * w.d + 12) + 8.0 * len(self.idx)
         gbs = nbytes / ms / 1e6
         out["pack_microbatch"] = {"tokens": t_mb, "bytes_per_token": 2 * (2 * w.d + 12), "ms": ms, "gbs": gbs,
-                                  "frac": gbs / peak_gbs, "where": "timed alone, 10 calls (2 kernels + metadata copy each)"}
+                                  "frac": gbs / peak_gbs, "where": "timed alone, 10 calls (one launch each up to 512 sequences, else table fetch + gather)"}
         # results written back by the same index list: 4 B read + 4 B written per token of one column
         col = torch.empty(int(self.off[-1]), device=dev)
         ms = avg_ms(lambda: c.unpack_microbatch(self.off, self.idx, [self.logp], [col]))

@@ -25,8 +25,9 @@
  *     call except af_pack_microbatch, af_unpack_microbatch, af_check_device_errors, af_reserve and
  *     af_destroy issues only kernel launches and asynchronous memsets on `stream`, so a sequence
  *     of them may be recorded into a CUDA graph and replayed on new contents of the same buffers.
- *     af_pack_microbatch and af_unpack_microbatch stage their index list through pinned host
- *     memory and wait on an event of their own; they cannot be recorded.  Nothing is claimed for
+ *     af_pack_microbatch and af_unpack_microbatch build a table from their host index list (and
+ *     for large batches stage it through pinned host memory, waiting on an event of their own);
+ *     they are not meant to be recorded.  Nothing is claimed for
  *     af_token_logprob_static.
  *   - Only compute capability 10.0 devices are accepted.  There is no CPU path.
  *   - Every entry point that enqueues work opens an NVTX range named after itself (a no-op unless
@@ -141,6 +142,12 @@ af_status af_check_device_errors(af_ctx* ctx, uint32_t* flags, void* stream);
  * capacities or T >= 2^31; AF_ERR_ALIGNMENT unless d % 8 == 0 and hidden pointers are 16-byte
  * aligned.  *T_out (host) receives the packed token count before the call returns.  B == 0 is
  * valid and writes cu_seqlens[0] = 0 only.
+ *
+ * The sequence table the kernels work from (first row, length and packed offset of each indexed
+ * sample) is built on the host in O(B).  For up to 512 sequences whose hidden rows are at most
+ * 32 KB it travels in the parameters of the one kernel that does the whole gather -- the call
+ * then waits for nothing and stages nothing; larger batches (or a call without the hidden
+ * column) stage it through pinned host memory, from where a small kernel brings it to the device.
  * ------------------------------------------------------------------------------------------- */
 typedef struct {
   int64_t n_samples;               /* N                                                       */

@@ -219,9 +219,38 @@ af_status af_reserve(af_ctx* c, int64_t max_T, int32_t max_B, int32_t d, int32_t
   return st;
 }
 
-// Builds the per-call sequence table ([src_row][cu][idx][chunk_cu]) in a pinned staging slot and
-// queues the kernel that brings it to the device.  *T receives the token count as soon as it is
-// known (also when the capacity check fails).
+// Fills the per-call sequence table from the host's offsets and index list: first store row, packed
+// offset, sample index and first bulk-copy chunk of every sequence.  *T receives the token count as
+// soon as it is known (also when the capacity check fails).
+static af_status fill_sequence_table(const int64_t* tok_offset_host, int64_t n_samples, const int32_t* idx_host,
+                                     int32_t B, int64_t rows_per_chunk, int64_t token_capacity, int64_t* h_src,
+                                     int32_t* h_cu, int32_t* h_idx, int32_t* h_chunk, int64_t* T_out,
+                                     int64_t* chunks_out) {
+  const int64_t rpc = rows_per_chunk;
+  int64_t T = 0, chunks = 0;
+  h_cu[0] = 0;
+  h_chunk[0] = 0;
+  for (int32_t j = 0; j < B; ++j) {
+    const int64_t i = idx_host[j];
+    if (i < 0 || i >= n_samples) return AF_ERR_INDEX;
+    const int64_t lo = tok_offset_host[i], hi = tok_offset_host[i + 1];
+    if (hi < lo) return AF_ERR_INVALID_ARG;
+    h_src[j] = lo;
+    h_idx[j] = (int32_t)i;
+    T += hi - lo;
+    if (T >= ((int64_t)1 << 31)) return AF_ERR_CAPACITY;
+    h_cu[j + 1] = (int32_t)T;
+    if (rpc > 0) chunks += (hi - lo + rpc - 1) / rpc;
+    h_chunk[j + 1] = (int32_t)chunks;   // chunks <= T + B < 2^31 + 2^31: checked below
+    if (chunks >= ((int64_t)1 << 31)) return AF_ERR_CAPACITY;
+  }
+  if (T_out) *T_out = T;
+  if (chunks_out) *chunks_out = chunks;
+  return T > token_capacity ? AF_ERR_CAPACITY : AF_OK;
+}
+
+// Builds the table ([src_row][cu][idx][chunk_cu]) in a pinned staging slot and queues the kernel
+// that brings it to the device.
 static af_status stage_sequence_table(af_ctx* c, const int64_t* tok_offset_host, int64_t n_samples,
                                       const int32_t* idx_host, int32_t B, int64_t rows_per_chunk,
                                       int64_t token_capacity, PackSeqTable* tab, int64_t* T_out, cudaStream_t s) {
@@ -242,32 +271,14 @@ static af_status stage_sequence_table(af_ctx* c, const int64_t* tok_offset_host,
 
   const size_t off_cu = ((size_t)B * 8 + 15) & ~(size_t)15;
   const size_t off_idx = off_cu + (((size_t)(B + 1) * 4 + 15) & ~(size_t)15);
-  char* hb = static_cast<char*>(c->pack_host[slot]);
-  int64_t* h_src = reinterpret_cast<int64_t*>(hb);
-  int32_t* h_cu = reinterpret_cast<int32_t*>(hb + off_cu);
-  int32_t* h_idx = reinterpret_cast<int32_t*>(hb + off_idx);
   const size_t off_chunk = off_idx + (((size_t)B * 4 + 15) & ~(size_t)15);
-  int32_t* h_chunk = reinterpret_cast<int32_t*>(hb + off_chunk);
-  const int64_t rpc = rows_per_chunk;
-  int64_t T = 0, chunks = 0;
-  h_cu[0] = 0;
-  h_chunk[0] = 0;
-  for (int32_t j = 0; j < B; ++j) {
-    const int64_t i = idx_host[j];
-    if (i < 0 || i >= n_samples) return AF_ERR_INDEX;
-    const int64_t lo = tok_offset_host[i], hi = tok_offset_host[i + 1];
-    if (hi < lo) return AF_ERR_INVALID_ARG;
-    h_src[j] = lo;
-    h_idx[j] = (int32_t)i;
-    T += hi - lo;
-    if (T >= ((int64_t)1 << 31)) return AF_ERR_CAPACITY;
-    h_cu[j + 1] = (int32_t)T;
-    if (rpc > 0) chunks += (hi - lo + rpc - 1) / rpc;
-    h_chunk[j + 1] = (int32_t)chunks;   // chunks <= T + B < 2^31 + 2^31: checked below
-    if (chunks >= ((int64_t)1 << 31)) return AF_ERR_CAPACITY;
-  }
-  if (T_out) *T_out = T;
-  if (T > token_capacity) return AF_ERR_CAPACITY;
+  char* hb = static_cast<char*>(c->pack_host[slot]);
+  int64_t chunks = 0;
+  st = fill_sequence_table(tok_offset_host, n_samples, idx_host, B, rows_per_chunk, token_capacity,
+                           reinterpret_cast<int64_t*>(hb), reinterpret_cast<int32_t*>(hb + off_cu),
+                           reinterpret_cast<int32_t*>(hb + off_idx), reinterpret_cast<int32_t*>(hb + off_chunk), T_out,
+                           &chunks);
+  if (st != AF_OK) return st;
 
   char* db = static_cast<char*>(c->pack_meta.p);
   if (launch_pack_meta_fetch(db, hb, bytes, s) != cudaSuccess) return AF_ERR_CUDA;
@@ -299,11 +310,24 @@ af_status af_pack_microbatch(af_ctx* c, const af_store_view* store, const int32_
   if (B > out->seq_capacity) return AF_ERR_CAPACITY;
   DeviceGuard guard(c->device);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  PackSeqTable tab{};
+  const int rpc = store->hidden ? pack_rows_per_chunk(store->d) : 0;
   int64_t T = 0;
-  const af_status st = stage_sequence_table(c, store->tok_offset_host, store->n_samples, idx_host, B,
-                                            store->hidden ? pack_rows_per_chunk(store->d) : 0, out->token_capacity,
-                                            &tab, &T, s);
+  if (B >= 1 && B <= kPackInlineSeqs && rpc > 0) {
+    // few sequences: the table travels in the kernel's parameters, one launch does everything
+    PackTableInline inl;
+    int64_t chunks = 0;
+    const af_status st = fill_sequence_table(store->tok_offset_host, store->n_samples, idx_host, B, rpc,
+                                             out->token_capacity, inl.src_row, inl.cu, inl.idx, inl.chunk_cu, &T,
+                                             &chunks);
+    if (T_out) *T_out = T;
+    if (st != AF_OK) return st;
+    if (T > 0)
+      return launch_pack_inline(*store, *out, inl, B, T, c->sm_count, c->d_err, s) == cudaSuccess ? AF_OK : AF_ERR_CUDA;
+    // only empty sequences: the staged path below writes cu_seqlens and the advantages
+  }
+  PackSeqTable tab{};
+  const af_status st = stage_sequence_table(c, store->tok_offset_host, store->n_samples, idx_host, B, rpc,
+                                            out->token_capacity, &tab, &T, s);
   if (T_out) *T_out = T;
   if (st != AF_OK) return st;
   return launch_pack(*store, *out, tab, B, T, c->sm_count, c->d_err, s) == cudaSuccess ? AF_OK : AF_ERR_CUDA;

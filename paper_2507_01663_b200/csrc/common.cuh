@@ -127,6 +127,19 @@ cudaError_t launch_unpack(const af_write_cols& cols, const PackSeqTable& tab, in
                           cudaStream_t s);
 cudaError_t launch_pack(const af_store_view& st, const af_packed& out, const PackSeqTable& tab,
                         int32_t B, int64_t T, int sm_count, unsigned int* d_err, cudaStream_t s);
+// The same table for a micro-batch of at most kPackInlineSeqs sequences, small enough to travel in the
+// kernel's parameters: no staging buffer, no fetch kernel, nothing for the host to wait on.
+constexpr int kPackInlineSeqs = 512;
+struct PackTableInline {
+  int64_t src_row[kPackInlineSeqs];
+  int32_t cu[kPackInlineSeqs + 1];
+  int32_t idx[kPackInlineSeqs];
+  int32_t chunk_cu[kPackInlineSeqs + 1];
+};
+// Packs with the table passed by value.  Needs hidden rows that fit a bulk-copy chunk, T > 0 and
+// 1 <= B <= kPackInlineSeqs (the caller checks).
+cudaError_t launch_pack_inline(const af_store_view& st, const af_packed& out, const PackTableInline& tab,
+                               int32_t B, int64_t T, int sm_count, unsigned int* d_err, cudaStream_t s);
 
 cudaError_t launch_advantage(const float* reward, int64_t N, int32_t n_groups, float eps_adv, int32_t ddof,
                              float* adv, int sm_count, cudaStream_t s);                  // contiguous groups

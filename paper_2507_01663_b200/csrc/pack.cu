@@ -11,6 +11,8 @@
 // than a chunk fall back to a warp-per-row copy with 128-bit loads and stores.  The 4-byte
 // columns are gathered one thread per token, by the other warps of the same CTAs (a kernel of its
 // own only on the fallback path).
+#include <cstring>
+
 #include "common.cuh"
 #include "device_util.cuh"
 #include "umma.cuh"
@@ -77,28 +79,33 @@ __device__ __forceinline__ void bulk_wait_read() {   // at most kPending stores 
 }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
+// Sequence of a packed token (see find_seq) by plain loads: the table may sit in shared memory.
+__device__ __forceinline__ int seq_of(const int32_t* cu, int B, int t) {
+  int lo = 0, hi = B;
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (cu[mid] <= t) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
 // Walks the chunks of consecutive sequences: sequence j owns chunks chunk_cu[j] .. chunk_cu[j+1]-1,
-// each `rows_per_chunk` rows except the last one of the sequence.
+// each `rows_per_chunk` rows except the last one of the sequence.  (Plain loads: global or shared table.)
 struct ChunkCursor {
   const int64_t* src_row; const int32_t* cu; const int32_t* chunk_cu;
   int B, rows_per_chunk;
   int j, first_chunk, next_first, dst_row0, len;
   int64_t src_row0;
   __device__ void seek(int c) {   // largest j with chunk_cu[j] <= c (sequences without rows own no chunk)
-    int lo = 0, hi = B;
-    while (hi - lo > 1) {
-      const int mid = (lo + hi) >> 1;
-      if (__ldg(chunk_cu + mid) <= c) lo = mid; else hi = mid;
-    }
-    j = lo;
+    j = seq_of(chunk_cu, B, c);
     load();
   }
   __device__ void load() {
-    first_chunk = __ldg(chunk_cu + j);
-    next_first = __ldg(chunk_cu + j + 1);
-    dst_row0 = __ldg(cu + j);
-    len = __ldg(cu + j + 1) - dst_row0;
-    src_row0 = __ldg(src_row + j);
+    first_chunk = chunk_cu[j];
+    next_first = chunk_cu[j + 1];
+    dst_row0 = cu[j];
+    len = cu[j + 1] - dst_row0;
+    src_row0 = src_row[j];
   }
   // source row, packed row and row count of chunk c (c never decreases between calls)
   __device__ void at(int c, int64_t& srow, int64_t& drow, int& rows) {
@@ -121,11 +128,11 @@ struct PackCols {
 // i <= B also cu_seqlens[i] and the advantage of sequence i.
 __device__ __forceinline__ void gather_cols(const PackCols& c, int64_t first, int64_t stride) {
   for (int64_t i = first; i < c.T || i <= c.B; i += stride) {
-    if (i <= c.B) c.o_cu[i] = __ldg(c.cu + i);
-    if (i < c.B && c.o_adv) c.o_adv[i] = __ldg(c.s_adv + __ldg(c.idx + i));
+    if (i <= c.B) c.o_cu[i] = c.cu[i];
+    if (i < c.B && c.o_adv) c.o_adv[i] = __ldg(c.s_adv + c.idx[i]);
     if (i < c.T) {
-      const int j = find_seq(c.cu, c.B, (int)i);
-      const int64_t srow = __ldg(c.src_row + j) + (i - __ldg(c.cu + j));
+      const int j = seq_of(c.cu, c.B, (int)i);
+      const int64_t srow = c.src_row[j] + (i - c.cu[j]);
       if (c.o_target) c.o_target[i] = __ldg(c.s_target + srow);
       if (c.o_old) c.o_old[i] = __ldg(c.s_old + srow);
       if (c.o_ref) c.o_ref[i] = __ldg(c.s_ref + srow);
@@ -139,12 +146,10 @@ __device__ __forceinline__ void gather_cols(const PackCols& c, int64_t first, in
 // meanwhile gather the 4-byte columns (grid-stride over the tokens), so that a micro-batch is packed
 // by one launch and the small columns cost no launch or drain of their own.
 constexpr int kBulkThreads = 256;
-__global__ void __launch_bounds__(kBulkThreads, 1) pack_rows_bulk_kernel(
-    const uint8_t* __restrict__ src, uint8_t* __restrict__ dst, const int64_t* __restrict__ src_row,
-    const int32_t* __restrict__ cu, const int32_t* __restrict__ chunk_cu, int B, int n_chunks,
-    int rows_per_chunk, int row_bytes, unsigned int* d_err, const PackCols cols) {
-  extern __shared__ uint8_t smem_raw[];
-  __shared__ int abort_flag;
+__device__ __forceinline__ void pack_bulk_body(
+    const uint8_t* __restrict__ src, uint8_t* __restrict__ dst, const int64_t* src_row, const int32_t* cu,
+    const int32_t* chunk_cu, int B, int n_chunks, int rows_per_chunk, int row_bytes, unsigned int* d_err,
+    const PackCols& cols, uint8_t* smem_raw, int* abort_flag) {
   if (threadIdx.x >= 32) {
     constexpr int kColThreads = kBulkThreads - 32;
     gather_cols(cols, (int64_t)blockIdx.x * kColThreads + (threadIdx.x - 32), (int64_t)gridDim.x * kColThreads);
@@ -154,7 +159,7 @@ __global__ void __launch_bounds__(kBulkThreads, 1) pack_rows_bulk_kernel(
   const uint32_t raw = umma::smem_u32(smem_raw);
   const uint32_t ring = (raw + 127u) & ~127u;
   const uint32_t bars = ring + kCopyStages * kChunkBytes;
-  abort_flag = 0;
+  *abort_flag = 0;
   for (int s = 0; s < kCopyStages; ++s) umma::mbar_init(bars + 8u * s, 1);
   umma::fence_mbar_init();
 
@@ -178,7 +183,7 @@ __global__ void __launch_bounds__(kBulkThreads, 1) pack_rows_bulk_kernel(
   for (int i = 0; i < kCopyAhead && i < n; ++i) issue_load(i);
   for (int i = 0; i < n; ++i) {
     const int st = i % kCopyStages;
-    if (!umma::mbar_wait(bars + 8u * st, (uint32_t)(i / kCopyStages) & 1u, &abort_flag)) break;
+    if (!umma::mbar_wait(bars + 8u * st, (uint32_t)(i / kCopyStages) & 1u, abort_flag)) break;
     int64_t srow, drow; int rows;
     sc.at(c_begin + i, srow, drow, rows);
     bulk_store(dst + drow * row_bytes, ring + st * kChunkBytes, (uint32_t)rows * (uint32_t)row_bytes);
@@ -190,7 +195,50 @@ __global__ void __launch_bounds__(kBulkThreads, 1) pack_rows_bulk_kernel(
     }
   }
   bulk_wait_all();
-  if (abort_flag) atomicOr(d_err, umma::kWatchdogBit);
+  if (*abort_flag) atomicOr(d_err, umma::kWatchdogBit);
+}
+
+__global__ void __launch_bounds__(kBulkThreads, 1) pack_rows_bulk_kernel(
+    const uint8_t* __restrict__ src, uint8_t* __restrict__ dst, const int64_t* __restrict__ src_row,
+    const int32_t* __restrict__ cu, const int32_t* __restrict__ chunk_cu, int B, int n_chunks,
+    int rows_per_chunk, int row_bytes, unsigned int* d_err, const PackCols cols) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ int abort_flag;
+  pack_bulk_body(src, dst, src_row, cu, chunk_cu, B, n_chunks, rows_per_chunk, row_bytes, d_err, cols, smem_raw,
+                 &abort_flag);
+}
+
+// The same with the sequence table in the kernel's parameters (B <= kSeqs): every CTA copies the B
+// entries it needs into shared memory and works from there.  Two sizes: parameters beyond 4 KB make
+// a launch noticeably slower on the host, so small batches use a table that stays below that.
+template <int kSeqs>
+struct InlineTable {
+  int64_t src_row[kSeqs];
+  int32_t cu[kSeqs + 1];
+  int32_t idx[kSeqs];
+  int32_t chunk_cu[kSeqs + 1];
+};
+constexpr int kSmallInlineSeqs = 128;
+static_assert(sizeof(InlineTable<kSmallInlineSeqs>) + 256 <= 4096, "the small table keeps the launch within 4 KB of parameters");
+
+template <int kSeqs>
+__global__ void __launch_bounds__(kBulkThreads, 1) pack_rows_bulk_inline_kernel(
+    const uint8_t* __restrict__ src, uint8_t* __restrict__ dst, const __grid_constant__ InlineTable<kSeqs> tab, int B,
+    int n_chunks, int rows_per_chunk, int row_bytes, unsigned int* d_err, const PackCols cols_in) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ int abort_flag;
+  __shared__ int64_t s_src_row[kSeqs];
+  __shared__ int32_t s_cu[kSeqs + 1], s_idx[kSeqs], s_chunk_cu[kSeqs + 1];
+  for (int i = threadIdx.x; i <= B; i += kBulkThreads) {
+    s_cu[i] = tab.cu[i];
+    s_chunk_cu[i] = tab.chunk_cu[i];
+    if (i < B) { s_src_row[i] = tab.src_row[i]; s_idx[i] = tab.idx[i]; }
+  }
+  __syncthreads();
+  PackCols cols = cols_in;
+  cols.src_row = s_src_row; cols.cu = s_cu; cols.idx = s_idx;
+  pack_bulk_body(src, dst, s_src_row, s_cu, s_chunk_cu, B, n_chunks, rows_per_chunk, row_bytes, d_err, cols,
+                 smem_raw, &abort_flag);
 }
 
 // One thread per packed token for the 4-byte columns; the first B threads also gather adv.
@@ -294,6 +342,35 @@ cudaError_t launch_pack(const af_store_view& st, const af_packed& out, const Pac
                                                  tab.src_row, tab.cu, B, (int)T, words);
   }
   return cudaGetLastError();
+}
+
+namespace {
+template <int kSeqs>
+cudaError_t launch_inline(const af_store_view& st, const af_packed& out, const PackTableInline& full, int32_t B,
+                          const PackCols& cols, int sm_count, unsigned int* d_err, cudaStream_t s) {
+  static SmemAttrOnce once;
+  cudaError_t e = set_smem_once(once, pack_rows_bulk_inline_kernel<kSeqs>, kCopySmemBytes);
+  if (e != cudaSuccess) return e;
+  InlineTable<kSeqs> tab;
+  std::memcpy(tab.src_row, full.src_row, sizeof(int64_t) * B);
+  std::memcpy(tab.cu, full.cu, sizeof(int32_t) * (B + 1));
+  std::memcpy(tab.idx, full.idx, sizeof(int32_t) * B);
+  std::memcpy(tab.chunk_cu, full.chunk_cu, sizeof(int32_t) * (B + 1));
+  const int n_chunks = full.chunk_cu[B];
+  const int grid = n_chunks < sm_count ? n_chunks : sm_count;
+  pack_rows_bulk_inline_kernel<kSeqs><<<grid, kBulkThreads, kCopySmemBytes, s>>>(
+      (const uint8_t*)st.hidden, (uint8_t*)out.hidden, tab, B, n_chunks, pack_rows_per_chunk(st.d), st.d * 2, d_err,
+      cols);
+  return cudaGetLastError();
+}
+}  // namespace
+
+cudaError_t launch_pack_inline(const af_store_view& st, const af_packed& out, const PackTableInline& tab,
+                               int32_t B, int64_t T, int sm_count, unsigned int* d_err, cudaStream_t s) {
+  const PackCols cols{st.target, st.old_logp, st.ref_logp, st.adv, out.target, out.old_logp, out.ref_logp,
+                      out.adv_seq, out.seq_id, out.cu_seqlens, nullptr, nullptr, nullptr, B, (int)T};
+  return B <= kSmallInlineSeqs ? launch_inline<kSmallInlineSeqs>(st, out, tab, B, cols, sm_count, d_err, s)
+                               : launch_inline<kPackInlineSeqs>(st, out, tab, B, cols, sm_count, d_err, s);
 }
 
 }  // namespace af

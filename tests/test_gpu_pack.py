@@ -110,6 +110,61 @@ def test_pack_empty_batch_and_zero_length_samples(ctx):
     assert np.array_equal(wl.bf16_bits(o["hidden"][:T]), ref["hidden"])
 
 
+@pytest.mark.parametrize("B", [1, 127, 128, 129, 511, 512, 513, 1500])
+def test_pack_around_the_inline_table_limit(ctx, B):
+    """Up to 512 sequences the table travels with the launch, beyond that through the staged device
+    copy: both sides of the limit, with duplicates, empty samples and every column, bit for bit."""
+    dev = device()
+    rng = np.random.default_rng(B)
+    lengths = rng.integers(0, 10, size=700).astype(np.int64)
+    off = np.concatenate([[0], np.cumsum(lengths)])
+    n_tok, d = int(off[-1]), 64
+    H = wl._normal_matrix(B, wl.S_HIDDEN, n_tok, d, 1.0, dev)
+    tgt = torch.arange(n_tok, dtype=torch.int32, device=dev)
+    old = wl.normal01(B, wl.S_OLD, 0, n_tok, dev)
+    adv = wl.normal01(B, wl.S_MISC, 0, 700, dev)
+    idx = rng.integers(0, 700, size=B).astype(np.int32)
+    T_cap = int(lengths[idx].sum())
+    o = {"cu_seqlens": torch.full((B + 2,), -7, dtype=torch.int32, device=dev),
+         "hidden": torch.zeros(T_cap + 2, d, dtype=torch.bfloat16, device=dev),
+         "target": torch.full((T_cap + 2,), -7, dtype=torch.int32, device=dev),
+         "old_logp": torch.zeros(T_cap + 2, device=dev),
+         "adv_seq": torch.zeros(B, device=dev),
+         "seq_id": torch.full((T_cap + 2,), -7, dtype=torch.int32, device=dev)}
+    T = ctx.pack_microbatch({"tok_offset_host": off, "d": d, "hidden": H, "target": tgt, "old_logp": old, "adv": adv},
+                            idx, o)
+    torch.cuda.synchronize()
+    ref = O.pack_microbatch_ref(off, idx, {"hidden": wl.bf16_bits(H), "target": np_of(tgt), "old_logp": np_of(old)},
+                                np_of(adv))
+    assert T == T_cap
+    assert np.array_equal(np_of(o["cu_seqlens"])[:B + 1], ref["cu_seqlens"]) and int(o["cu_seqlens"][B + 1]) == -7
+    assert np.array_equal(np_of(o["target"])[:T], ref["target"]) and np.all(np_of(o["target"])[T:] == -7)
+    assert np.array_equal(np_of(o["seq_id"])[:T], ref["seq_id"]) and np.all(np_of(o["seq_id"])[T:] == -7)
+    assert np_of(o["old_logp"])[:T].tobytes() == ref["old_logp"].tobytes()
+    assert np_of(o["adv_seq"]).tobytes() == ref["adv_seq"].astype(np.float32).tobytes()
+    assert np.array_equal(wl.bf16_bits(o["hidden"][:T]), ref["hidden"])
+    assert not bool(o["hidden"][T:].any())
+    assert ctx.check_device_errors() == 0
+
+
+def test_pack_of_empty_samples_only(ctx):
+    """Sequences without tokens still get their cu_seqlens entries and advantages."""
+    dev = device()
+    off = np.array([0, 0, 4, 4, 4], np.int64)
+    d = 32
+    H = wl._normal_matrix(3, wl.S_HIDDEN, 4, d, 1.0, dev)
+    adv = torch.tensor([1.5, -2.0, 0.25, 8.0], device=dev)
+    idx = np.array([0, 2, 3, 0], np.int32)
+    o = {"cu_seqlens": torch.full((6,), -7, dtype=torch.int32, device=dev),
+         "hidden": torch.zeros(4, d, dtype=torch.bfloat16, device=dev), "adv_seq": torch.zeros(4, device=dev)}
+    T = ctx.pack_microbatch({"tok_offset_host": off, "d": d, "hidden": H, "adv": adv}, idx, o)
+    torch.cuda.synchronize()
+    assert T == 0
+    assert np_of(o["cu_seqlens"]).tolist() == [0, 0, 0, 0, 0, -7]
+    assert np_of(o["adv_seq"]).tolist() == [1.5, 0.25, 8.0, 1.5]
+    assert not bool(o["hidden"].any()) and ctx.check_device_errors() == 0
+
+
 def test_pack_host_errors(ctx):
     from paper_2507_01663_b200.binding import AfError
     dev = device()
