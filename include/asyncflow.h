@@ -429,6 +429,39 @@ af_status af_unpack_microbatch(af_ctx* ctx, const int64_t* tok_offset_host, int6
 
 
 /* ---------------------------------------------------------------------------------------------
+ * af_plan_token_logprob / af_plan_units -- how af_token_logprob cuts its work (host calls, no GPU).
+ *
+ * The paper leaves kernel design to the platform; this is the library's own work decomposition,
+ * exposed so that it can be inspected and checked without a device.  The fused LM-head kernel
+ * processes units: a unit is one row tile of tokens (256 rows for CTA pairs, 128 for single CTAs)
+ * times one of v_splits contiguous ranges of 256-column vocabulary tiles; unit u is row tile
+ * u / v_splits, range u % v_splits.  `workers` persistent CTA pairs (or CTAs) share the units.
+ * Dealt plainly, worker r takes units r, r + workers, ...  Dealt by die (die0_workers > 0), the first
+ * die0_workers workers share the units of the first die0_row_tiles row tiles among themselves and
+ * the others the rest, so that a row tile's hidden-state panel is cached in one half of L2 only.
+ *
+ * af_plan_token_logprob fills *plan for a batch of T >= 1 tokens at head shape (d, V) on a part
+ * with sm_count SMs of which die0_sms share a die (0: unknown, deal plainly); v_splits and
+ * gemm_variant as in af_set_tuning (0 = the library's choice).  af_plan_units gives the units of
+ * worker `rank` in [0, workers): *first, *first + *stride, ... below *end.  Over all ranks these
+ * lists hold every unit in [0, m_tiles * v_splits) exactly once.  AF_ERR_INVALID_ARG for null
+ * pointers, sizes below 1, die0_sms outside [0, sm_count] or a rank outside [0, workers).
+ * ------------------------------------------------------------------------------------------- */
+typedef struct {
+  int32_t m_tiles;         /* row tiles of the batch                                          */
+  int32_t n_tiles;         /* vocabulary tiles of 256 columns                                 */
+  int32_t v_splits;        /* vocabulary ranges per row tile                                  */
+  int32_t workers;         /* CTA pairs (or CTAs) the launch starts                           */
+  int32_t die0_workers;    /* > 0: dealt by die, workers running on the first die             */
+  int32_t die0_row_tiles;  /* row tiles whose units the first die's workers share             */
+} af_gemm_plan;
+
+af_status af_plan_token_logprob(int64_t T, int32_t d, int32_t V, int32_t sm_count, int32_t die0_sms,
+                                int32_t v_splits, int32_t gemm_variant, af_gemm_plan* plan);
+af_status af_plan_units(const af_gemm_plan* plan, int32_t rank, int32_t* first, int32_t* stride,
+                        int32_t* end);
+
+/* ---------------------------------------------------------------------------------------------
  * af_balance_partitions -- token-balanced split of a batch over k groups (host call, no GPU).
  *
  * The controller's load balancing (Section 4.4, last paragraph): a one-dimensional bin-packing

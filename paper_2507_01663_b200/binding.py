@@ -27,7 +27,8 @@ EXPORTS = ["af_create", "af_destroy", "af_status_string", "af_reserve", "af_work
            "af_set_tuning", "af_check_device_errors", "af_pack_microbatch", "af_token_logprob",
            "af_grpo_advantage", "af_policy_loss", "af_policy_loss_backward", "af_token_logprob_static",
            "af_controller_put", "af_controller_get", "af_controller_clear", "af_balance_partitions",
-           "af_token_logprob_shard", "af_merge_logprob_shards", "af_policy_update", "af_unpack_microbatch", "af_policy_loss_backward_shard", "af_set_dw_ready_event", "af_die_split", "af_selftest_bounded_wait"]
+           "af_token_logprob_shard", "af_merge_logprob_shards", "af_policy_update", "af_unpack_microbatch", "af_policy_loss_backward_shard", "af_set_dw_ready_event", "af_die_split", "af_selftest_bounded_wait",
+           "af_plan_token_logprob", "af_plan_units"]
 MAX_WRITE_COLS = 4
 
 
@@ -359,6 +360,29 @@ class Context:
         tv = self._table(table)
         _check(self.lib.af_controller_clear(self.handle, C.byref(tv), column_bits, task_bits, _stream(stream)),
                "af_controller_clear")
+
+
+class GemmPlan(C.Structure):
+    """Mirror of ``af_gemm_plan``."""
+    _fields_ = [("m_tiles", C.c_int32), ("n_tiles", C.c_int32), ("v_splits", C.c_int32), ("workers", C.c_int32),
+                ("die0_workers", C.c_int32), ("die0_row_tiles", C.c_int32)]
+
+
+def plan_token_logprob(T: int, d: int, V: int, sm_count: int, die0_sms: int = 0, v_splits: int = 0,
+                       gemm_variant: int = 0) -> GemmPlan:
+    """``af_plan_token_logprob`` (host): the work decomposition of a scoring call."""
+    plan = GemmPlan()
+    _check(load_library().af_plan_token_logprob(C.c_int64(T), d, V, sm_count, die0_sms, v_splits, gemm_variant,
+                                                C.byref(plan)), "af_plan_token_logprob")
+    return plan
+
+
+def plan_units(plan: GemmPlan, rank: int) -> range:
+    """``af_plan_units`` (host): the units worker ``rank`` processes."""
+    first, stride, end = C.c_int32(), C.c_int32(), C.c_int32()
+    _check(load_library().af_plan_units(C.byref(plan), rank, C.byref(first), C.byref(stride), C.byref(end)),
+           "af_plan_units")
+    return range(first.value, end.value, stride.value)
 
 
 def balance_partitions(length, k: int, equal_size: bool):

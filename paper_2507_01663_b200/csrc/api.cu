@@ -154,6 +154,28 @@ af_status af_set_tuning(af_ctx* c, int32_t v_splits, int32_t bwd_token_block, in
   return AF_OK;
 }
 
+af_status af_plan_token_logprob(int64_t T, int32_t d, int32_t V, int32_t sm_count, int32_t die0_sms,
+                                int32_t v_splits, int32_t gemm_variant, af_gemm_plan* plan) {
+  if (!plan || T < 1 || d < 1 || V < 1 || sm_count < 1 || die0_sms < 0 || die0_sms > sm_count || v_splits < 0 ||
+      gemm_variant < 0 || gemm_variant > 3)
+    return AF_ERR_INVALID_ARG;
+  if (T >= ((int64_t)1 << 31)) return AF_ERR_SHAPE;
+  const bool pair = gemm_variant != 1 && sm_count >= 2;          // as af_set_tuning reads the variant
+  plan_token_logprob(T, d, V, sm_count, die0_sms, v_splits, pair, gemm_variant != 2, plan);
+  return AF_OK;
+}
+
+af_status af_plan_units(const af_gemm_plan* plan, int32_t rank, int32_t* first, int32_t* stride, int32_t* end) {
+  if (!plan || !first || !stride || !end || plan->workers < 1 || rank < 0 || rank >= plan->workers ||
+      plan->m_tiles < 1 || plan->v_splits < 1 || plan->die0_workers < 0 || (plan->die0_workers > 0 && plan->die0_workers >= plan->workers) ||
+      plan->die0_row_tiles < 0 || plan->die0_row_tiles > plan->m_tiles)
+    return AF_ERR_INVALID_ARG;
+  int f = 0, st = 1, e = 0;
+  plan_units(*plan, rank, &f, &st, &e);
+  *first = f; *stride = st; *end = e;
+  return AF_OK;
+}
+
 af_status af_set_dw_ready_event(af_ctx* c, void* event) {
   if (!c) return AF_ERR_INVALID_ARG;
   c->dw_ready = static_cast<cudaEvent_t>(event);

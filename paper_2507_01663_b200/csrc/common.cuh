@@ -165,6 +165,10 @@ cudaError_t launch_controller_get(const af_controller_view& v, uint32_t mask, ui
                                   int sm_count, cudaStream_t s);
 
 int logprob_pick_splits(int64_t T, int32_t d, int32_t V, int sm_count, bool pair, int requested, int die0_pairs);
+// The work decomposition launch_token_logprob would use (no device needed); see af_plan_token_logprob.
+void plan_token_logprob(int64_t T, int32_t d, int32_t V, int sm_count, int die0_sms, int requested_splits, bool pair,
+                        bool die_aware, af_gemm_plan* plan);
+void plan_units(const af_gemm_plan& plan, int rank, int* first, int* stride, int* end);
 af_status launch_token_logprob(af_ctx* ctx, const void* hidden, const void* W,
                                const int32_t* target, int64_t T, int32_t d, int32_t V,
                                float* logp, float* entropy, float* lse, cudaStream_t s);

@@ -44,6 +44,31 @@ inline int die_split_rows(int64_t m_tiles, int64_t splits, int64_t pairs, int64_
   return best_rows > 0 && best_rounds <= plain_rounds ? (int)best_rows : 0;
 }
 
+// Tiles, vocabulary ranges and K blocks of C[M,N] = sum_k A(m,k) B(n,k); `splits` <= 0 means one unit
+// per B tile.  Dealt plainly until deal_by_die says otherwise.
+inline umma::GemmShape gemm_shape(uint64_t M, uint64_t N, uint64_t K, int splits, bool pair) {
+  const int tile_rows = pair ? umma::kPairBM : umma::kBM;
+  umma::GemmShape g;
+  g.M = (int)M; g.N = (int)N; g.K = (int)K;
+  g.m_tiles = (int)((M + tile_rows - 1) / tile_rows);
+  g.n_tiles = (int)((N + umma::kBN - 1) / umma::kBN);
+  g.splits = splits > 0 && splits < g.n_tiles ? splits : g.n_tiles;
+  g.k_blocks = (int)((K + umma::kBK - 1) / umma::kBK);
+  g.die0_pairs = 0;
+  g.die0_rows = 0;
+  return g;
+}
+// Die-aware dealing of a pair launch: only when every SM pair gets a CTA pair and it costs no extra
+// round of units.  Fills g.die0_pairs / g.die0_rows and returns true if so.
+inline bool deal_by_die(umma::GemmShape& g, int pairs, int die0_pairs) {
+  const int64_t units = (int64_t)g.m_tiles * g.splits;
+  const int rows0 = die0_pairs > 0 && units >= pairs ? die_split_rows(g.m_tiles, g.splits, pairs, die0_pairs) : 0;
+  if (rows0 <= 0) return false;
+  g.die0_pairs = die0_pairs;
+  g.die0_rows = rows0;
+  return true;
+}
+
 inline af_status encode_operand(const GemmEnv& env, CUtensorMap* map, const Operand& op, uint32_t box_rows) {
   TmapCache::Entry* slot = nullptr;
   if (env.cache) {
@@ -81,15 +106,7 @@ af_status run_gemm(const GemmEnv& env, const Operand& A, const Operand& B, int s
   if (st != AF_OK) return st;
   const uint64_t M = kAMN ? A.cols : A.rows, K = kAMN ? A.rows : A.cols;
   const uint64_t N = kBMN ? B.cols : B.rows;
-  const int tile_rows = env.pair ? umma::kPairBM : umma::kBM;
-  umma::GemmShape g;
-  g.M = (int)M; g.N = (int)N; g.K = (int)K;
-  g.m_tiles = (int)((M + tile_rows - 1) / tile_rows);
-  g.n_tiles = (int)((N + umma::kBN - 1) / umma::kBN);
-  g.splits = splits > 0 && splits < g.n_tiles ? splits : g.n_tiles;
-  g.k_blocks = (int)((K + umma::kBK - 1) / umma::kBK);
-  g.die0_pairs = 0;
-  g.die0_rows = 0;
+  umma::GemmShape g = gemm_shape(M, N, K, splits, env.pair);
   const int64_t units = (int64_t)g.m_tiles * g.splits;
   if (env.pair) {
     constexpr int smem = E::kStaged ? umma::kPairSmemBytesStaged : umma::kPairSmemBytes;
@@ -98,11 +115,7 @@ af_status run_gemm(const GemmEnv& env, const Operand& A, const Operand& B, int s
     const int pairs = env.sm_count / 2;
     const int grid = 2 * (int)(units < pairs ? units : pairs);
     unsigned int* clock = env.tile_clock;
-    // die-aware dealing when every SM pair gets a CTA pair and it costs no extra round of units
-    const int rows0 = env.die0_pairs > 0 && env.die_of_sm && clock && units >= pairs
-                          ? die_split_rows(g.m_tiles, g.splits, pairs, env.die0_pairs) : 0;
-    const bool by_die = rows0 > 0;
-    if (by_die) { g.die0_pairs = env.die0_pairs; g.die0_rows = rows0; }
+    const bool by_die = env.die_of_sm && clock && deal_by_die(g, pairs, env.die0_pairs);
     if (clock && cudaMemsetAsync(clock, 0, (by_die ? 3 : 1) * sizeof(unsigned int), s) != cudaSuccess) return AF_ERR_CUDA;
     umma::gemm_pair_kernel<E, kAMN, kBMN><<<grid, umma::kThreads, smem, s>>>(ta, tb, g, ep, env.d_err, clock,
                                                                              by_die ? clock + 1 : nullptr, env.die_of_sm);

@@ -167,6 +167,34 @@ int logprob_pick_splits(int64_t T, int32_t d, int32_t V, int sm_count, bool pair
   return best;
 }
 
+void plan_token_logprob(int64_t T, int32_t d, int32_t V, int sm_count, int die0_sms, int requested_splits, bool pair,
+                        bool die_aware, af_gemm_plan* plan) {
+  const int die0_pairs = pair && die_aware && die0_sms > 0 ? die0_sms / 2 : 0;
+  const int S = logprob_pick_splits(T, d, V, sm_count, pair, requested_splits, die0_pairs);
+  umma::GemmShape g = gemm_shape((uint64_t)T, (uint64_t)V, (uint64_t)d, S, pair);
+  const int64_t units = (int64_t)g.m_tiles * g.splits;
+  const int64_t slots = pair ? sm_count / 2 : sm_count;
+  if (pair) deal_by_die(g, (int)slots, die0_pairs);
+  plan->m_tiles = g.m_tiles;
+  plan->n_tiles = g.n_tiles;
+  plan->v_splits = g.splits;
+  plan->workers = (int32_t)(units < slots ? units : slots);
+  plan->die0_workers = g.die0_pairs;
+  plan->die0_row_tiles = g.die0_rows;
+}
+
+void plan_units(const af_gemm_plan& plan, int rank, int* first, int* stride, int* end) {
+  umma::GemmShape g{};
+  g.m_tiles = plan.m_tiles;
+  g.splits = plan.v_splits;
+  g.die0_pairs = plan.die0_workers;
+  g.die0_rows = plan.die0_row_tiles;
+  const umma::PairWork w = umma::pair_work(g, rank, plan.workers);   // plain dealing when die0_pairs is 0
+  *first = w.base_unit + w.first;
+  *stride = w.step;
+  *end = w.base_unit + w.end;
+}
+
 af_status launch_token_logprob_z(af_ctx* ctx, const void* hidden, const void* W,
                                  const int32_t* target, int64_t T, int32_t d, int32_t V,
                                  float* logp, float* entropy, float* lse, float* z, cudaStream_t s) {

@@ -462,7 +462,7 @@ __device__ __forceinline__ uint32_t ld_shared_cluster_u32(uint32_t cluster_addr)
 struct PairWork {
   int first, step, end, base_unit;     // units base_unit + first, base_unit + first + step, ... below base_unit + end
 };
-__device__ __forceinline__ PairWork pair_work(const GemmShape& g, int rank, int n_pairs) {
+__host__ __device__ __forceinline__ PairWork pair_work(const GemmShape& g, int rank, int n_pairs) {
   const int total = g.m_tiles * g.splits;
   const int n0 = g.die0_pairs, n1 = n_pairs - n0;
   if (n0 <= 0 || n1 <= 0) return PairWork{rank, n_pairs, total, 0};
