@@ -336,6 +336,32 @@ def test_die_aware_dealing_of_row_tiles(ctx):
         assert torch.equal(again, logp)              # the claimed ranks may differ between launches, the bits may not
 
 
+def test_the_plan_is_what_the_call_does(ctx):
+    """af_plan_token_logprob, fed with this part's SM count and measured die split, names the number
+    of vocabulary ranges the call itself picks: asking for exactly that number gives the same bits
+    (the ranges' partial statistics are merged in range order, so another number gives others),
+    and the workspace holds one partial per range and token."""
+    from paper_2507_01663_b200 import binding as B
+    dev = device()
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    die0 = max(ctx.die_split()[0], 0)
+    for T, d, V in [(40000, 64, 4096), (9000, 512, 8200)]:
+        H, W, y = random_case(T, d, V, seed=T + 1)
+        Hd, Wd, yd = H.to(dev), W.to(dev), y.to(dev)
+        plan = B.plan_token_logprob(T, d, V, sms, die0)
+        own, asked, other = (torch.empty(T, device=dev) for _ in range(3))
+        ctx.token_logprob(Hd, Wd, yd, own)
+        ctx.set_tuning(plan.v_splits, 0)
+        ctx.token_logprob(Hd, Wd, yd, asked)
+        ctx.set_tuning(plan.v_splits + 1, 0)
+        ctx.token_logprob(Hd, Wd, yd, other)
+        ctx.set_tuning(0, 0)
+        assert ctx.check_device_errors() == 0
+        assert torch.equal(own, asked)
+        assert not torch.equal(own, other)
+        assert (other - own).abs().max().item() <= LOGP_TOL
+
+
 def test_die_split_measured_at_creation(ctx):
     """The latency probe behind die-aware dealing: either a clean split of the SMs into two dies (even
     counts that add up to the SM count, neither die tiny) or a stated reason for having none."""
