@@ -411,8 +411,8 @@ af_status af_controller_clear(af_ctx* ctx, const af_controller_view* table, uint
  * (two writers of one row have no defined order), for n_cols outside [0, AF_MAX_WRITE_COLS], a
  * NULL column pointer while there are tokens to move, or a table whose n_samples differs from
  * N; AF_ERR_CAPACITY if the listed samples hold 2^31 tokens or more.  *T_out (host, nullable) receives the token count.  B == 0 is
- * valid and writes nothing.  Like af_pack_microbatch the call stages the list through pinned
- * host memory and cannot be recorded into a CUDA graph.
+ * valid and writes nothing.  The call stages its sequence table through pinned host memory (it may
+ * wait for the staging slot it reuses) and cannot be recorded into a CUDA graph.
  * ------------------------------------------------------------------------------------------- */
 #define AF_MAX_WRITE_COLS 4
 typedef struct {
